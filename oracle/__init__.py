@@ -1,0 +1,6 @@
+"""CPU oracle of the gate-and-route simulation.  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference legs may import this
+package.  It shares nothing with the CUDA library: its own C source, its own ctypes layouts.
+"""
+from .qsim_oracle import OracleSim, build_oracle, lib, run_oracle  # noqa: F401

@@ -1,0 +1,127 @@
+"""Plain-data description of one simulation instance.
+
+This module holds no simulation arithmetic.  It only fixes the names, enums and
+array shapes of the inputs that both the CPU oracle wrapper and the CUDA binding
+marshal into their own C structures, and the names of the statistics they return.
+
+Notation follows the paper: I classes, n = N GPUs, B decode cap per GPU, C prefill
+chunk size, (P_i, D_i) prompt/output lengths, lambda_i per-GPU arrival rates,
+theta_i patience rates, (c_p, c_d) token prices, x*_i / q*_p,i / y*_m,i / y*_s,i the
+steady-state LP targets, M the number of mixed GPUs.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field, replace
+from typing import Optional
+
+import numpy as np
+
+MAXI = 8          # max number of classes
+LMAX = 8192       # max token length; length tables hold LMAX-1 thresholds per (class, kind)
+NBIN = 1024       # bins of the log-linear latency histograms (32 octaves x 32 sub-bins)
+
+# prefill gate
+GATE_OCCUPANCY = 0   # occupancy-deviation gate (Section 4.1, "Upstream (prefill) gate")
+GATE_PRIORITY = 1    # largest D_i/P_i first (Section 5.1.1, Prioritize-and-Route)
+# decode router
+ROUTER_SOLO_FIRST = 0      # single FCFS buffer, solo GPUs first (Section 4.1, "Downstream routing")
+ROUTER_SLI = 1             # randomized split with p_s,i, two buffers (Section 5.2)
+# choice of GPU inside the eligible set
+PLACE_RANDOM = 0           # uniformly at random (paper)
+PLACE_LEAST_LOADED = 1     # fewest decodes, lowest index on ties
+# revenue that is reported as "the" revenue (both are always computed)
+PRICING_BUNDLED = 0        # Eq. (21)-(22)
+PRICING_SEPARATE = 1       # Eq. (23)
+# request lengths
+LENGTH_FIXED = 0           # every class-i request has (P_i, D_i)
+LENGTH_TABLE = 1           # integer lengths drawn through per-class threshold tables
+
+
+@dataclass
+class SimInputs:
+    """Everything a simulator needs; arrays are C-contiguous numpy arrays."""
+    name: str
+    I: int
+    N: int
+    R: int
+    B: int
+    C: int
+    nblk: int = 1
+    gate: int = GATE_OCCUPANCY
+    router: int = ROUTER_SOLO_FIRST
+    placement: int = PLACE_RANDOM
+    pricing: int = PRICING_BUNDLED
+    length_mode: int = LENGTH_FIXED
+    qcap: int = 4096            # capacity (entries) of each per-class prefill queue and of each decode buffer
+    hist: int = 0               # 1: record TTFT / TPOT histograms
+    seed: int = 0
+    rep_offset: int = 0         # global index of replication 0 (sharding across handles / GPUs)
+    block_len: float = 0.0      # seconds per block; ignored when nblk == 1
+    # per class
+    P: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint32))       # [I] fixed prompt length
+    D: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint32))       # [I] fixed output length
+    theta: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float64))  # [I] patience rate (1/s)
+    prio_rank: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint32))  # [I] 0 = served first
+    rates: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))         # [nblk, I] per-GPU lambda_i
+    lengths: Optional[np.ndarray] = None   # None or uint32 [I, 2, LMAX] thresholds (kind 0 = prompt, 1 = output)
+    prices: np.ndarray = field(default_factory=lambda: np.zeros(2))             # (c_p, c_d)
+    coeffs: np.ndarray = field(default_factory=lambda: np.zeros(6))             # alpha_m, beta, delta_m, alpha_s, delta_s, kappa
+    # LP targets per block
+    M: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint32))       # [nblk]
+    xstar: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))         # [nblk, I]   x*_i
+    n_xstar: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))       # [nblk, I]   n x*_i
+    n_qpstar: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))      # [nblk, I]   n q*_p,i
+    p_solo: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))        # [nblk, I]   p_s,i
+    # optional injected arrivals replacing the Poisson source (same list for every replication):
+    # times [K] ascending, and (class, P, D) [K, 3]
+    inject_t: Optional[np.ndarray] = None
+    inject_job: Optional[np.ndarray] = None
+    # free-form notes from the recipe (LP optimum, fluid capacity, class means ...); never read by a simulator
+    meta: dict = field(default_factory=dict)
+
+    def with_(self, **kw) -> "SimInputs":
+        return replace(self, **kw)
+
+    def validate(self) -> None:
+        I, nblk = self.I, self.nblk
+        assert 1 <= I <= MAXI and self.N >= 1 and self.R >= 1 and self.B >= 1 and self.C >= 1 and nblk >= 1
+        assert self.P.shape == (I,) and self.D.shape == (I,) and self.theta.shape == (I,)
+        assert self.prio_rank.shape == (I,)
+        assert self.rates.shape == (nblk, I)
+        assert self.prices.shape == (2,) and self.coeffs.shape == (6,)
+        assert self.M.shape == (nblk,)
+        for a in (self.xstar, self.n_xstar, self.n_qpstar, self.p_solo):
+            assert a.shape == (nblk, I)
+        if self.length_mode == LENGTH_TABLE:
+            assert self.lengths is not None and self.lengths.shape == (I, 2, LMAX)
+            assert self.lengths.dtype == np.uint32
+        if self.inject_t is not None:
+            K = self.inject_t.shape[0]
+            assert self.inject_t.dtype == np.float64 and self.inject_job.shape == (K, 3)
+            assert self.inject_job.dtype == np.uint32 and np.all(np.diff(self.inject_t) >= 0)
+
+
+# Names of the per-class integer counters every simulator returns (uint64 [R, I]).
+CLASS_COUNTERS = (
+    "arrivals",              # A_i
+    "admitted",              # U_p,i
+    "prefill_done",          # S_p,i
+    "placed_mixed",          # U_dm,i
+    "placed_solo",           # U_ds,i
+    "done_mixed",            # S_dm,i
+    "done_solo",             # S_ds,i
+    "abandoned_p",           # B_p,i
+    "abandoned_d",           # B_d,i
+    "overflow",              # arrivals dropped because the bounded prefill queue was full (0 in conforming runs)
+    "overflow_d",            # finished prefills dropped because the bounded decode buffer was full (0 likewise)
+    "tokens_in_prefilled",   # sum of P over completed prefills
+    "tokens_in_completed",   # sum of P over completed requests
+    "tokens_out_completed",  # sum of D over completed requests
+)
+# Per-class end-of-run state (uint32 [R, I]).
+CLASS_STATE = ("Qp", "X", "Qd", "Ym", "Ys")
+# Per-class fp64 accumulators (float64 [R, I]).
+CLASS_SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_tpot")
+# Per-replication scalars.
+REP_COUNTERS = ("iters_mixed", "iters_solo", "events")      # uint64 [R]
+REP_SUMS = ("busy_mixed", "busy_solo", "T_elapsed")          # float64 [R]
