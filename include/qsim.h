@@ -1,0 +1,187 @@
+/*
+ * qsim: many-replication simulation of a multiclass LLM-inference queueing network under the
+ * gate-and-route policy, on one NVIDIA B200 (sm_100a).  C ABI; no C++ or framework types cross it.
+ *
+ * Model (paper sections in brackets).  A replication is a cluster of n = N GPUs.  Each GPU holds at
+ * most one prefill and at most B decode streams; a prefill advances C tokens per iteration and every
+ * active decode emits one token per iteration [Sections 2.1-2.2].  An iteration whose batch holds p
+ * prefill tokens, d decodes and K resident KV tokens lasts
+ *     tau = (p > 0 ? alpha_m + beta p + delta_m d : alpha_s + delta_s d) + kappa K,
+ * which contains the paper's two regimes tau_mix(C) = alpha + beta C and tau_solo = c  [Eq. (1)-(3)]
+ * and its solo fit with a KV slope [Section 6.1].  Class-i requests arrive as a Poisson process of
+ * rate n lambda_i and wait with exponential patience theta_i in the prefill queue and in the decode
+ * buffer [Section 2.3, Eq. (7)-(9)].  GPUs 0..M-1 are mixed (they keep one slot for prefill, so at most
+ * B-1 decodes), GPUs M..N-1 are solo [Section 4.1, Static Planning].  The prefill gate admits the
+ * waiting class with the smallest occupancy deviation (X_i - n x*_i)/x*_i, ties to the largest
+ * Q_p,i - n q*_p,i [Section 4.1], or the class with the largest D_i/P_i [Section 5.1.1].  The decode
+ * router serves one FCFS buffer, solo GPUs first [Section 4.1], or splits jobs between a solo and a
+ * mixed buffer with probability p_s,i [Section 5.2].  Rates and targets are piecewise constant over
+ * blocks of block_len seconds and switch without pre-emption [Section 6.2].  Revenue is reported
+ * under bundled and separate charging [Eq. (21)-(23)] from integer token counters.
+ *
+ * Determinism.  Random numbers are Philox4x32-10 with key = seed and counter =
+ * (index, stream, replication); clocks are IEEE doubles, every operation rounded to nearest and never
+ * contracted to FMA.  Integer results do not depend on the launch shape or on how replications are
+ * split over handles (rep_offset).
+ *
+ * Pointers: every argument marked [host] is ordinary host memory owned by the caller and is copied
+ * before the call returns; [device] is device memory owned by the caller that must stay valid until
+ * qsim_destroy.  All functions return QSIM_OK (0) or a negative error; qsim_last_error() gives the
+ * calling thread's last message.  A handle must not be used from two threads at once.
+ */
+#ifndef QSIM_H
+#define QSIM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QSIM_MAXI 8       /* classes */
+#define QSIM_LMAX 8192    /* largest request length; stride of the length tables */
+#define QSIM_NBIN 1024    /* histogram bins: 32 per octave from 2^-20 s */
+
+enum {
+    QSIM_OK = 0,
+    QSIM_EINVAL = -1,      /* bad argument or unsupported size */
+    QSIM_ENOMEM = -2,      /* host or device allocation failed */
+    QSIM_EWORKSPACE = -3,  /* workspace missing, too small or misaligned */
+    QSIM_ECUDA = -4,       /* a CUDA call failed; the message names it */
+    QSIM_EOVERFLOW = -5,   /* a replication hit an internal bound (message names replication and bound) */
+    QSIM_ESTATE = -6       /* call out of order (run before bind, ...) */
+};
+
+enum { QSIM_GATE_OCCUPANCY = 0, QSIM_GATE_PRIORITY = 1 };
+enum { QSIM_ROUTER_SOLO_FIRST = 0, QSIM_ROUTER_SLI = 1 };
+enum { QSIM_PLACE_RANDOM = 0, QSIM_PLACE_LEAST_LOADED = 1 };
+enum { QSIM_PRICING_BUNDLED = 0, QSIM_PRICING_SEPARATE = 1 };
+enum { QSIM_LENGTH_FIXED = 0, QSIM_LENGTH_TABLE = 1 };
+
+typedef struct qsim qsim_t;
+
+typedef struct {
+    uint32_t size;         /* sizeof(qsim_config), checked */
+    uint32_t I, N, R;      /* classes (<= 8), GPUs per replication (<= 4096), replications of this handle */
+    uint32_t B, C;         /* decode cap per GPU (<= 4096), prefill chunk in tokens (<= 65535) */
+    uint32_t nblk;         /* number of rate/target blocks (>= 1) */
+    uint32_t gate, router, placement, pricing, length_mode;
+    uint32_t qcap;         /* capacity, in requests, of each per-class prefill queue and each decode buffer */
+    uint32_t hist;         /* 1: record TTFT / TPOT histograms */
+    uint64_t seed;
+    uint64_t rep_offset;   /* global index of this handle's replication 0 (sharding over handles / GPUs) */
+    double block_len;      /* seconds; ignored when nblk == 1 */
+} qsim_config;
+
+typedef struct {
+    uint32_t P, D;         /* prompt / output tokens of a class-i request when length_mode is FIXED (1..8192) */
+    uint32_t prio_rank;    /* priority gate: smaller rank is served first */
+    uint32_t reserved;
+    double theta;          /* patience rate theta_i >= 0 (1/s); 0 disables abandonment */
+} qsim_class;
+
+typedef struct {           /* policy parameters of one block, from the steady-state LP (Eq. (36), (38)) */
+    uint32_t M;            /* number of mixed GPUs, ceil(n sum_i x*_i) */
+    uint32_t reserved;
+    double xstar[QSIM_MAXI];     /* x*_i   (a class with x*_i = 0 is never admitted by the occupancy gate) */
+    double n_xstar[QSIM_MAXI];   /* n x*_i */
+    double n_qpstar[QSIM_MAXI];  /* n q*_p,i */
+    double p_solo[QSIM_MAXI];    /* p_s,i of the SLI-aware router */
+} qsim_targets;
+
+typedef struct {
+    /* cumulative counts since the last qsim_reset_stats: A, U_p, S_p, U_dm, U_ds, S_dm, S_ds, B_p, B_d */
+    uint64_t arrivals, admitted, prefill_done, placed_mixed, placed_solo, done_mixed, done_solo;
+    uint64_t abandoned_p, abandoned_d;
+    uint64_t overflow, overflow_d;       /* requests dropped at a full prefill queue / decode buffer (0 when qcap fits) */
+    uint64_t tokens_in_prefilled;        /* sum of P over finished prefills (separate charging credits c_p here) */
+    uint64_t tokens_in_completed;        /* sum of P over finished requests (bundled charging credits c_p here) */
+    uint64_t tokens_out_completed;       /* sum of D over finished requests */
+    uint32_t Qp, X, Qd, Ym, Ys, reserved;  /* state at the end of the run; Ym / Ys by the group of the GPU at placement */
+    double area_Qp, area_X, area_Qd, area_Ym, area_Ys;   /* time integrals of those counts */
+    double sum_ttft, sum_tpot;           /* sums over finished prefills / finished requests */
+} qsim_class_stats;
+
+typedef struct {
+    qsim_class_stats cls[QSIM_MAXI];
+    uint64_t iters_mixed, iters_solo;    /* finished iterations with / without a prefill chunk */
+    uint64_t events;                     /* arrivals + abandonments + block switches + iteration ends */
+    double busy_mixed, busy_solo;        /* total duration of those iterations */
+    double T_elapsed;                    /* simulated seconds since the last reset */
+} qsim_rep_stats;
+
+/*
+ * Create a handle [Sections 2.3, 4.1: primitives and policy parameters].  [host] cfg, classes[I],
+ * rates[nblk][I] (per-GPU lambda_i; the cluster rate is N lambda_i), lengths (NULL, or
+ * [I][2][QSIM_LMAX] non-decreasing thresholds: a uniform 32-bit word w maps to length
+ * 1 + #{j < QSIM_LMAX-1 : thr[j] <= w}; kind 0 = prompt, 1 = output), prices {c_p, c_d},
+ * iter_time_coeffs {alpha_m, beta, delta_m, alpha_s, delta_s, kappa}, lp_targets[nblk].
+ * Allocates a few hundred KB of device memory for the tables on the current device.
+ */
+int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                const uint32_t *lengths, const double *prices, const double *iter_time_coeffs,
+                const qsim_targets *lp_targets);
+
+/* Bytes of device memory qsim_bind needs for this handle (state of all R replications). */
+int qsim_workspace_bytes(const qsim_t *h, size_t *bytes);
+
+/*
+ * Give the handle its state memory: [device] workspace of at least qsim_workspace_bytes, 256-byte
+ * aligned; cuda_stream is a cudaStream_t (NULL = default stream) on which every later launch and copy
+ * of this handle is ordered.  Initialises all replications to the empty system at t = 0 (any converging
+ * initial state is admissible, Assumption 1).
+ */
+int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
+
+/*
+ * Advance every replication by horizon_iters * tau_ref simulated seconds, tau_ref = tau(0, B, 0) (one
+ * full solo iteration) [event-driven dynamics of Section 2.3 under the policies of Sections 4-5].
+ * Events with time <= the new end are processed.  Calls compose: run(a); run(b) leaves exactly the
+ * state of run(a + b).  qsim_stats / qsim_sync wait for completion.
+ */
+int qsim_run(qsim_t *h, uint64_t horizon_iters);
+
+/* Wait until all work queued on the handle's stream has finished; reports sticky replication errors. */
+int qsim_sync(qsim_t *h);
+
+/*
+ * Copy statistics [Eq. (15)-(23): cumulative flows, state, revenue counters] to [host] per_rep[R] (may
+ * be NULL), totals (sums over replications taken in replication order; may be NULL), hist_ttft /
+ * hist_tpot (uint64 [R][I][QSIM_NBIN]; may be NULL; zeros unless cfg.hist).  Bin of a latency x:
+ * clamp((bits(x) >> 47) - ((1023 - 20) << 5), 0, QSIM_NBIN - 1).  Synchronises the stream.
+ */
+int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint64_t *hist_ttft,
+               uint64_t *hist_tpot);
+
+/* Zero all counters, integrals and histograms and restart T_elapsed; the simulated state is kept. */
+int qsim_reset_stats(qsim_t *h);
+
+/* Revenue per GPU per second since the last reset from totals [Eq. (22), (23)]:
+ * (c_p tokens_in + c_d tokens_out) / (N sum_r T_elapsed). */
+int qsim_revenue(const qsim_t *h, const qsim_rep_stats *totals, double *bundled_rate, double *separate_rate);
+
+/* Per-GPU snapshot of replication r into [host] arrays of N entries (any may be NULL): decodes held,
+ * finished iterations, end of the running iteration (+inf when idle), prefill tokens left. */
+int qsim_server_state(qsim_t *h, uint32_t r, uint32_t *n_dec, uint32_t *it, double *t_next, uint32_t *pf_rem);
+
+/*
+ * One call from host buffers to host results: create, allocate the workspace with cudaMalloc, bind, run
+ * horizon_iters, copy statistics back, free everything.  Arguments as in qsim_create / qsim_stats.
+ */
+int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                  const uint32_t *lengths, const double *prices, const double *iter_time_coeffs,
+                  const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
+                  qsim_rep_stats *per_rep);
+
+/* Kernel launches issued by this handle so far (for accounting in benchmarks). */
+int qsim_launch_count(const qsim_t *h, uint64_t *launches);
+
+int qsim_destroy(qsim_t *h);
+
+const char *qsim_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,986 @@
+// Device side of qsim: one warp simulates one replication, event by event.
+//
+// Ownership inside the warp (no two lanes ever write the same word, so the only synchronisation is a
+// few __syncwarp per event):
+//   * lane i (< I) owns class i: its arrival clock, prefill queue cursor, abandonment clocks, counts,
+//     time integrals and statistics (struct ClassState, in shared memory);
+//   * lane l owns GPUs l, l+32, l+64, ...: their clocks and batch state (structure-of-arrays in shared
+//     memory, staged from / to global memory at kernel entry / exit);
+//   * scalars every lane needs (event time, block, buffer cursors, ordinals) are kept replicated in
+//     registers and updated identically by all lanes.
+// The next event is a warp-wide argmin over every lane's earliest source (three redux.sync on the bit
+// pattern of the positive doubles plus the source id, which encodes the tie order).  Decisions that look
+// at all GPUs (least-loaded / k-th eligible GPU) are evaluated by the owners and reduced the same way.
+//
+// All clock arithmetic is IEEE double, one rounding per operation, never contracted (the file is also
+// compiled with --fmad=false).
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace qsimdev {
+
+constexpr int MAXI = 8;
+constexpr int LMAX = 8192;
+constexpr int NBIN = 1024;
+constexpr unsigned FULL = 0xffffffffu;
+constexpr uint32_t NONE32 = 0xffffffffu;
+constexpr int TOUCH_CAP = 48;
+
+// source ids: smaller id wins an exact tie in time
+constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
+
+enum { STREAM_ARRIVAL = 0, STREAM_ABANDON_P = 1, STREAM_ABANDON_D0 = 2, STREAM_ABANDON_D1 = 3,
+       STREAM_PLACEMENT = 4, STREAM_SLI = 5 };
+enum { WANT_SOLO = 0, WANT_MIX = 1, WANT_PREFILL = 2 };
+enum { ERR_NONE = 0, ERR_INTERNAL = 1 };
+
+struct AbClock { double acc, lvl, t_last, t_ab; unsigned long long m; };
+struct Area { double area, t_last; };
+
+struct ClassState {
+    double ta;
+    unsigned long long adraw, sli_ord;
+    uint32_t ablk, nextP, nextD, pq_head, pq_n, X, Ym, Ys, Qd0, Qd1;
+    AbClock abp, abd0, abd1;
+    Area aQp, aX, aQd, aYm, aYs;
+    unsigned long long arrivals, admitted, prefill_done, placed_mixed, placed_solo, done_mixed, done_solo,
+        abandoned_p, abandoned_d, overflow, overflow_d, tok_in_pf, tok_in_done, tok_out_done;
+    double sum_ttft, sum_tpot;
+};
+
+struct RepHeader {
+    double T_end, T_reset;
+    unsigned long long place_ord, events;
+    uint32_t blk, done, err, pad;
+    uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
+    unsigned long long iters_mixed[32], iters_solo[32];
+    double busy_mixed[32], busy_solo[32];
+    ClassState cs[MAXI];
+};
+
+static_assert(sizeof(ClassState) % 8 == 0 && (sizeof(ClassState) * MAXI) % 16 == 0, "ClassState is copied in 16-byte words");
+static_assert(sizeof(RepHeader) % 16 == 0 && offsetof(RepHeader, cs) % 16 == 0, "RepHeader layout");
+
+struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
+
+struct ClassPar { double theta; uint32_t P, D, prio, pad; };
+struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI]; };
+
+struct Params {
+    uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance;
+    unsigned long long seed, rep_offset, horizon_iters, event_budget;
+    double block_len;
+    double coef[6];
+    ClassPar cls[MAXI];
+    const BlockPar *blocks;      // [nblk]
+    const uint32_t *lengths;     // [I][2][LMAX] or null
+    // workspace sections (all arrays are [R][...])
+    RepHeader *hdr;
+    char *srv;                   // per replication: server structure-of-arrays image, srv_bytes each
+    uint32_t *slot_fin;          // [R][N][B]
+    double *slot_tpf;            // [R][N][B]
+    uint32_t *slot_pk;           // [R][N][B]
+    QEntry *pq;                  // [R][I][qcap]
+    QEntry *dq;                  // [R][2][qcap]
+    uint32_t *hist_mem;          // [R][I][2][NBIN] or null
+    uint32_t *not_done;          // single counter: replications that stopped on the event budget
+    uint32_t srv_bytes;
+};
+
+// ---------------------------------------------------------------------------------------------
+// random numbers and elementary functions
+// ---------------------------------------------------------------------------------------------
+
+// Philox4x32-10 (Salmon et al., SC'11): counter (c0..c3), key (k0,k1).
+__device__ __forceinline__ void philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                       uint32_t &o0, uint32_t &o1, uint32_t &o2, uint32_t &o3)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    o0 = c0; o1 = c1; o2 = c2; o3 = c3;
+}
+
+__device__ __forceinline__ void draw(const Params &p, uint32_t rep, uint32_t stream, unsigned long long index,
+                                     uint32_t &w0, uint32_t &w1, uint32_t &w2, uint32_t &w3)
+{
+    const unsigned long long grep = p.rep_offset + rep;
+    philox((uint32_t)index, (uint32_t)(index >> 32), stream, (uint32_t)grep, (uint32_t)p.seed,
+           (uint32_t)(p.seed >> 32), w0, w1, w2, w3);
+}
+
+// uniform on (0,1]: (top 53 bits of w0:w1, plus one) / 2^53
+__device__ __forceinline__ double u53(uint32_t w0, uint32_t w1)
+{
+    const unsigned long long h = ((unsigned long long)w0 << 21) | (unsigned long long)(w1 >> 11);
+    return __dmul_rn((double)(h + 1ull), 1.1102230246251565e-16);   // 2^-53
+}
+
+// ln x for x in (0,1] as a fixed chain of rounded operations: x = m 2^e, m in [sqrt(1/2), sqrt(2)),
+// s = (m-1)/(m+1), ln m = 2 s sum_{k=0..12} s^(2k)/(2k+1), result = e ln2 + ln m.
+__device__ __forceinline__ double qlog(double x)
+{
+    const long long bits = __double_as_longlong(x);
+    int e = (int)((bits >> 52) & 0x7ff) - 1023;
+    double m = __longlong_as_double((bits & 0x000fffffffffffffLL) | 0x3ff0000000000000LL);
+    if (m > 1.4142135623730951) {
+        m = __dmul_rn(m, 0.5);
+        e += 1;
+    }
+    const double s = __ddiv_rn(__dsub_rn(m, 1.0), __dadd_rn(m, 1.0));
+    const double z = __dmul_rn(s, s);
+    double acc = __ddiv_rn(1.0, 25.0);
+#pragma unroll
+    for (int k = 11; k >= 0; --k)
+        acc = __dadd_rn(__dmul_rn(acc, z), __ddiv_rn(1.0, (double)(2 * k + 1)));
+    const double logm = __dmul_rn(__dmul_rn(2.0, s), acc);
+    return __dadd_rn(__dmul_rn((double)e, 0.6931471805599453), logm);
+}
+
+// iteration time of a batch with pf prefill tokens, d decodes, K resident KV tokens (Eq. (1)-(3))
+__device__ __forceinline__ double iter_time(const Params &p, uint32_t pf, uint32_t d, uint32_t K)
+{
+    double t;
+    if (pf > 0) {
+        t = __dadd_rn(p.coef[0], __dmul_rn(p.coef[1], (double)pf));
+        t = __dadd_rn(t, __dmul_rn(p.coef[2], (double)d));
+    } else {
+        t = __dadd_rn(p.coef[3], __dmul_rn(p.coef[4], (double)d));
+    }
+    if (p.coef[5] != 0.0)
+        t = __dadd_rn(t, __dmul_rn(p.coef[5], (double)K));
+    return t;
+}
+
+__device__ __forceinline__ uint32_t hist_bin(double x)
+{
+    long long b = (long long)((unsigned long long)__double_as_longlong(x) >> 47) - ((long long)(1023 - 20) << 5);
+    b = b < 0 ? 0 : (b > NBIN - 1 ? NBIN - 1 : b);
+    return (uint32_t)b;
+}
+
+// Cooperative table look-up: 1 + #{j < LMAX-1 : thr[j] <= w} in three 32-way probes (8192 = 32*32*8).
+__device__ __forceinline__ uint32_t table_length(const uint32_t *thr, uint32_t w, int lane)
+{
+    uint32_t idx = (uint32_t)lane * 256u + 255u;
+    bool ok = idx < LMAX - 1 && __ldg(thr + idx) <= w;
+    uint32_t base = (uint32_t)__popc(__ballot_sync(FULL, ok)) * 256u;
+    idx = base + (uint32_t)lane * 8u + 7u;
+    ok = idx < LMAX - 1 && __ldg(thr + idx) <= w;
+    base += (uint32_t)__popc(__ballot_sync(FULL, ok)) * 8u;
+    idx = base + (uint32_t)lane;
+    ok = lane < 8 && idx < LMAX - 1 && __ldg(thr + idx) <= w;
+    return 1u + base + (uint32_t)__popc(__ballot_sync(FULL, ok));
+}
+
+__device__ __forceinline__ uint32_t pack_job(uint32_t P, uint32_t D, uint32_t cls, uint32_t flag)
+{
+    return (P - 1u) | ((D - 1u) << 13) | (cls << 26) | (flag << 31);
+}
+__device__ __forceinline__ uint32_t job_P(uint32_t pk) { return (pk & 0x1fffu) + 1u; }
+__device__ __forceinline__ uint32_t job_D(uint32_t pk) { return ((pk >> 13) & 0x1fffu) + 1u; }
+__device__ __forceinline__ uint32_t job_cls(uint32_t pk) { return (pk >> 26) & 7u; }
+__device__ __forceinline__ uint32_t job_flag(uint32_t pk) { return pk >> 31; }
+
+__device__ __forceinline__ double dinf() { return __longlong_as_double(0x7ff0000000000000LL); }
+
+__device__ __forceinline__ void area_touch(Area &a, uint32_t count, double t)
+{
+    a.area = __dadd_rn(a.area, __dmul_rn((double)count, __dsub_rn(t, a.t_last)));
+    a.t_last = t;
+}
+
+// Abandonment clock of one (class, queue): integrated hazard acc against the exponential level lvl
+// (random time change, Eq. (8)-(9)); called by the owning class lane before the count changes.
+__device__ __forceinline__ void ab_change(AbClock &c, double theta, uint32_t Q_old, uint32_t Q_new, double t)
+{
+    if (!(theta > 0.0)) return;
+    c.acc = __dadd_rn(c.acc, __dmul_rn(__dmul_rn(theta, (double)Q_old), __dsub_rn(t, c.t_last)));
+    c.t_last = t;
+    if (Q_new > 0) {
+        double rem = __dsub_rn(c.lvl, c.acc);
+        if (rem < 0.0) rem = 0.0;
+        c.t_ab = __dadd_rn(t, __ddiv_rn(rem, __dmul_rn(theta, (double)Q_new)));
+    } else {
+        c.t_ab = dinf();
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// the per-warp simulator
+// ---------------------------------------------------------------------------------------------
+
+struct Sim {
+    const Params &p;
+    const int lane;
+    const uint32_t rep;
+    // shared memory (lane-owned entries)
+    double *tnext, *pf_tarr;
+    uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
+    uint16_t *ndec, *nact, *pfcur;
+    uint32_t *touch;
+    double *gate_xi, *gate_dq;
+    uint32_t *gate_ok;
+    ClassState *cs;
+    // global memory of this replication
+    uint32_t *s_fin;
+    double *s_tpf;
+    uint32_t *s_pk;
+    QEntry *pq, *dq;
+    uint32_t *hist;
+    // replicated scalars
+    double t, T_end, T_blk_next;
+    uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
+    unsigned long long place_ord, events;
+    bool drain_dirty, gate_dirty, touch_all;
+    // per-lane partial sums
+    unsigned long long it_mixed, it_solo;
+    double busy_mixed, busy_solo;
+    // block parameters of the current block (lane i holds class i)
+    double b_xstar, b_nx, b_nq, b_ps;
+
+    __device__ Sim(const Params &p_, int lane_, uint32_t rep_) : p(p_), lane(lane_), rep(rep_) {}
+
+    __device__ __forceinline__ double block_start(uint32_t b) const { return __dmul_rn((double)b, p.block_len); }
+
+    __device__ __forceinline__ void load_block(uint32_t b)
+    {
+        blk = b;
+        const BlockPar &bp = p.blocks[b];
+        M = bp.M;
+        b_xstar = 0.0; b_nx = 0.0; b_nq = 0.0; b_ps = 0.0;
+        if (lane < (int)p.I) {
+            b_xstar = bp.xstar[lane]; b_nx = bp.nx[lane]; b_nq = bp.nq[lane]; b_ps = bp.ps[lane];
+        }
+        T_blk_next = (b + 1 < p.nblk) ? block_start(b + 1) : dinf();
+    }
+
+    // --- arrivals ------------------------------------------------------------------------------
+    // Next class-i arrival after t0 (all lanes compute the same draw; lane i stores the result).
+    // A candidate at or past the end of its block is discarded and drawn again from the boundary under
+    // the next block's rate (memorylessness of the Poisson process).
+    __device__ void schedule_arrival(uint32_t i, double t0)
+    {
+        unsigned long long k = __shfl_sync(FULL, cs[lane & 7].adraw, i);
+        uint32_t b = __shfl_sync(FULL, cs[lane & 7].ablk, i);
+        double ta = dinf();
+        uint32_t nP = p.cls[i].P, nD = p.cls[i].D;
+        for (;;) {
+            const double Lam = __dmul_rn((double)p.N, p.blocks[b].rate[i]);
+            const bool has_next = b + 1 < p.nblk;
+            if (!(Lam > 0.0)) {
+                if (!has_next) break;
+                ++b; t0 = block_start(b);
+                continue;
+            }
+            uint32_t w0, w1, w2, w3;
+            draw(p, rep, (STREAM_ARRIVAL << 8) | i, k++, w0, w1, w2, w3);
+            const double E = -qlog(u53(w0, w1));
+            const double cand = __dadd_rn(t0, __ddiv_rn(E, Lam));
+            if (has_next && cand >= block_start(b + 1)) {
+                ++b; t0 = block_start(b);
+                continue;
+            }
+            ta = cand;
+            if (p.length_mode == 1) {
+                nP = table_length(p.lengths + ((size_t)i * 2 + 0) * LMAX, w2, lane);
+                nD = table_length(p.lengths + ((size_t)i * 2 + 1) * LMAX, w3, lane);
+            }
+            break;
+        }
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            c.ta = ta; c.adraw = k; c.ablk = b; c.nextP = nP; c.nextD = nD;
+        }
+    }
+
+    __device__ void on_arrival(uint32_t i)
+    {
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            c.arrivals++;
+            if (c.pq_n >= p.qcap) {
+                c.overflow++;
+            } else {
+                ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n + 1, t);
+                area_touch(c.aQp, c.pq_n, t);
+                uint32_t pos = c.pq_head + c.pq_n;
+                if (pos >= p.qcap) pos -= p.qcap;
+                QEntry e; e.t = t; e.pk = pack_job(c.nextP, c.nextD, i, 0); e.cls = i;
+                pq[(size_t)i * p.qcap + pos] = e;
+                c.pq_n++;
+            }
+        }
+        schedule_arrival(i, t);
+        gate_dirty = true;
+    }
+
+    // --- abandonment ---------------------------------------------------------------------------
+    // Remove entry `pos` (offset from head) of a ring of n entries, keeping order: shift the tail down.
+    __device__ void ring_remove(QEntry *ring, uint32_t head, uint32_t n, uint32_t pos)
+    {
+        const uint32_t cap = p.qcap;
+        for (uint32_t k = pos; k + 1 < n; k += 32) {
+            const uint32_t j = k + (uint32_t)lane;
+            QEntry e;
+            const bool act = j + 1 < n;
+            if (act) {
+                uint32_t src = head + j + 1; if (src >= cap) src -= cap;
+                e = ring[src];
+            }
+            __syncwarp();
+            if (act) {
+                uint32_t dst = head + j; if (dst >= cap) dst -= cap;
+                ring[dst] = e;
+            }
+            __syncwarp();
+        }
+    }
+
+    __device__ void on_abandon_p(uint32_t i)
+    {
+        const uint32_t Q = __shfl_sync(FULL, cs[lane & 7].pq_n, i);
+        const uint32_t head = __shfl_sync(FULL, cs[lane & 7].pq_head, i);
+        const unsigned long long m = __shfl_sync(FULL, cs[lane & 7].abp.m, i);
+        uint32_t w0, w1, w2, w3;
+        draw(p, rep, (STREAM_ABANDON_P << 8) | i, m, w0, w1, w2, w3);
+        const uint32_t rank = __umulhi(w2, Q);       // uniformly chosen waiting job, in FCFS rank
+        ring_remove(pq + (size_t)i * p.qcap, head, Q, rank);
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            area_touch(c.aQp, Q, t);
+            c.pq_n = Q - 1;
+            c.abandoned_p++;
+            AbClock &a = c.abp;
+            a.m = m + 1; a.acc = 0.0; a.lvl = -qlog(u53(w0, w1)); a.t_last = t;
+            a.t_ab = (Q - 1 > 0) ? __dadd_rn(t, __ddiv_rn(a.lvl, __dmul_rn(p.cls[i].theta, (double)(Q - 1)))) : dinf();
+        }
+    }
+
+    __device__ void on_abandon_d(uint32_t pool, uint32_t i)
+    {
+        const uint32_t Q = __shfl_sync(FULL, pool ? cs[lane & 7].Qd1 : cs[lane & 7].Qd0, i);
+        const unsigned long long m = __shfl_sync(FULL, pool ? cs[lane & 7].abd1.m : cs[lane & 7].abd0.m, i);
+        uint32_t w0, w1, w2, w3;
+        draw(p, rep, ((pool ? STREAM_ABANDON_D1 : STREAM_ABANDON_D0) << 8) | i, m, w0, w1, w2, w3);
+        uint32_t rank = __umulhi(w2, Q);
+        QEntry *ring = dq + (size_t)pool * p.qcap;
+        const uint32_t head = pool ? dq_head1 : dq_head0, n = pool ? dq_n1 : dq_n0;
+        // position of the rank-th class-i entry in buffer order
+        uint32_t pos = NONE32;
+        for (uint32_t k = 0; k < n && pos == NONE32; k += 32) {
+            const uint32_t j = k + (uint32_t)lane;
+            bool mine = false;
+            if (j < n) {
+                uint32_t src = head + j; if (src >= p.qcap) src -= p.qcap;
+                mine = ring[src].cls == i;
+            }
+            const uint32_t b = __ballot_sync(FULL, mine);
+            const uint32_t c = (uint32_t)__popc(b);
+            if (rank < c) pos = k + (uint32_t)__fns(b, 0, (int)rank + 1);
+            else rank -= c;
+        }
+        if (pos == NONE32) { err = ERR_INTERNAL; return; }
+        ring_remove(ring, head, n, pos);
+        if (pool) dq_n1--; else dq_n0--;
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            area_touch(c.aQd, c.Qd0 + c.Qd1, t);
+            if (pool) c.Qd1 = Q - 1; else c.Qd0 = Q - 1;
+            c.abandoned_d++;
+            AbClock &a = pool ? c.abd1 : c.abd0;
+            a.m = m + 1; a.acc = 0.0; a.lvl = -qlog(u53(w0, w1)); a.t_last = t;
+            a.t_ab = (Q - 1 > 0) ? __dadd_rn(t, __ddiv_rn(a.lvl, __dmul_rn(p.cls[i].theta, (double)(Q - 1)))) : dinf();
+        }
+    }
+
+    // --- GPU choice ----------------------------------------------------------------------------
+    __device__ __forceinline__ bool eligible(uint32_t g, int want) const
+    {
+        if (g >= p.N) return false;
+        const uint32_t nd = ndec[g];
+        const bool pf = (pfjob[g] >> 31) != 0;
+        const uint32_t cap = (g < M || pf) ? p.B - 1 : p.B;   // a mixed GPU keeps one slot for prefill
+        if (want == WANT_SOLO) return g >= M && nd < cap;
+        if (want == WANT_MIX) return g < M && nd < cap;
+        return g < M && !pf && nd <= p.B - 1;
+    }
+
+    // uniformly at random among the eligible GPUs (k-th in index order) or least loaded, lowest index
+    __device__ uint32_t choose_server(int want)
+    {
+        const uint32_t rows = p.Npad >> 5;
+        if (p.placement == 1) {
+            uint32_t best = NONE32;
+            for (uint32_t k = 0; k < rows; ++k) {
+                const uint32_t g = (k << 5) + (uint32_t)lane;
+                if (eligible(g, want)) best = min(best, ((uint32_t)ndec[g] << 16) | g);
+            }
+            best = __reduce_min_sync(FULL, best);
+            return best == NONE32 ? NONE32 : (best & 0xffffu);
+        }
+        uint32_t cnt = 0;
+        for (uint32_t k = 0; k < rows; ++k)
+            cnt += (uint32_t)__popc(__ballot_sync(FULL, eligible((k << 5) + (uint32_t)lane, want)));
+        if (cnt == 0) return NONE32;
+        uint32_t idx = 0;
+        if (cnt > 1) {
+            uint32_t w0, w1, w2, w3;
+            draw(p, rep, STREAM_PLACEMENT << 8, place_ord++, w0, w1, w2, w3);
+            idx = __umulhi(w0, cnt);
+        }
+        for (uint32_t k = 0; k < rows; ++k) {
+            const uint32_t b = __ballot_sync(FULL, eligible((k << 5) + (uint32_t)lane, want));
+            const uint32_t c = (uint32_t)__popc(b);
+            if (idx < c) return (k << 5) + (uint32_t)__fns(b, 0, (int)idx + 1);
+            idx -= c;
+        }
+        err = ERR_INTERNAL;
+        return NONE32;
+    }
+
+    __device__ __forceinline__ void touch_server(uint32_t g)
+    {
+        if (n_touch < TOUCH_CAP) { if (lane == 0) touch[n_touch] = g; n_touch++; }
+        else touch_all = true;
+    }
+
+    // --- decode placement ------------------------------------------------------------------------
+    __device__ void place_decode(uint32_t pool, uint32_t g)
+    {
+        const uint32_t head = pool ? dq_head1 : dq_head0;
+        const QEntry e = dq[(size_t)pool * p.qcap + head];
+        const uint32_t i = e.cls, P = job_P(e.pk), D = job_D(e.pk);
+        if (pool) { dq_head1 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n1--; }
+        else      { dq_head0 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n0--; }
+        const bool mixed = g < M;
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
+            ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd - 1, t);
+            area_touch(c.aQd, c.Qd0 + c.Qd1, t);
+            if (pool) c.Qd1--; else c.Qd0--;
+            if (mixed) { area_touch(c.aYm, c.Ym, t); c.Ym++; c.placed_mixed++; }
+            else       { area_touch(c.aYs, c.Ys, t); c.Ys++; c.placed_solo++; }
+        }
+        if (lane == (int)(g & 31u)) {
+            const uint32_t sl = ndec[g];
+            const bool running = tnext[g] < dinf();
+            // joins the iteration that starts next: a running iteration first finishes as it+1
+            const uint32_t fin = it[g] + (running ? 1u : 0u) + D;
+            const size_t o = (size_t)g * p.B + sl;
+            s_fin[o] = fin;
+            s_tpf[o] = e.t;
+            s_pk[o] = pack_job(P, D, i, mixed ? 1u : 0u);
+            ndec[g] = (uint16_t)(sl + 1);
+            nfin[g] = min(nfin[g], fin);
+            Kpend[g] += P;
+        }
+        touch_server(g);
+    }
+
+    // --- prefill gate ------------------------------------------------------------------------------
+    __device__ uint32_t gate_class()
+    {
+        if (p.gate == 1) {
+            // Prioritize-and-Route: largest D_i/P_i among waiting classes = smallest static rank
+            uint32_t key = NONE32;
+            if (lane < (int)p.I && cs[lane].pq_n > 0) key = (p.cls[lane].prio << 8) | (uint32_t)lane;
+            key = __reduce_min_sync(FULL, key);
+            return key == NONE32 ? NONE32 : (key & 0xffu);
+        }
+        if (lane < (int)p.I) {
+            const ClassState &c = cs[lane];
+            gate_ok[lane] = (c.pq_n > 0 && b_xstar > 0.0) ? 1u : 0u;
+            gate_xi[lane] = __ddiv_rn(__dsub_rn((double)c.X, b_nx), b_xstar);   // xi_i = (X_i - n x*_i)/x*_i
+            gate_dq[lane] = __dsub_rn((double)c.pq_n, b_nq);                     // Q_p,i - n q*_p,i
+        }
+        __syncwarp();
+        uint32_t best = NONE32;
+        double bxi = 0.0, bdq = 0.0;
+        for (uint32_t i = 0; i < p.I; ++i) {
+            if (!gate_ok[i]) continue;
+            const double xi = gate_xi[i], dqv = gate_dq[i];
+            if (best == NONE32 || xi < bxi || (xi == bxi && dqv > bdq)) { best = i; bxi = xi; bdq = dqv; }
+        }
+        __syncwarp();
+        return best;
+    }
+
+    __device__ void admit(uint32_t i, uint32_t g)
+    {
+        const uint32_t head = __shfl_sync(FULL, cs[lane & 7].pq_head, i);
+        const QEntry e = pq[(size_t)i * p.qcap + head];
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n - 1, t);
+            area_touch(c.aQp, c.pq_n, t);
+            c.pq_n--;
+            c.pq_head = (head + 1 == p.qcap) ? 0 : head + 1;
+            area_touch(c.aX, c.X, t);
+            c.X++;
+            c.admitted++;
+        }
+        if (lane == (int)(g & 31u)) {
+            pfjob[g] = e.pk | 0x80000000u;
+            pfrem[g] = job_P(e.pk);
+            pf_tarr[g] = e.t;
+        }
+        touch_server(g);
+    }
+
+    __device__ __forceinline__ void start_if_needed(uint32_t g)
+    {
+        // called by the owner: a GPU with work that is between iterations starts one now;
+        // the batch (prefill chunk, decodes) is frozen here for the whole iteration
+        if (!(tnext[g] < dinf())) {
+            const uint32_t nd = ndec[g];
+            const uint32_t pj = pfjob[g];
+            if (nd > 0 || (pj >> 31)) {
+                const uint32_t Kg = K[g] + Kpend[g];
+                K[g] = Kg; Kpend[g] = 0;
+                nact[g] = (uint16_t)nd;
+                const uint32_t pc = (pj >> 31) ? min(p.C, pfrem[g]) : 0u;
+                pfcur[g] = (uint16_t)pc;
+                tnext[g] = __dadd_rn(t, iter_time(p, pc, nd, Kg));
+            }
+        }
+    }
+
+    __device__ void dispatch()
+    {
+        __syncwarp();   // queue entries and GPU state written by the event handler are visible to every lane
+        // decode routing: buffered jobs first (FCFS), solo GPUs before mixed ones
+        if (drain_dirty && (dq_n0 | dq_n1)) {
+            if (p.router == 0) {
+                while (dq_n0 > 0) {
+                    uint32_t g = choose_server(WANT_SOLO);
+                    if (g == NONE32) g = choose_server(WANT_MIX);
+                    if (g == NONE32) break;
+                    place_decode(0, g);
+                    __syncwarp();
+                }
+            } else {
+                while (dq_n0 > 0) {
+                    const uint32_t g = choose_server(WANT_SOLO);
+                    if (g == NONE32) break;
+                    place_decode(0, g);
+                    __syncwarp();
+                }
+                while (dq_n1 > 0) {
+                    const uint32_t g = choose_server(WANT_MIX);
+                    if (g == NONE32) break;
+                    place_decode(1, g);
+                    __syncwarp();
+                }
+            }
+        }
+        drain_dirty = false;
+        // prefill gate on mixed GPUs whose prefill slot is idle
+        if (gate_dirty) {
+            for (;;) {
+                const uint32_t i = gate_class();
+                if (i == NONE32) break;
+                const uint32_t g = choose_server(WANT_PREFILL);
+                if (g == NONE32) break;
+                admit(i, g);
+                __syncwarp();
+            }
+        }
+        gate_dirty = false;
+        // start the next iteration on every GPU that was touched and is between iterations
+        __syncwarp();
+        if (touch_all) {
+            for (uint32_t k = 0; k < (p.Npad >> 5); ++k) {
+                const uint32_t g = (k << 5) + (uint32_t)lane;
+                if (g < p.N) start_if_needed(g);
+            }
+        } else {
+            for (uint32_t k = 0; k < n_touch; ++k) {
+                const uint32_t g = touch[k];
+                if (lane == (int)(g & 31u)) start_if_needed(g);
+            }
+        }
+        n_touch = 0;
+        touch_all = false;
+    }
+
+    // --- end of an iteration on GPU g ------------------------------------------------------------
+    __device__ void on_server(uint32_t g)
+    {
+        const int owner = (int)(g & 31u);
+        uint32_t flags = 0, itg = 0, nd = 0;
+        if (lane == owner) {
+            itg = it[g] + 1;
+            it[g] = itg;
+            const uint32_t na = nact[g], pc = pfcur[g], Kg = K[g];
+            const double tau = iter_time(p, pc, na, Kg);
+            if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
+            else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
+            K[g] = Kg + na;
+            tnext[g] = dinf();
+            nd = ndec[g];
+            if (nfin[g] == itg) flags |= 1u;
+            if (pc > 0) {
+                const uint32_t rem = pfrem[g] - pc;
+                pfrem[g] = rem;
+                if (rem == 0) flags |= 2u;
+            }
+            pfcur[g] = 0;
+        }
+        flags = __shfl_sync(FULL, flags, owner);
+        if (flags & 1u) {
+            // some decode emitted its last token: scan the GPU's slot list from the tail, close the gaps
+            itg = __shfl_sync(FULL, itg, owner);
+            nd = __shfl_sync(FULL, nd, owner);
+            uint32_t n = nd, newmin = NONE32, Kdrop = 0;
+            const size_t base = (size_t)g * p.B;
+            for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
+                const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
+                const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
+                const bool hit = f == itg;
+                if (!hit) newmin = min(newmin, f);
+                uint32_t hits = __ballot_sync(FULL, hit);
+                while (hits) {
+                    const int hl = 31 - __clz(hits);
+                    hits &= ~(1u << hl);
+                    const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
+                    const double tpf = s_tpf[base + h];
+                    const uint32_t pk = s_pk[base + h];
+                    const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
+                    if (lane == (int)i) {
+                        ClassState &c = cs[i];
+                        if (job_flag(pk)) { area_touch(c.aYm, c.Ym, t); c.Ym--; c.done_mixed++; }
+                        else              { area_touch(c.aYs, c.Ys, t); c.Ys--; c.done_solo++; }
+                        c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
+                        c.tok_out_done += D;
+                        const double tpot = __ddiv_rn(__dsub_rn(t, tpf), (double)D);
+                        c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
+                        if (hist) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
+                    }
+                    Kdrop += P + D;
+                    const uint32_t last = n - 1;
+                    __syncwarp();
+                    if (lane == 0 && h != last) {
+                        s_fin[base + h] = s_fin[base + last];
+                        s_tpf[base + h] = s_tpf[base + last];
+                        s_pk[base + h] = s_pk[base + last];
+                    }
+                    n = last;
+                }
+            }
+            newmin = __reduce_min_sync(FULL, newmin);
+            if (lane == owner) {
+                ndec[g] = (uint16_t)n;
+                nfin[g] = newmin;
+                K[g] -= Kdrop;
+            }
+            drain_dirty = true;
+            gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
+        }
+        if (flags & 2u) {
+            // prefill finished: account, then hand the request to the decode stage
+            const uint32_t pk = pfjob[g];
+            const double tarr = pf_tarr[g];
+            const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
+            uint32_t pool = 0;
+            if (p.router == 1) {
+                // SLI-aware router: one uniform per finished prefill decides the pool
+                const unsigned long long ord = __shfl_sync(FULL, cs[lane & 7].sli_ord, i);
+                const double ps = __shfl_sync(FULL, b_ps, i);
+                uint32_t w0, w1, w2, w3;
+                draw(p, rep, (STREAM_SLI << 8) | i, ord, w0, w1, w2, w3);
+                pool = (u53(w0, w1) <= ps) ? 0u : 1u;
+            }
+            const uint32_t n = pool ? dq_n1 : dq_n0;
+            const bool full = n >= p.qcap;
+            if (lane == (int)i) {
+                ClassState &c = cs[i];
+                area_touch(c.aX, c.X, t);
+                c.X--;
+                c.prefill_done++;
+                c.tok_in_pf += P;                  // separate charging credits the prompt here, Eq. (23)
+                const double ttft = __dsub_rn(t, tarr);
+                c.sum_ttft = __dadd_rn(c.sum_ttft, ttft);
+                if (hist) hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)]++;
+                if (p.router == 1) c.sli_ord++;
+                if (full) {
+                    c.overflow_d++;
+                } else {
+                    const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
+                    ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd + 1, t);
+                    area_touch(c.aQd, c.Qd0 + c.Qd1, t);
+                    if (pool) c.Qd1++; else c.Qd0++;
+                }
+            }
+            if (!full) {
+                uint32_t pos = (pool ? dq_head1 : dq_head0) + n;
+                if (pos >= p.qcap) pos -= p.qcap;
+                if (lane == 0) {
+                    QEntry e; e.t = t; e.pk = pack_job(P, D, i, 0); e.cls = i;
+                    dq[(size_t)pool * p.qcap + pos] = e;
+                }
+                if (pool) dq_n1++; else dq_n0++;
+            }
+            __syncwarp();   // every lane has read the finished job before its owner clears it
+            if (lane == owner) pfjob[g] = 0;
+            drain_dirty = true;
+            gate_dirty = true;
+        }
+        touch_server(g);
+    }
+
+    // --- event loop ----------------------------------------------------------------------------------
+    __device__ bool run()
+    {
+        const uint32_t rows = p.Npad >> 5;
+        unsigned long long budget = p.event_budget;
+        for (;;) {
+            __syncwarp();
+            // earliest source of this lane; scanning in id order with '<' keeps the tie order
+            unsigned long long bt = 0x7ff0000000000000ull;
+            uint32_t bs = NONE32;
+            if (lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
+            if (lane < (int)p.I) {
+                const ClassState &c = cs[lane];
+                unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
+                if (v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
+                v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
+                if (v < bt) { bt = v; bs = SRC_ABP + lane; }
+                v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
+                if (v < bt) { bt = v; bs = SRC_ABD0 + lane; }
+                v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
+                if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
+            }
+            for (uint32_t k = 0; k < rows; ++k) {
+                const uint32_t g = (k << 5) + (uint32_t)lane;
+                const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+                if (v < bt) { bt = v; bs = SRC_SERVER + g; }
+            }
+            // warp argmin of (time bits, source id)
+            const uint32_t hi = (uint32_t)(bt >> 32), lo = (uint32_t)bt;
+            const uint32_t mhi = __reduce_min_sync(FULL, hi);
+            const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : NONE32);
+            const uint32_t src = __reduce_min_sync(FULL, (hi == mhi && lo == mlo) ? bs : NONE32);
+            const double te = __longlong_as_double((long long)(((unsigned long long)mhi << 32) | mlo));
+            if (src == NONE32 || te > T_end) return true;
+            if (budget == 0) return false;
+            --budget;
+            ++events;
+            t = te;
+            if (src >= SRC_SERVER) {
+                on_server(src - SRC_SERVER);
+            } else if (src >= SRC_ABD1) {
+                on_abandon_d(1, src - SRC_ABD1);
+            } else if (src >= SRC_ABD0) {
+                on_abandon_d(0, src - SRC_ABD0);
+            } else if (src >= SRC_ABP) {
+                on_abandon_p(src - SRC_ABP);
+            } else if (src >= SRC_ARRIVAL) {
+                on_arrival(src - SRC_ARRIVAL);
+            } else {
+                load_block(blk + 1);
+                drain_dirty = true;
+                gate_dirty = true;
+            }
+            if (err) return true;
+            dispatch();
+        }
+    }
+};
+
+// shared-memory carve-up for one replication (one warp per block)
+struct SmemLayout {
+    uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
+        off_pfcur, srv_bytes, off_touch, off_gate, off_cs, total;
+};
+
+__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
+{
+    SmemLayout L;
+    uint32_t o = 0;
+    L.off_tnext = o; o += 8 * Npad;
+    L.off_tarr = o; o += 8 * Npad;
+    L.off_it = o; o += 4 * Npad;
+    L.off_nfin = o; o += 4 * Npad;
+    L.off_pfrem = o; o += 4 * Npad;
+    L.off_pfjob = o; o += 4 * Npad;
+    L.off_K = o; o += 4 * Npad;
+    L.off_Kpend = o; o += 4 * Npad;
+    L.off_ndec = o; o += 2 * Npad;
+    L.off_nact = o; o += 2 * Npad;
+    L.off_pfcur = o; o += 2 * Npad;
+    o = (o + 15u) & ~15u;
+    L.srv_bytes = o;
+    L.off_touch = o; o += 4 * TOUCH_CAP;
+    o = (o + 7u) & ~7u;
+    L.off_gate = o; o += (8 + 8 + 4) * MAXI;
+    o = (o + 15u) & ~15u;
+    L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
+    L.total = (o + 15u) & ~15u;
+    return L;
+}
+
+__device__ __forceinline__ void bind_pointers(Sim &s, char *sm, const SmemLayout &L)
+{
+    s.tnext = reinterpret_cast<double *>(sm + L.off_tnext);
+    s.pf_tarr = reinterpret_cast<double *>(sm + L.off_tarr);
+    s.it = reinterpret_cast<uint32_t *>(sm + L.off_it);
+    s.nfin = reinterpret_cast<uint32_t *>(sm + L.off_nfin);
+    s.pfrem = reinterpret_cast<uint32_t *>(sm + L.off_pfrem);
+    s.pfjob = reinterpret_cast<uint32_t *>(sm + L.off_pfjob);
+    s.K = reinterpret_cast<uint32_t *>(sm + L.off_K);
+    s.Kpend = reinterpret_cast<uint32_t *>(sm + L.off_Kpend);
+    s.ndec = reinterpret_cast<uint16_t *>(sm + L.off_ndec);
+    s.nact = reinterpret_cast<uint16_t *>(sm + L.off_nact);
+    s.pfcur = reinterpret_cast<uint16_t *>(sm + L.off_pfcur);
+    s.touch = reinterpret_cast<uint32_t *>(sm + L.off_touch);
+    s.gate_xi = reinterpret_cast<double *>(sm + L.off_gate);
+    s.gate_dq = s.gate_xi + MAXI;
+    s.gate_ok = reinterpret_cast<uint32_t *>(s.gate_dq + MAXI);
+    s.cs = reinterpret_cast<ClassState *>(sm + L.off_cs);
+    const Params &p = s.p;
+    const size_t r = s.rep;
+    s.s_fin = p.slot_fin + r * (size_t)p.N * p.B;
+    s.s_tpf = p.slot_tpf + r * (size_t)p.N * p.B;
+    s.s_pk = p.slot_pk + r * (size_t)p.N * p.B;
+    s.pq = p.pq + r * (size_t)p.I * p.qcap;
+    s.dq = p.dq + r * (size_t)2 * p.qcap;
+    s.hist = p.hist_mem ? p.hist_mem + r * (size_t)p.I * 2 * NBIN : nullptr;
+}
+
+// Empty system at t = 0: idle GPUs, first arrival of every class scheduled, abandonment levels drawn.
+__global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
+{
+    extern __shared__ __align__(16) char sm[];
+    const int lane = threadIdx.x;
+    for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
+        const SmemLayout L = smem_layout(p.Npad);
+        Sim s(p, lane, rep);
+        bind_pointers(s, sm, L);
+        __syncwarp();
+        for (uint32_t o = lane * 4; o < L.total; o += 128) *reinterpret_cast<uint32_t *>(sm + o) = 0;
+        __syncwarp();
+        for (uint32_t g = lane; g < p.Npad; g += 32) { s.tnext[g] = dinf(); s.nfin[g] = NONE32; }
+        if (lane < MAXI) {
+            ClassState &c = s.cs[lane];
+            c.ta = dinf();
+            AbClock *clk[3] = { &c.abp, &c.abd0, &c.abd1 };
+            const uint32_t streams[3] = { STREAM_ABANDON_P, STREAM_ABANDON_D0, STREAM_ABANDON_D1 };
+            for (int k = 0; k < 3; ++k) {
+                uint32_t w0, w1, w2, w3;
+                draw(p, rep, (streams[k] << 8) | (uint32_t)lane, 0, w0, w1, w2, w3);
+                clk[k]->acc = 0.0; clk[k]->lvl = -qlog(u53(w0, w1)); clk[k]->t_last = 0.0; clk[k]->t_ab = dinf();
+                clk[k]->m = 1;
+            }
+        }
+        __syncwarp();
+        for (uint32_t i = 0; i < p.I; ++i) { s.schedule_arrival(i, 0.0); __syncwarp(); }
+        // write everything out
+        RepHeader &h = p.hdr[rep];
+        for (uint32_t o = lane * 4; o < sizeof(RepHeader); o += 128)
+            *reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(&h) + o) = 0;
+        __syncwarp();
+        if (lane < MAXI) h.cs[lane] = s.cs[lane];
+        char *img = p.srv + (size_t)rep * p.srv_bytes;
+        for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
+            *reinterpret_cast<uint4 *>(img + o) = *reinterpret_cast<const uint4 *>(sm + o);
+        if (p.hist_mem)
+            for (uint32_t o = lane; o < p.I * 2 * NBIN; o += 32) s.hist[o] = 0;
+        __syncwarp();
+    }
+}
+
+// Advance replications to their new end time (or until the per-launch event budget runs out).
+__global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
+{
+    extern __shared__ __align__(16) char sm[];
+    const int lane = threadIdx.x;
+    for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
+        RepHeader &h = p.hdr[rep];
+        if (!p.advance && h.done) continue;
+        const SmemLayout L = smem_layout(p.Npad);
+        Sim s(p, lane, rep);
+        bind_pointers(s, sm, L);
+        __syncwarp();
+        // stage state: server arrays (coalesced 16-byte copies) and the class records
+        const char *img = p.srv + (size_t)rep * p.srv_bytes;
+        for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
+            *reinterpret_cast<uint4 *>(sm + o) = *reinterpret_cast<const uint4 *>(img + o);
+        {
+            const uint4 *src = reinterpret_cast<const uint4 *>(h.cs);
+            uint4 *dst = reinterpret_cast<uint4 *>(s.cs);
+            for (uint32_t o = lane; o < sizeof(ClassState) * MAXI / 16; o += 32) dst[o] = src[o];
+        }
+        __syncwarp();
+        double T_end = h.T_end;
+        if (p.advance) T_end = __dadd_rn(T_end, __dmul_rn((double)p.horizon_iters, iter_time(p, 0, p.B, 0)));
+        s.T_end = T_end;
+        s.t = 0.0;
+        s.load_block(h.blk);
+        s.dq_head0 = h.dq_head0; s.dq_head1 = h.dq_head1; s.dq_n0 = h.dq_n0; s.dq_n1 = h.dq_n1;
+        s.place_ord = h.place_ord; s.events = h.events;
+        s.n_touch = 0; s.touch_all = false; s.err = h.err;
+        s.drain_dirty = true; s.gate_dirty = true;
+        s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
+        s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
+        const bool finished = s.err ? true : s.run();
+        __syncwarp();
+        // stage back
+        char *out = p.srv + (size_t)rep * p.srv_bytes;
+        for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
+            *reinterpret_cast<uint4 *>(out + o) = *reinterpret_cast<const uint4 *>(sm + o);
+        {
+            uint4 *dst = reinterpret_cast<uint4 *>(h.cs);
+            const uint4 *src = reinterpret_cast<const uint4 *>(s.cs);
+            for (uint32_t o = lane; o < sizeof(ClassState) * MAXI / 16; o += 32) dst[o] = src[o];
+        }
+        h.iters_mixed[lane] = s.it_mixed; h.iters_solo[lane] = s.it_solo;
+        h.busy_mixed[lane] = s.busy_mixed; h.busy_solo[lane] = s.busy_solo;
+        if (lane == 0) {
+            h.T_end = T_end; h.blk = s.blk;
+            h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
+            h.place_ord = s.place_ord; h.events = s.events; h.err = s.err;
+            h.done = finished ? 1u : 0u;
+            if (!finished) atomicAdd(p.not_done, 1u);
+        }
+        __syncwarp();
+    }
+}
+
+// Zero the statistics of every replication, keep the simulated state.
+__global__ void qsim_reset_kernel(Params p)
+{
+    const uint32_t rep = blockIdx.x * blockDim.x + threadIdx.x;
+    if (rep >= p.R) return;
+    RepHeader &h = p.hdr[rep];
+    const double T = h.T_end;
+    h.T_reset = T;
+    h.events = 0;
+    for (int l = 0; l < 32; ++l) { h.iters_mixed[l] = 0; h.iters_solo[l] = 0; h.busy_mixed[l] = 0.0; h.busy_solo[l] = 0.0; }
+    for (uint32_t i = 0; i < MAXI; ++i) {
+        ClassState &c = h.cs[i];
+        Area *as[5] = { &c.aQp, &c.aX, &c.aQd, &c.aYm, &c.aYs };
+        for (int k = 0; k < 5; ++k) { as[k]->area = 0.0; as[k]->t_last = T; }
+        c.arrivals = c.admitted = c.prefill_done = c.placed_mixed = c.placed_solo = c.done_mixed = c.done_solo = 0;
+        c.abandoned_p = c.abandoned_d = c.overflow = c.overflow_d = c.tok_in_pf = c.tok_in_done = c.tok_out_done = 0;
+        c.sum_ttft = 0.0; c.sum_tpot = 0.0;
+    }
+    if (p.hist_mem) {
+        uint32_t *hm = p.hist_mem + (size_t)rep * p.I * 2 * NBIN;
+        for (uint32_t o = 0; o < p.I * 2 * NBIN; ++o) hm[o] = 0;
+    }
+}
+
+}  // namespace qsimdev
