@@ -142,6 +142,10 @@ int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
  */
 int qsim_run(qsim_t *h, uint64_t horizon_iters);
 
+/* Upper bound on events one replication processes per kernel launch (default 2^40, i.e. one launch per
+ * qsim_run); a replication that reaches it is continued by further launches with identical results. */
+int qsim_set_event_budget(qsim_t *h, uint64_t events_per_launch);
+
 /* Wait until all work queued on the handle's stream has finished; reports sticky replication errors. */
 int qsim_sync(qsim_t *h);
 

@@ -1,0 +1,240 @@
+"""ctypes binding of libqsim.so with the same names as include/qsim.h (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from .build import LIB
+
+MAXI, LMAX, NBIN = 8, 8192, 1024
+
+_COUNTERS = ("arrivals", "admitted", "prefill_done", "placed_mixed", "placed_solo", "done_mixed", "done_solo",
+             "abandoned_p", "abandoned_d", "overflow", "overflow_d", "tokens_in_prefilled",
+             "tokens_in_completed", "tokens_out_completed")
+_STATE = ("Qp", "X", "Qd", "Ym", "Ys")
+_SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_tpot")
+
+EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_set_event_budget", "qsim_sync",
+           "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
+           "qsim_launch_count", "qsim_destroy", "qsim_last_error")
+
+
+class QSimError(RuntimeError):
+    pass
+
+
+class qsim_config(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("size", "I", "N", "R", "B", "C", "nblk", "gate", "router", "placement",
+                                           "pricing", "length_mode", "qcap", "hist")] + \
+               [("seed", C.c_uint64), ("rep_offset", C.c_uint64), ("block_len", C.c_double)]
+
+
+class qsim_class(C.Structure):
+    _fields_ = [("P", C.c_uint32), ("D", C.c_uint32), ("prio_rank", C.c_uint32), ("reserved", C.c_uint32),
+                ("theta", C.c_double)]
+
+
+class qsim_targets(C.Structure):
+    _fields_ = [("M", C.c_uint32), ("reserved", C.c_uint32), ("xstar", C.c_double * MAXI),
+                ("n_xstar", C.c_double * MAXI), ("n_qpstar", C.c_double * MAXI), ("p_solo", C.c_double * MAXI)]
+
+
+class qsim_class_stats(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in _COUNTERS] + [(n, C.c_uint32) for n in _STATE] + \
+               [("reserved", C.c_uint32)] + [(n, C.c_double) for n in _SUMS]
+
+
+class qsim_rep_stats(C.Structure):
+    _fields_ = [("cls", qsim_class_stats * MAXI), ("iters_mixed", C.c_uint64), ("iters_solo", C.c_uint64),
+                ("events", C.c_uint64), ("busy_mixed", C.c_double), ("busy_solo", C.c_double),
+                ("T_elapsed", C.c_double)]
+
+
+_lib = None
+
+
+def load_library():
+    """Load the in-tree libqsim.so; fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB):
+            raise QSimError(f"{LIB} is missing: build it with `python -m paper_2602_02987_b200.build` "
+                            "(there is no CPU fallback)")
+        L = C.CDLL(LIB)
+        vp = C.c_void_p
+        L.qsim_create.argtypes = [C.POINTER(vp), C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
+                                  C.POINTER(qsim_targets)]
+        L.qsim_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+        L.qsim_bind.argtypes = [vp, vp, C.c_size_t, vp]
+        L.qsim_run.argtypes = [vp, C.c_uint64]
+        L.qsim_set_event_budget.argtypes = [vp, C.c_uint64]
+        L.qsim_sync.argtypes = [vp]
+        L.qsim_stats.argtypes = [vp, vp, vp, vp, vp]
+        L.qsim_reset_stats.argtypes = [vp]
+        L.qsim_revenue.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.qsim_server_state.argtypes = [vp, C.c_uint32, vp, vp, vp, vp]
+        L.qsim_simulate.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
+                                    C.POINTER(qsim_targets), C.c_uint64, vp, vp]
+        L.qsim_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.qsim_destroy.argtypes = [vp]
+        L.qsim_last_error.restype = C.c_char_p
+        for n in EXPORTS:
+            if n != "qsim_last_error":
+                getattr(L, n).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise QSimError(f"qsim error {rc}: {load_library().qsim_last_error().decode()}")
+
+
+def _ptr(a):
+    return a.ctypes.data_as(C.c_void_p) if a is not None else None
+
+
+def marshal(inp):
+    """SimInputs -> the C structs and arrays of qsim_create (kept alive by the returned tuple)."""
+    I, nblk = inp.I, inp.nblk
+    if getattr(inp, "inject_t", None) is not None:
+        raise QSimError("injected arrivals are not supported by the CUDA library")
+    cfg = qsim_config(size=C.sizeof(qsim_config), I=I, N=inp.N, R=inp.R, B=inp.B, C=inp.C, nblk=nblk,
+                      gate=inp.gate, router=inp.router, placement=inp.placement, pricing=inp.pricing,
+                      length_mode=inp.length_mode, qcap=inp.qcap, hist=inp.hist, seed=inp.seed,
+                      rep_offset=inp.rep_offset, block_len=inp.block_len)
+    classes = (qsim_class * I)()
+    for i in range(I):
+        classes[i] = qsim_class(P=int(inp.P[i]), D=int(inp.D[i]), prio_rank=int(inp.prio_rank[i]), reserved=0,
+                                theta=float(inp.theta[i]))
+    tg = (qsim_targets * nblk)()
+    for b in range(nblk):
+        tg[b].M = int(inp.M[b])
+        for i in range(I):
+            tg[b].xstar[i] = float(inp.xstar[b, i])
+            tg[b].n_xstar[i] = float(inp.n_xstar[b, i])
+            tg[b].n_qpstar[i] = float(inp.n_qpstar[b, i])
+            tg[b].p_solo[i] = float(inp.p_solo[b, i])
+    rates = np.ascontiguousarray(inp.rates, np.float64)
+    lengths = None if inp.lengths is None else np.ascontiguousarray(inp.lengths, np.uint32)
+    prices = np.ascontiguousarray(inp.prices, np.float64)
+    coeffs = np.ascontiguousarray(inp.coeffs, np.float64)
+    return cfg, classes, rates, lengths, prices, coeffs, tg
+
+
+def _unpack(per, R, I, T_hist=None):
+    out = {}
+    for n in _COUNTERS:
+        out[n] = np.array([[getattr(per[r].cls[i], n) for i in range(I)] for r in range(R)], np.uint64)
+    for n in _STATE:
+        out[n] = np.array([[getattr(per[r].cls[i], n) for i in range(I)] for r in range(R)], np.uint32)
+    for n in _SUMS:
+        out[n] = np.array([[getattr(per[r].cls[i], n) for i in range(I)] for r in range(R)], np.float64)
+    for n in ("iters_mixed", "iters_solo", "events"):
+        out[n] = np.array([getattr(per[r], n) for r in range(R)], np.uint64)
+    for n in ("busy_mixed", "busy_solo", "T_elapsed"):
+        out[n] = np.array([getattr(per[r], n) for r in range(R)], np.float64)
+    return out
+
+
+class QSim:
+    """One handle of the CUDA library; the workspace is a torch tensor on the chosen device."""
+
+    def __init__(self, inp, device="cuda:0", stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise QSimError("no CUDA device: the simulator has no CPU path")
+        self.L = load_library()
+        self.inp = inp
+        self.device = torch.device(device)
+        self._keep = marshal(inp)
+        cfg, classes, rates, lengths, prices, coeffs, tg = self._keep
+        self.h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(self.L.qsim_create(C.byref(self.h), C.byref(cfg), classes, _ptr(rates), _ptr(lengths),
+                                      _ptr(prices), _ptr(coeffs), tg))
+            nbytes = C.c_size_t()
+            _check(self.L.qsim_workspace_bytes(self.h, C.byref(nbytes)))
+            self.workspace_bytes = int(nbytes.value)
+            self.ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
+            base = (self.ws.data_ptr() + 255) & ~255
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            _check(self.L.qsim_bind(self.h, C.c_void_p(base), self.workspace_bytes, C.c_void_p(self.stream.cuda_stream)))
+
+    def set_event_budget(self, n: int) -> None:
+        _check(self.L.qsim_set_event_budget(self.h, int(n)))
+
+    def run(self, horizon_iters: int) -> None:
+        _check(self.L.qsim_run(self.h, int(horizon_iters)))
+
+    def sync(self) -> None:
+        _check(self.L.qsim_sync(self.h))
+
+    def reset_stats(self) -> None:
+        _check(self.L.qsim_reset_stats(self.h))
+
+    def launch_count(self) -> int:
+        n = C.c_uint64()
+        _check(self.L.qsim_launch_count(self.h, C.byref(n)))
+        return int(n.value)
+
+    def stats(self, with_totals=False) -> dict:
+        R, I = self.inp.R, self.inp.I
+        per = (qsim_rep_stats * R)()
+        tot = qsim_rep_stats()
+        ht = hp = None
+        if self.inp.hist:
+            ht = np.zeros((R, I, NBIN), np.uint64)
+            hp = np.zeros((R, I, NBIN), np.uint64)
+        _check(self.L.qsim_stats(self.h, C.byref(tot), per, _ptr(ht), _ptr(hp)))
+        out = _unpack(per, R, I)
+        if self.inp.hist:
+            out["hist_ttft"] = ht
+            out["hist_tpot"] = hp
+        if with_totals:
+            b, s = C.c_double(), C.c_double()
+            _check(self.L.qsim_revenue(self.h, C.byref(tot), C.byref(b), C.byref(s)))
+            out["_totals"] = _unpack((tot,), 1, I)
+            out["_revenue_bundled"] = b.value
+            out["_revenue_separate"] = s.value
+        return out
+
+    def totals(self):
+        """(server iterations, events) summed over replications, cheaply."""
+        tot = qsim_rep_stats()
+        _check(self.L.qsim_stats(self.h, C.byref(tot), None, None, None))
+        return int(tot.iters_mixed + tot.iters_solo), int(tot.events), tot
+
+    def server_state(self, r: int) -> dict:
+        N = self.inp.N
+        n_dec = np.zeros(N, np.uint32); it = np.zeros(N, np.uint32)
+        t_next = np.zeros(N, np.float64); pf_rem = np.zeros(N, np.uint32)
+        _check(self.L.qsim_server_state(self.h, r, _ptr(n_dec), _ptr(it), _ptr(t_next), _ptr(pf_rem)))
+        return dict(n_dec=n_dec, it=it, t_next=t_next, pf_rem=pf_rem)
+
+    def close(self) -> None:
+        if getattr(self, "h", None):
+            self.L.qsim_destroy(self.h)
+            self.h = None
+            self.ws = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def simulate_host(inp, horizon_iters: int) -> dict:
+    """qsim_simulate: host buffers in, host statistics out (allocates and frees its own device memory)."""
+    L = load_library()
+    cfg, classes, rates, lengths, prices, coeffs, tg = marshal(inp)
+    per = (qsim_rep_stats * inp.R)()
+    tot = qsim_rep_stats()
+    _check(L.qsim_simulate(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
+                           int(horizon_iters), C.byref(tot), per))
+    out = _unpack(per, inp.R, inp.I)
+    out["_totals"] = _unpack((tot,), 1, inp.I)
+    return out

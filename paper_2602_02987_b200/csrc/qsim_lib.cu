@@ -1,0 +1,450 @@
+// Host side of libqsim: the C ABI declared in include/qsim.h.
+// Validates arguments, lays out the caller's workspace, launches the kernels of qsim_device.cuh and
+// converts the device records into the public statistics structs.  No CPU simulation path exists here:
+// without a CUDA device every entry point that needs one fails with QSIM_ECUDA.
+#include "qsim.h"
+#include "qsim_device.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace qsimdev;
+
+namespace {
+
+thread_local std::string g_err;
+
+int fail(int code, const std::string &msg)
+{
+    g_err = msg;
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                         \
+    do {                                                                                       \
+        cudaError_t e_ = (expr);                                                               \
+        if (e_ != cudaSuccess)                                                                 \
+            return fail(QSIM_ECUDA, std::string(#expr) + ": " + cudaGetErrorString(e_));       \
+    } while (0)
+
+size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+struct Sections {
+    size_t hdr, srv, fin, tpf, pk, pq, dq, hist, flag, total;
+};
+
+}  // namespace
+
+struct qsim {
+    qsim_config cfg{};
+    qsim_class cls[QSIM_MAXI]{};
+    double prices[2]{};
+    Params par{};
+    SmemLayout lay{};
+    Sections sec{};
+    BlockPar *d_blocks = nullptr;
+    uint32_t *d_lengths = nullptr;
+    uint32_t *h_flag = nullptr;   // pinned
+    void *ws = nullptr;
+    cudaStream_t stream = nullptr;
+    bool bound = false;
+    uint64_t launches = 0;
+    int device = 0;
+};
+
+namespace {
+
+Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
+{
+    Sections s{};
+    size_t o = 0;
+    const size_t R = c.R, NB = (size_t)c.N * c.B;
+    s.hdr = o; o = align256(o + R * sizeof(RepHeader));
+    s.srv = o; o = align256(o + R * (size_t)srv_bytes);
+    s.fin = o; o = align256(o + R * NB * 4);
+    s.tpf = o; o = align256(o + R * NB * 8);
+    s.pk = o; o = align256(o + R * NB * 4);
+    s.pq = o; o = align256(o + R * (size_t)c.I * c.qcap * sizeof(QEntry));
+    s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
+    s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
+    s.flag = o; o = align256(o + 256);
+    s.total = o;
+    return s;
+}
+
+int validate(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
+             const double *prices, const double *coef, const qsim_targets *tg)
+{
+    if (!cfg || !classes || !rates || !prices || !coef || !tg) return fail(QSIM_EINVAL, "null argument");
+    if (cfg->size != sizeof(qsim_config)) return fail(QSIM_EINVAL, "qsim_config.size does not match this library");
+    if (cfg->I < 1 || cfg->I > QSIM_MAXI) return fail(QSIM_EINVAL, "I must be in 1..8");
+    if (cfg->N < 1 || cfg->N > 4096) return fail(QSIM_EINVAL, "N must be in 1..4096");
+    if (cfg->R < 1) return fail(QSIM_EINVAL, "R must be >= 1");
+    if (cfg->B < 1 || cfg->B > 4096) return fail(QSIM_EINVAL, "B must be in 1..4096");
+    if (cfg->C < 1 || cfg->C > 65535) return fail(QSIM_EINVAL, "C must be in 1..65535");
+    if (cfg->nblk < 1) return fail(QSIM_EINVAL, "nblk must be >= 1");
+    if (cfg->qcap < 1 || cfg->qcap > (1u << 24)) return fail(QSIM_EINVAL, "qcap must be in 1..2^24");
+    if (cfg->gate > 1 || cfg->router > 1 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
+        return fail(QSIM_EINVAL, "enum out of range");
+    if (cfg->nblk > 1 && !(cfg->block_len > 0.0 && std::isfinite(cfg->block_len)))
+        return fail(QSIM_EINVAL, "block_len must be positive when nblk > 1");
+    if (cfg->length_mode == QSIM_LENGTH_TABLE && !lengths) return fail(QSIM_EINVAL, "length tables missing");
+    for (uint32_t i = 0; i < cfg->I; ++i) {
+        if (classes[i].P < 1 || classes[i].P > QSIM_LMAX || classes[i].D < 1 || classes[i].D > QSIM_LMAX)
+            return fail(QSIM_EINVAL, "class lengths must be in 1..8192");
+        if (!(classes[i].theta >= 0.0) || !std::isfinite(classes[i].theta)) return fail(QSIM_EINVAL, "theta must be >= 0");
+    }
+    for (size_t k = 0; k < (size_t)cfg->nblk * cfg->I; ++k)
+        if (!(rates[k] >= 0.0) || !std::isfinite(rates[k])) return fail(QSIM_EINVAL, "rates must be finite and >= 0");
+    for (int k = 0; k < 6; ++k)
+        if (!std::isfinite(coef[k]) || coef[k] < 0.0) return fail(QSIM_EINVAL, "iteration-time coefficients must be finite and >= 0");
+    if (!(coef[0] > 0.0) || !(coef[3] > 0.0)) return fail(QSIM_EINVAL, "alpha_m and alpha_s must be positive");
+    if (!std::isfinite(prices[0]) || !std::isfinite(prices[1])) return fail(QSIM_EINVAL, "prices must be finite");
+    for (uint32_t b = 0; b < cfg->nblk; ++b) {
+        if (tg[b].M > cfg->N) return fail(QSIM_EINVAL, "M must be <= N");
+        for (uint32_t i = 0; i < cfg->I; ++i) {
+            if (!std::isfinite(tg[b].xstar[i]) || tg[b].xstar[i] < 0.0 || !std::isfinite(tg[b].n_xstar[i]) ||
+                !std::isfinite(tg[b].n_qpstar[i]) || !(tg[b].p_solo[i] >= 0.0 && tg[b].p_solo[i] <= 1.0))
+                return fail(QSIM_EINVAL, "LP targets out of range");
+        }
+    }
+    if (lengths && cfg->length_mode == QSIM_LENGTH_TABLE)
+        for (uint32_t t = 0; t < cfg->I * 2; ++t) {
+            const uint32_t *thr = lengths + (size_t)t * QSIM_LMAX;
+            for (uint32_t j = 1; j < QSIM_LMAX - 1; ++j)
+                if (thr[j] < thr[j - 1]) return fail(QSIM_EINVAL, "length thresholds must be non-decreasing");
+        }
+    return QSIM_OK;
+}
+
+int launch_run(qsim *h, bool advance, uint64_t horizon)
+{
+    Params p = h->par;
+    p.advance = advance ? 1u : 0u;
+    p.horizon_iters = horizon;
+    CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
+    qsim_run_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    h->launches++;
+    CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
+    return QSIM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *qsim_last_error(void) { return g_err.c_str(); }
+
+int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                const uint32_t *lengths, const double *prices, const double *coef, const qsim_targets *tg)
+{
+    if (!out) return fail(QSIM_EINVAL, "null out pointer");
+    *out = nullptr;
+    int rc = validate(cfg, classes, rates, lengths, prices, coef, tg);
+    if (rc != QSIM_OK) return rc;
+    int ndev = 0;
+    CUDA_TRY(cudaGetDeviceCount(&ndev));
+    if (ndev < 1) return fail(QSIM_ECUDA, "no CUDA device");
+    qsim *h = new (std::nothrow) qsim();
+    if (!h) return fail(QSIM_ENOMEM, "host allocation failed");
+    CUDA_TRY(cudaGetDevice(&h->device));
+    h->cfg = *cfg;
+    std::memcpy(h->cls, classes, cfg->I * sizeof(qsim_class));
+    h->prices[0] = prices[0];
+    h->prices[1] = prices[1];
+    Params &p = h->par;
+    p.I = cfg->I; p.N = cfg->N; p.Npad = (cfg->N + 31u) & ~31u; p.R = cfg->R; p.B = cfg->B; p.C = cfg->C;
+    p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
+    p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = cfg->hist;
+    p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
+    p.event_budget = 1ull << 40;
+    for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
+    for (uint32_t i = 0; i < cfg->I; ++i) {
+        p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
+        p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
+    }
+    h->lay = smem_layout(p.Npad);
+    p.srv_bytes = h->lay.srv_bytes;
+    if (h->lay.total > 227u * 1024u) {
+        delete h;
+        return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
+    }
+    h->sec = layout_sections(*cfg, p.srv_bytes);
+    std::vector<BlockPar> blocks(cfg->nblk);
+    for (uint32_t b = 0; b < cfg->nblk; ++b) {
+        BlockPar &bp = blocks[b];
+        std::memset(&bp, 0, sizeof bp);
+        bp.M = tg[b].M;
+        for (uint32_t i = 0; i < cfg->I; ++i) {
+            bp.xstar[i] = tg[b].xstar[i]; bp.nx[i] = tg[b].n_xstar[i]; bp.nq[i] = tg[b].n_qpstar[i];
+            bp.ps[i] = tg[b].p_solo[i]; bp.rate[i] = rates[(size_t)b * cfg->I + i];
+        }
+    }
+    cudaError_t e = cudaMalloc(&h->d_blocks, blocks.size() * sizeof(BlockPar));
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_blocks, blocks.data(), blocks.size() * sizeof(BlockPar), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && cfg->length_mode == QSIM_LENGTH_TABLE) {
+        const size_t nb = (size_t)cfg->I * 2 * QSIM_LMAX * 4;
+        e = cudaMalloc(&h->d_lengths, nb);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_lengths, lengths, nb, cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) e = cudaMallocHost(&h->h_flag, 256);
+    if (e == cudaSuccess && h->lay.total > 48u * 1024u) {
+        e = cudaFuncSetAttribute(qsim_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(qsim_init_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total);
+    }
+    if (e != cudaSuccess) {
+        std::string msg = std::string("device set-up failed: ") + cudaGetErrorString(e);
+        qsim_destroy(h);
+        return fail(e == cudaErrorMemoryAllocation ? QSIM_ENOMEM : QSIM_ECUDA, msg);
+    }
+    p.blocks = h->d_blocks;
+    p.lengths = h->d_lengths;
+    *out = h;
+    return QSIM_OK;
+}
+
+int qsim_workspace_bytes(const qsim_t *h, size_t *bytes)
+{
+    if (!h || !bytes) return fail(QSIM_EINVAL, "null argument");
+    *bytes = h->sec.total;
+    return QSIM_OK;
+}
+
+int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!ws) return fail(QSIM_EWORKSPACE, "workspace pointer is null");
+    if (bytes < h->sec.total) return fail(QSIM_EWORKSPACE, "workspace too small: need " + std::to_string(h->sec.total) + " bytes");
+    if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return fail(QSIM_EWORKSPACE, "workspace must be 256-byte aligned");
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, ws) != cudaSuccess || (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged)) {
+        cudaGetLastError();
+        return fail(QSIM_EWORKSPACE, "workspace is not device memory");
+    }
+    h->ws = ws;
+    h->stream = static_cast<cudaStream_t>(cuda_stream);
+    char *base = static_cast<char *>(ws);
+    Params &p = h->par;
+    p.hdr = reinterpret_cast<RepHeader *>(base + h->sec.hdr);
+    p.srv = base + h->sec.srv;
+    p.slot_fin = reinterpret_cast<uint32_t *>(base + h->sec.fin);
+    p.slot_tpf = reinterpret_cast<double *>(base + h->sec.tpf);
+    p.slot_pk = reinterpret_cast<uint32_t *>(base + h->sec.pk);
+    p.pq = reinterpret_cast<QEntry *>(base + h->sec.pq);
+    p.dq = reinterpret_cast<QEntry *>(base + h->sec.dq);
+    p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
+    p.not_done = reinterpret_cast<uint32_t *>(base + h->sec.flag);
+    qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    h->launches++;
+    h->bound = true;
+    return QSIM_OK;
+}
+
+int qsim_run(qsim_t *h, uint64_t horizon_iters)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_run before qsim_bind");
+    int rc = launch_run(h, true, horizon_iters);
+    if (rc != QSIM_OK) return rc;
+    // a replication that used up its per-launch event budget is continued by further launches
+    for (;;) {
+        CUDA_TRY(cudaStreamSynchronize(h->stream));
+        if (*h->h_flag == 0) break;
+        rc = launch_run(h, false, 0);
+        if (rc != QSIM_OK) return rc;
+    }
+    return QSIM_OK;
+}
+
+int qsim_set_event_budget(qsim_t *h, uint64_t events_per_launch)
+{
+    if (!h || events_per_launch == 0) return fail(QSIM_EINVAL, "bad event budget");
+    h->par.event_budget = events_per_launch;
+    return QSIM_OK;
+}
+
+int qsim_sync(qsim_t *h)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    return QSIM_OK;
+}
+
+int qsim_launch_count(const qsim_t *h, uint64_t *launches)
+{
+    if (!h || !launches) return fail(QSIM_EINVAL, "null argument");
+    *launches = h->launches;
+    return QSIM_OK;
+}
+
+int qsim_reset_stats(qsim_t *h)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_reset_stats before qsim_bind");
+    qsim_reset_kernel<<<(h->cfg.R + 127) / 128, 128, 0, h->stream>>>(h->par);
+    CUDA_TRY(cudaGetLastError());
+    h->launches++;
+    return QSIM_OK;
+}
+
+int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint64_t *hist_ttft, uint64_t *hist_tpot)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_stats before qsim_bind");
+    const uint32_t R = h->cfg.R, I = h->cfg.I;
+    std::vector<RepHeader> hdr(R);
+    CUDA_TRY(cudaMemcpyAsync(hdr.data(), h->par.hdr, (size_t)R * sizeof(RepHeader), cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    qsim_rep_stats tot;
+    std::memset(&tot, 0, sizeof tot);
+    for (uint32_t r = 0; r < R; ++r) {
+        const RepHeader &H = hdr[r];
+        if (H.err) return fail(QSIM_EOVERFLOW, "replication " + std::to_string(r) + " hit an internal bound (code " + std::to_string(H.err) + ")");
+        qsim_rep_stats st;
+        std::memset(&st, 0, sizeof st);
+        const double T = H.T_end;
+        st.T_elapsed = T - H.T_reset;
+        st.events = H.events;
+        for (int l = 0; l < 32; ++l) {
+            st.iters_mixed += H.iters_mixed[l];
+            st.iters_solo += H.iters_solo[l];
+            st.busy_mixed = st.busy_mixed + H.busy_mixed[l];
+            st.busy_solo = st.busy_solo + H.busy_solo[l];
+        }
+        for (uint32_t i = 0; i < I; ++i) {
+            const ClassState &c = H.cs[i];
+            qsim_class_stats &o = st.cls[i];
+            o.arrivals = c.arrivals; o.admitted = c.admitted; o.prefill_done = c.prefill_done;
+            o.placed_mixed = c.placed_mixed; o.placed_solo = c.placed_solo; o.done_mixed = c.done_mixed;
+            o.done_solo = c.done_solo; o.abandoned_p = c.abandoned_p; o.abandoned_d = c.abandoned_d;
+            o.overflow = c.overflow; o.overflow_d = c.overflow_d; o.tokens_in_prefilled = c.tok_in_pf;
+            o.tokens_in_completed = c.tok_in_done; o.tokens_out_completed = c.tok_out_done;
+            const uint32_t Qd = c.Qd0 + c.Qd1;
+            o.Qp = c.pq_n; o.X = c.X; o.Qd = Qd; o.Ym = c.Ym; o.Ys = c.Ys;
+            // integrals are reported up to the end of the run without touching the stored state
+            o.area_Qp = c.aQp.area + (double)c.pq_n * (T - c.aQp.t_last);
+            o.area_X = c.aX.area + (double)c.X * (T - c.aX.t_last);
+            o.area_Qd = c.aQd.area + (double)Qd * (T - c.aQd.t_last);
+            o.area_Ym = c.aYm.area + (double)c.Ym * (T - c.aYm.t_last);
+            o.area_Ys = c.aYs.area + (double)c.Ys * (T - c.aYs.t_last);
+            o.sum_ttft = c.sum_ttft; o.sum_tpot = c.sum_tpot;
+        }
+        if (per_rep) per_rep[r] = st;
+        tot.iters_mixed += st.iters_mixed; tot.iters_solo += st.iters_solo; tot.events += st.events;
+        tot.busy_mixed += st.busy_mixed; tot.busy_solo += st.busy_solo; tot.T_elapsed += st.T_elapsed;
+        for (uint32_t i = 0; i < I; ++i) {
+            const qsim_class_stats &a = st.cls[i];
+            qsim_class_stats &b = tot.cls[i];
+            b.arrivals += a.arrivals; b.admitted += a.admitted; b.prefill_done += a.prefill_done;
+            b.placed_mixed += a.placed_mixed; b.placed_solo += a.placed_solo; b.done_mixed += a.done_mixed;
+            b.done_solo += a.done_solo; b.abandoned_p += a.abandoned_p; b.abandoned_d += a.abandoned_d;
+            b.overflow += a.overflow; b.overflow_d += a.overflow_d; b.tokens_in_prefilled += a.tokens_in_prefilled;
+            b.tokens_in_completed += a.tokens_in_completed; b.tokens_out_completed += a.tokens_out_completed;
+            b.Qp += a.Qp; b.X += a.X; b.Qd += a.Qd; b.Ym += a.Ym; b.Ys += a.Ys;
+            b.area_Qp += a.area_Qp; b.area_X += a.area_X; b.area_Qd += a.area_Qd; b.area_Ym += a.area_Ym;
+            b.area_Ys += a.area_Ys; b.sum_ttft += a.sum_ttft; b.sum_tpot += a.sum_tpot;
+        }
+    }
+    if (totals) *totals = tot;
+    if (hist_ttft || hist_tpot) {
+        const size_t per = (size_t)I * NBIN;
+        if (hist_ttft) std::memset(hist_ttft, 0, (size_t)R * per * 8);
+        if (hist_tpot) std::memset(hist_tpot, 0, (size_t)R * per * 8);
+        if (h->cfg.hist) {
+            std::vector<uint32_t> raw((size_t)R * per * 2);
+            CUDA_TRY(cudaMemcpyAsync(raw.data(), h->par.hist_mem, raw.size() * 4, cudaMemcpyDeviceToHost, h->stream));
+            CUDA_TRY(cudaStreamSynchronize(h->stream));
+            for (uint32_t r = 0; r < R; ++r)
+                for (uint32_t i = 0; i < I; ++i)
+                    for (uint32_t b = 0; b < NBIN; ++b) {
+                        const size_t src = (((size_t)r * I + i) * 2) * NBIN + b;
+                        const size_t dst = ((size_t)r * I + i) * NBIN + b;
+                        if (hist_ttft) hist_ttft[dst] = raw[src];
+                        if (hist_tpot) hist_tpot[dst] = raw[src + NBIN];
+                    }
+        }
+    }
+    return QSIM_OK;
+}
+
+int qsim_revenue(const qsim_t *h, const qsim_rep_stats *totals, double *bundled_rate, double *separate_rate)
+{
+    if (!h || !totals) return fail(QSIM_EINVAL, "null argument");
+    double tin_done = 0, tin_pf = 0, tout = 0;
+    for (uint32_t i = 0; i < h->cfg.I; ++i) {
+        tin_done += (double)totals->cls[i].tokens_in_completed;
+        tin_pf += (double)totals->cls[i].tokens_in_prefilled;
+        tout += (double)totals->cls[i].tokens_out_completed;
+    }
+    const double denom = (double)h->cfg.N * totals->T_elapsed;
+    if (!(denom > 0.0)) return fail(QSIM_ESTATE, "no simulated time has elapsed");
+    if (bundled_rate) *bundled_rate = (h->prices[0] * tin_done + h->prices[1] * tout) / denom;
+    if (separate_rate) *separate_rate = (h->prices[0] * tin_pf + h->prices[1] * tout) / denom;
+    return QSIM_OK;
+}
+
+int qsim_server_state(qsim_t *h, uint32_t r, uint32_t *n_dec, uint32_t *it, double *t_next, uint32_t *pf_rem)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_server_state before qsim_bind");
+    if (r >= h->cfg.R) return fail(QSIM_EINVAL, "replication index out of range");
+    std::vector<char> img(h->lay.srv_bytes);
+    CUDA_TRY(cudaMemcpyAsync(img.data(), h->par.srv + (size_t)r * h->lay.srv_bytes, img.size(), cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    const double *tn = reinterpret_cast<const double *>(img.data() + h->lay.off_tnext);
+    const uint32_t *itv = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_it);
+    const uint32_t *rem = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_pfrem);
+    const uint32_t *pj = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_pfjob);
+    const uint16_t *nd = reinterpret_cast<const uint16_t *>(img.data() + h->lay.off_ndec);
+    for (uint32_t g = 0; g < h->cfg.N; ++g) {
+        if (n_dec) n_dec[g] = nd[g];
+        if (it) it[g] = itv[g];
+        if (t_next) t_next[g] = tn[g];
+        if (pf_rem) pf_rem[g] = (pj[g] >> 31) ? rem[g] : 0u;
+    }
+    return QSIM_OK;
+}
+
+int qsim_destroy(qsim_t *h)
+{
+    if (!h) return QSIM_OK;
+    if (h->bound) cudaStreamSynchronize(h->stream);
+    if (h->d_blocks) cudaFree(h->d_blocks);
+    if (h->d_lengths) cudaFree(h->d_lengths);
+    if (h->h_flag) cudaFreeHost(h->h_flag);
+    delete h;
+    return QSIM_OK;
+}
+
+int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
+                  const double *prices, const double *coef, const qsim_targets *tg, uint64_t horizon_iters,
+                  qsim_rep_stats *totals, qsim_rep_stats *per_rep)
+{
+    qsim_t *h = nullptr;
+    int rc = qsim_create(&h, cfg, classes, rates, lengths, prices, coef, tg);
+    if (rc != QSIM_OK) return rc;
+    void *ws = nullptr;
+    cudaError_t e = cudaMalloc(&ws, h->sec.total);
+    if (e != cudaSuccess) {
+        qsim_destroy(h);
+        return fail(QSIM_ENOMEM, std::string("cudaMalloc(workspace): ") + cudaGetErrorString(e));
+    }
+    rc = qsim_bind(h, ws, h->sec.total, nullptr);
+    if (rc == QSIM_OK) rc = qsim_run(h, horizon_iters);
+    if (rc == QSIM_OK) rc = qsim_stats(h, totals, per_rep, nullptr, nullptr);
+    const std::string keep = g_err;
+    qsim_destroy(h);
+    cudaFree(ws);
+    if (rc != QSIM_OK) g_err = keep;
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,170 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from qsim_inputs import presets
+from qsim_inputs.spec import (GATE_OCCUPANCY, GATE_PRIORITY, PLACE_LEAST_LOADED, PLACE_RANDOM, ROUTER_SLI,
+                              ROUTER_SOLO_FIRST)
+
+from parity import assert_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def gpu_run(inp, horizon, chunks=None, budget=None):
+    from paper_2602_02987_b200 import QSim
+    sim = QSim(inp)
+    if budget:
+        sim.set_event_budget(budget)
+    for h in (chunks or [horizon]):
+        sim.run(h)
+    st = sim.stats()
+    state = [sim.server_state(r) for r in range(min(inp.R, 2))]
+    sim.close()
+    return st, state
+
+
+def oracle_run(inp, horizon, reps=None):
+    from oracle import OracleSim
+    sim = OracleSim(inp)
+    if reps is None:
+        sim.run(horizon)
+    else:
+        for r in reps:
+            sim.run(horizon, r, r + 1)
+    st = sim.stats()
+    state = [sim.server_state(r) for r in range(min(inp.R, 2))]
+    sim.close()
+    return st, state
+
+
+def check(inp, horizon, reps=None, **kw):
+    g, gs = gpu_run(inp, horizon, **kw)
+    o, os_ = oracle_run(inp, horizon, reps)
+    assert_parity(g, o, rows=reps, what=inp.name)
+    if reps is None:
+        for a, b in zip(gs, os_):
+            for k in a:
+                assert np.array_equal(a[k], b[k]), (inp.name, "server state", k)
+    return g
+
+
+def test_cfg0_whole_both_placements():
+    for placement in (PLACE_LEAST_LOADED, PLACE_RANDOM):
+        inp = presets.cfg0(placement=placement)
+        st = check(inp, 10_000)
+        assert st["overflow"].sum() == 0
+        assert int(st["iters_mixed"].sum() + st["iters_solo"].sum()) > 400_000
+
+
+@pytest.mark.parametrize("gate", [GATE_OCCUPANCY, GATE_PRIORITY])
+@pytest.mark.parametrize("placement", [PLACE_RANDOM, PLACE_LEAST_LOADED])
+@pytest.mark.parametrize("router", [ROUTER_SOLO_FIRST, ROUTER_SLI])
+def test_paper_instance_all_policy_modes(gate, placement, router):
+    # abandonment in both queues, decode backlog, N not a multiple of 32
+    inp = presets.paper_instance(n=37, R=6, gate=gate, placement=placement, router=router)
+    check(inp, 6000)
+
+
+def test_cfg1_subset_lognormal_tables_priority_gate():
+    inp = presets.cfg1(R=8)
+    check(inp, 1500)
+
+
+def test_cfg2_subset_overload_with_abandonment():
+    inp = presets.cfg2(N=512, R=3)
+    st = check(inp, 400)
+    assert st["abandoned_p"].sum() > 0
+
+
+def test_cfg3_subset_block_tables_and_histograms():
+    inp = presets.cfg3(N=96, R=4, block_len=1.0)
+    H = inp.meta["horizon_iters"]
+    st = check(inp, H)
+    assert st["hist_ttft"].sum() == st["prefill_done"].sum()
+    assert st["hist_tpot"].sum() == (st["done_mixed"] + st["done_solo"]).sum()
+
+
+def test_cfg4_subset_sli_router_constrained_targets():
+    for N in (16, 256):
+        inp = presets.cfg4(N=N, R=3)
+        check(inp, 1200 if N == 16 else 500)
+
+
+def test_large_n_one_replication():
+    inp = presets.cfg4(N=4096, R=1)
+    check(inp, 60)
+
+
+def test_kv_slope_coefficients():
+    inp = presets.paper_instance(n=12, R=4, coeffs=presets.COEFFS_PAPER_KV)
+    check(inp, 20_000)
+
+
+def test_resumable_and_event_budget_do_not_change_results():
+    inp = presets.cfg2(N=48, R=4)
+    a, _ = gpu_run(inp, 3000)
+    b, _ = gpu_run(inp, 3000, chunks=[700, 1300, 1000])
+    c, _ = gpu_run(inp, 3000, budget=5000)
+    for k in a:
+        assert np.array_equal(a[k], b[k]), ("chunks", k)
+        assert np.array_equal(a[k], c[k]), ("budget", k)
+
+
+def test_replication_offset_shards_compose():
+    inp = presets.cfg0(R=8, horizon_iters=2000)
+    whole, _ = gpu_run(inp, 2000)
+    lo, _ = gpu_run(inp.with_(R=5), 2000)
+    hi, _ = gpu_run(inp.with_(R=3, rep_offset=5), 2000)
+    for k in whole:
+        assert np.array_equal(whole[k], np.concatenate([lo[k], hi[k]])), k
+
+
+def test_reset_stats_and_host_entry_point():
+    from paper_2602_02987_b200 import QSim, simulate_host
+    inp = presets.cfg0(R=4, horizon_iters=3000)
+    sim = QSim(inp)
+    sim.run(1000); sim.reset_stats(); sim.run(2000)
+    g = sim.stats(with_totals=True)
+    sim.close()
+    from oracle import OracleSim
+    o = OracleSim(inp); o.run(1000); o.reset_stats(); o.run(2000)
+    assert_parity(g, o.stats(), what="after reset")
+    o.close()
+    # totals are the sums over replications; revenue follows Eq. (22)
+    assert int(g["_totals"]["arrivals"].sum()) == int(g["arrivals"].sum())
+    T = g["T_elapsed"].sum()
+    rev = (1.0 * g["tokens_in_completed"].sum() + 2.0 * g["tokens_out_completed"].sum()) / (inp.N * T)
+    assert abs(g["_revenue_bundled"] - rev) <= 1e-12 * rev
+    # the one-call host entry point gives the same statistics
+    h = simulate_host(inp, 3000)
+    ref, _ = gpu_run(inp, 3000)
+    for k in ref:
+        assert np.array_equal(ref[k], h[k]), k
+
+
+def test_degenerate_sizes():
+    # one GPU, one class, B = 1 (a mixed GPU then has no decode slot: jobs wait for the solo GPU)
+    inp = presets.single_class(N=2, B=1, P=300, D=3, lam=5.0, theta=0.5, R=3, M=1)
+    check(inp, 20_000)
+    inp = presets.single_class(N=1, B=4, P=8192, D=8192, lam=0.05, R=2, M=1)
+    check(inp, 40_000)
+    # zero arrival rate: nothing ever happens
+    inp = presets.single_class(N=3, B=4, lam=1.0, R=2)
+    st, _ = gpu_run(inp.with_(rates=np.zeros((1, 1))), 1000)
+    assert st["events"].sum() == 0 and st["T_elapsed"][0] > 0
+
+
+def test_tiny_queue_capacity_overflows_identically():
+    inp = presets.cfg0(R=3, horizon_iters=3000).with_(qcap=2)
+    st = check(inp, 3000)
+    assert st["overflow"].sum() > 0
+
+
+def test_bad_arguments_are_rejected():
+    from paper_2602_02987_b200 import QSim, QSimError
+    good = presets.cfg0(R=2)
+    for bad in (good.with_(N=5000), good.with_(qcap=0), good.with_(C=70000),
+                good.with_(coeffs=np.array([0.0, 1e-5, 0, 0.005, 0, 0]))):
+        with pytest.raises(QSimError):
+            QSim(bad)
