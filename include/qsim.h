@@ -135,10 +135,11 @@ int qsim_workspace_bytes(const qsim_t *h, size_t *bytes);
 int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
 
 /*
- * Advance every replication by horizon_iters * tau_ref simulated seconds, tau_ref = tau(0, B, 0) (one
- * full solo iteration) [event-driven dynamics of Section 2.3 under the policies of Sections 4-5].
- * Events with time <= the new end are processed.  Calls compose: run(a); run(b) leaves exactly the
- * state of run(a + b).  qsim_stats / qsim_sync wait for completion.
+ * Advance every replication by horizon_iters more iterations of horizon [event-driven dynamics of
+ * Section 2.3 under the policies of Sections 4-5]: the new end time is H * tau_ref, H the total horizon
+ * requested so far and tau_ref = tau(0, B, 0) (one full solo iteration).  Events with time <= the new end
+ * are processed.  Calls compose: run(a); run(b) leaves exactly the state of run(a + b).
+ * qsim_stats / qsim_sync wait for completion.
  */
 int qsim_run(qsim_t *h, uint64_t horizon_iters);
 

@@ -131,6 +131,7 @@ typedef struct { double area, t_last; } area_t;
 
 typedef struct {
     double T_end, T_reset;
+    uint64_t H_total;           /* iterations of horizon requested so far: T_end = H_total * tau_ref */
     uint32_t blk;
     /* arrivals */
     double ta[ORC_MAXI];
@@ -664,9 +665,12 @@ uint64_t orc_trace_count(const orc_sim *s) { return s ? s->trace_n : 0; }
 int orc_run(orc_sim *s, uint64_t horizon_iters, uint32_t rep_lo, uint32_t rep_hi)
 {
     if (!s || rep_lo > rep_hi || rep_hi > s->cfg.R) return -1;
-    double dT = (double)horizon_iters * tau_ref(s);
-    for (uint32_t r = rep_lo; r < rep_hi; ++r)
-        run_rep(s, r, s->reps[r].T_end + dT);
+    for (uint32_t r = rep_lo; r < rep_hi; ++r) {
+        /* the end time is one rounded product of the cumulative horizon, so run(a); run(b) ends
+         * exactly where run(a + b) ends */
+        s->reps[r].H_total += horizon_iters;
+        run_rep(s, r, (double)s->reps[r].H_total * tau_ref(s));
+    }
     return 0;
 }
 

@@ -93,7 +93,8 @@ int orc_create(orc_sim **out, const orc_config *cfg, const orc_class *classes, c
 /* Optional trace sink; records beyond cap are counted but dropped. */
 int orc_set_trace(orc_sim *s, orc_trace_rec *buf, uint64_t cap);
 uint64_t orc_trace_count(const orc_sim *s);
-/* Advance replications [rep_lo, rep_hi) by horizon_iters * tau_ref seconds (tau_ref = full solo iteration). */
+/* Advance replications [rep_lo, rep_hi) by horizon_iters more iterations of horizon: the new end time is
+ * (total horizon so far) * tau_ref, tau_ref = one full solo iteration. */
 int orc_run(orc_sim *s, uint64_t horizon_iters, uint32_t rep_lo, uint32_t rep_hi);
 int orc_reset_stats(orc_sim *s);
 /* per_rep: [R]; hist_ttft / hist_tpot: NULL or uint64 [R][I][ORC_NBIN] */

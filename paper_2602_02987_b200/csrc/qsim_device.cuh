@@ -53,7 +53,7 @@ struct ClassState {
 
 struct RepHeader {
     double T_end, T_reset;
-    unsigned long long place_ord, events;
+    unsigned long long place_ord, events, H_total, pad64;
     uint32_t blk, done, err, pad;
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
     unsigned long long iters_mixed[32], iters_solo[32];
@@ -924,8 +924,10 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
             for (uint32_t o = lane; o < sizeof(ClassState) * MAXI / 16; o += 32) dst[o] = src[o];
         }
         __syncwarp();
+        // the end time is one rounded product of the cumulative horizon: run(a); run(b) ends where run(a+b) ends
         double T_end = h.T_end;
-        if (p.advance) T_end = __dadd_rn(T_end, __dmul_rn((double)p.horizon_iters, iter_time(p, 0, p.B, 0)));
+        const unsigned long long H_total = h.H_total + (p.advance ? p.horizon_iters : 0ull);
+        if (p.advance) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
         s.T_end = T_end;
         s.t = 0.0;
         s.load_block(h.blk);
@@ -949,7 +951,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         h.iters_mixed[lane] = s.it_mixed; h.iters_solo[lane] = s.it_solo;
         h.busy_mixed[lane] = s.busy_mixed; h.busy_solo[lane] = s.busy_solo;
         if (lane == 0) {
-            h.T_end = T_end; h.blk = s.blk;
+            h.T_end = T_end; h.H_total = H_total; h.blk = s.blk;
             h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
             h.place_ord = s.place_ord; h.events = s.events; h.err = s.err;
             h.done = finished ? 1u : 0u;

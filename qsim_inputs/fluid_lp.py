@@ -47,6 +47,36 @@ def service_rates(P, D, C: int, tau_mix: float, tau_solo: float):
     return mu_p, mu_m, mu_s
 
 
+def consistent_taus(coeffs, B: int, C: int, solve, iters: int = 40, tol: float = 1e-10, start=None):
+    """Planning constants (tau_mix, tau_solo) when the iteration time depends on the decode count.
+
+    The paper's law (Eq. (2)-(3)) has constant tau_mix and tau_solo; with a per-decode slope the LP needs
+    the batch sizes it induces.  Fixed point: solve the LP under the current constants (`solve` maps
+    (tau_mix, tau_solo) to a Plan), read the mean decodes per mixed GPU  sum y_m / sum x  and per solo GPU
+    sum y_s / (1 - sum x), and re-evaluate tau there.  Starts from full batches, which is exact when
+    the slopes are zero (or from `start`).  Returns (tau_mix, tau_solo, plan).
+    """
+    tm, ts = start if start is not None else nominal_taus(coeffs, B, C)
+    plan = solve(tm, ts)
+    if coeffs[2] == 0.0 and coeffs[4] == 0.0:
+        return tm, ts, plan
+    for _ in range(iters):
+        X = float(plan.x.sum())
+        d_m = float(plan.ym.sum()) / X if X > 1e-12 else 0.0
+        d_s = float(plan.ys.sum()) / (1.0 - X) if 1.0 - X > 1e-12 else float(B)
+        d_m = min(max(d_m, 0.0), B - 1)
+        d_s = min(max(d_s, 1.0), B)
+        # damped update keeps the iteration from oscillating between vertex solutions
+        tm_new = 0.5 * tm + 0.5 * (coeffs[0] + coeffs[1] * C + coeffs[2] * d_m)
+        ts_new = 0.5 * ts + 0.5 * (coeffs[3] + coeffs[4] * d_s)
+        done = abs(tm_new - tm) < tol and abs(ts_new - ts) < tol
+        tm, ts = tm_new, ts_new
+        plan = solve(tm, ts)
+        if done:
+            break
+    return tm, ts, plan
+
+
 def fluid_capacity(pi, P, D, B: int, C: int, tau_mix: float, tau_solo: float) -> float:
     """Largest total per-GPU arrival rate s such that lambda = s*pi is servable with empty queues.
 

@@ -7,6 +7,7 @@ two-class experiment of the paper's convergence study (Section EC "Convergence A
 """
 from __future__ import annotations
 
+import functools
 import math
 
 import numpy as np
@@ -37,9 +38,18 @@ def _next_pow2(v: float) -> int:
 
 
 def _plan_block(lam, Pm, Dm, theta, N, B, C, coeffs, prices, separate, **sli):
-    tau_mix, tau_solo = lp.nominal_taus(coeffs, B, C)
-    plan = lp.solve_plan(lam, Pm, Dm, theta, B, C, tau_mix, tau_solo, prices[0], prices[1],
-                         separate=separate, **sli)
+    def solve(tm, ts):
+        return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate, **sli)
+
+    start = None
+    if sli:
+        # SLI rows can be infeasible under the slow full-batch constants: settle the constants on the
+        # unconstrained plan first, then iterate with the constraints
+        def relaxed(tm, ts):
+            return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate)
+        tm0, ts0, _ = lp.consistent_taus(coeffs, B, C, relaxed)
+        start = (tm0, ts0)
+    tau_mix, tau_solo, plan = lp.consistent_taus(coeffs, B, C, solve, start=start)
     _, mu_m, mu_s = lp.service_rates(Pm, Dm, C, tau_mix, tau_solo)
     return plan, plan.M(N), plan.p_solo(mu_m, mu_s)
 
@@ -84,8 +94,39 @@ def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, 
 
 
 def _capacity(pi, Pm, Dm, B, C, coeffs):
-    tau_mix, tau_solo = lp.nominal_taus(coeffs, B, C)
-    return lp.fluid_capacity(pi, Pm, Dm, B, C, tau_mix, tau_solo)
+    return _capacity_cached(tuple(map(float, pi)), tuple(map(float, Pm)), tuple(map(float, Dm)), int(B), int(C),
+                            tuple(map(float, coeffs)))
+
+
+@functools.lru_cache(maxsize=None)
+def _capacity_cached(pi, Pm, Dm, B, C, coeffs):
+    """Fluid capacity: the largest total per-GPU rate s with lambda = s*pi servable without queues, the
+    iteration times being those of the batches that this load itself induces (bisection on s)."""
+    pi = np.asarray(pi, float)
+    coeffs = np.asarray(coeffs, float)
+    w = np.asarray(Pm, float) + np.asarray(Dm, float)      # any positive weights: the question is feasibility
+
+    def served_all(s):
+        lam = s * pi
+        def solve(tm, ts):
+            return lp.solve_plan(lam, Pm, Dm, np.zeros(len(pi)), B, C, tm, ts, 1.0, 1.0)
+        _, _, plan = lp.consistent_taus(coeffs, B, C, solve)
+        return plan.value >= float(np.dot(lam, w)) * (1.0 - 1e-7)
+
+    tm, ts = lp.nominal_taus(coeffs, B, C)
+    lo = lp.fluid_capacity(pi, Pm, Dm, B, C, tm, ts)       # full batches are the slowest: a safe lower bound
+    if coeffs[2] == 0.0 and coeffs[4] == 0.0:
+        return lo
+    hi = lo
+    while served_all(hi):
+        lo, hi = hi, hi * 1.5
+    for _ in range(40):
+        mid = 0.5 * (lo + hi)
+        if served_all(mid):
+            lo = mid
+        else:
+            hi = mid
+    return lo
 
 
 def cfg0(placement=PLACE_LEAST_LOADED, R=16, horizon_iters=10_000) -> SimInputs:
@@ -105,7 +146,7 @@ _LN2CLASS = (((5.0, 0.5), (6.0, 0.5)), ((7.5, 0.6), (4.0, 0.5)))
 
 def cfg1(placement=PLACE_LEAST_LOADED, R=1024, horizon_iters=100_000) -> SimInputs:
     """Two lognormal classes, N=64, B=128, separate pricing (0.5, 1.5), 0.9 of fluid capacity."""
-    tabs = lognormal_tables(_LN2CLASS)
+    tabs = _two_class_tables()
     Pm = [table_mean(tabs[i, 0]) for i in range(2)]
     Dm = [table_mean(tabs[i, 1]) for i in range(2)]
     pi = np.array([0.5, 0.5])
@@ -123,10 +164,19 @@ _OUT_MED = (512, 256, 128, 32)
 _MIX4 = np.array([0.4, 0.3, 0.2, 0.1])
 
 
+@functools.lru_cache(maxsize=None)
+def _two_class_tables():
+    tabs = lognormal_tables(_LN2CLASS)
+    tabs.setflags(write=False)
+    return tabs
+
+
+@functools.lru_cache(maxsize=None)
 def _four_class():
     tabs = lognormal_tables([((math.log(a), 0.7), (math.log(b), 0.7)) for a, b in zip(_IN_MED, _OUT_MED)])
     Pm = [table_mean(tabs[i, 0]) for i in range(4)]
     Dm = [table_mean(tabs[i, 1]) for i in range(4)]
+    tabs.setflags(write=False)
     return tabs, Pm, Dm
 
 

@@ -72,8 +72,8 @@ def test_cfg1_subset_lognormal_tables_priority_gate():
 
 
 def test_cfg2_subset_overload_with_abandonment():
-    inp = presets.cfg2(N=512, R=3)
-    st = check(inp, 400)
+    check(presets.cfg2(N=512, R=3), 400)
+    st = check(presets.cfg2(N=64, R=4), 4000)
     assert st["abandoned_p"].sum() > 0
 
 
