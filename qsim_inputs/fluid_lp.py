@@ -37,11 +37,16 @@ def nominal_taus(coeffs: Sequence[float], B: int, C: int) -> tuple[float, float]
     return iteration_time(coeffs, C, B - 1), iteration_time(coeffs, 0, B)
 
 
-def service_rates(P, D, C: int, tau_mix: float, tau_solo: float):
-    """Eq. (4)."""
+def service_rates(P, D, C: int, tau_mix: float, tau_solo: float, beta=None, nchunks=None):
+    """Eq. (4).  With `nchunks` (mean number of prefill iterations per request, E ceil(P/C)) and the
+    per-token slope `beta`, the prefill rate accounts for chunking: a request then spends
+    nchunks * (tau_mix - beta C) + beta P in prefill, which equals (P/C) tau_mix when P is a multiple of C."""
     P = np.asarray(P, float)
     D = np.asarray(D, float)
-    mu_p = C / (P * tau_mix)
+    if nchunks is None:
+        mu_p = C / (P * tau_mix)
+    else:
+        mu_p = 1.0 / (np.asarray(nchunks, float) * (tau_mix - beta * C) + beta * P)
     mu_m = 1.0 / (D * tau_mix)
     mu_s = (1.0 / tau_solo) / D
     return mu_p, mu_m, mu_s
@@ -77,7 +82,7 @@ def consistent_taus(coeffs, B: int, C: int, solve, iters: int = 40, tol: float =
     return tm, ts, plan
 
 
-def fluid_capacity(pi, P, D, B: int, C: int, tau_mix: float, tau_solo: float) -> float:
+def fluid_capacity(pi, P, D, B: int, C: int, tau_mix: float, tau_solo: float, beta=None, nchunks=None) -> float:
     """Largest total per-GPU arrival rate s such that lambda = s*pi is servable with empty queues.
 
     From the capacity and flow-balance rows of Eq. (36) with theta = 0, q = 0:
@@ -86,8 +91,9 @@ def fluid_capacity(pi, P, D, B: int, C: int, tau_mix: float, tau_solo: float) ->
     y_m + y_s/kappa' ... which gives s <= kB / (a + (kB - (B-1)) b), k = tau_mix/tau_solo.
     """
     pi = np.asarray(pi, float)
+    mu_p, _, _ = service_rates(P, D, C, tau_mix, tau_solo, beta, nchunks)
     a = tau_mix * float(np.dot(pi, D))
-    b = (tau_mix / C) * float(np.dot(pi, P))
+    b = float(np.sum(pi / mu_p))
     k = tau_mix / tau_solo
     return min(1.0 / b, k * B / (a + (k * B - (B - 1)) * b))
 
@@ -123,7 +129,8 @@ def solve_plan(lam, P, D, theta, B: int, C: int, tau_mix: float, tau_solo: float
                prefill_fair: Optional[float] = None,
                decode_fair: Optional[float] = None,
                min_admit_ratio: Optional[float] = None,
-               max_prefill_wait: Optional[float] = None) -> Plan:
+               max_prefill_wait: Optional[float] = None,
+               beta=None, nchunks=None) -> Plan:
     """Solve Eq. (36) (or its Eq. (38) objective) with optional SLI rows.
 
     Variable order: x[0:I], ym[I:2I], ys[2I:3I], qp[3I:4I], qd[4I:5I].
@@ -138,13 +145,13 @@ def solve_plan(lam, P, D, theta, B: int, C: int, tau_mix: float, tau_solo: float
     D = np.asarray(D, float)
     theta = np.asarray(theta, float)
     I = len(lam)
-    mu_p, mu_m, mu_s = service_rates(P, D, C, tau_mix, tau_solo)
+    mu_p, mu_m, mu_s = service_rates(P, D, C, tau_mix, tau_solo, beta, nchunks)
     nv = 5 * I
     ix, iym, iys, iqp, iqd = (slice(k * I, (k + 1) * I) for k in range(5))
 
     c = np.zeros(nv)
     if separate:
-        c[ix] = c_p * C / tau_mix
+        c[ix] = c_p * P * mu_p          # = c_p C / tau_mix under Eq. (4)
         c[iym] = c_d / tau_mix
         c[iys] = c_d / tau_solo
     else:
@@ -193,7 +200,7 @@ def solve_plan(lam, P, D, theta, B: int, C: int, tau_mix: float, tau_solo: float
             r = row(); r[ix.start + i] = -mu_p[i]; A_ub.append(r); b_ub.append(-min_admit_ratio * lam[i])
     if max_prefill_wait is not None:
         for i in range(I):
-            slack = max(max_prefill_wait - P[i] * tau_mix / C, 0.0)
+            slack = max(max_prefill_wait - 1.0 / mu_p[i], 0.0)
             r = row(); r[iqp.start + i] = 1.0; r[ix.start + i] = -slack * mu_p[i]
             A_ub.append(r); b_ub.append(0.0)
 

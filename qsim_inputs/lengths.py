@@ -56,3 +56,9 @@ def lognormal_tables(params) -> np.ndarray:
         for kind, (mu, sigma) in enumerate(pair):
             out[i, kind] = thresholds_from_cdf(lognormal_cdf_int(mu, sigma))
     return np.ascontiguousarray(out)
+
+
+def table_mean_chunks(thr: np.ndarray, C: int) -> float:
+    """E ceil(len / C): mean number of prefill iterations of a request drawn from the table."""
+    k = np.arange(1, LMAX + 1, dtype=np.float64)
+    return float(np.dot(np.ceil(k / C), table_pmf(thr)))

@@ -13,7 +13,7 @@ import math
 import numpy as np
 
 from . import fluid_lp as lp
-from .lengths import lognormal_tables, table_mean
+from .lengths import lognormal_tables, table_mean, table_mean_chunks
 from .spec import (GATE_OCCUPANCY, GATE_PRIORITY, LENGTH_FIXED, LENGTH_TABLE, PLACE_LEAST_LOADED,
                    PLACE_RANDOM, PRICING_BUNDLED, PRICING_SEPARATE, ROUTER_SLI, ROUTER_SOLO_FIRST,
                    SimInputs)
@@ -37,27 +37,30 @@ def _next_pow2(v: float) -> int:
     return 1 << max(0, int(math.ceil(math.log2(max(v, 1.0)))))
 
 
-def _plan_block(lam, Pm, Dm, theta, N, B, C, coeffs, prices, separate, **sli):
+def _plan_block(lam, Pm, Dm, theta, N, B, C, coeffs, prices, separate, nchunks=None, **sli):
+    ck = dict(beta=float(coeffs[1]), nchunks=nchunks) if nchunks is not None else {}
+
     def solve(tm, ts):
-        return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate, **sli)
+        return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate, **sli, **ck)
 
     start = None
     if sli:
         # SLI rows can be infeasible under the slow full-batch constants: settle the constants on the
         # unconstrained plan first, then iterate with the constraints
         def relaxed(tm, ts):
-            return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate)
+            return lp.solve_plan(lam, Pm, Dm, theta, B, C, tm, ts, prices[0], prices[1], separate=separate, **ck)
         tm0, ts0, _ = lp.consistent_taus(coeffs, B, C, relaxed)
         start = (tm0, ts0)
     tau_mix, tau_solo, plan = lp.consistent_taus(coeffs, B, C, solve, start=start)
-    _, mu_m, mu_s = lp.service_rates(Pm, Dm, C, tau_mix, tau_solo)
+    _, mu_m, mu_s = lp.service_rates(Pm, Dm, C, tau_mix, tau_solo, **ck)
     return plan, plan.M(N), plan.p_solo(mu_m, mu_s)
 
 
 def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, router, placement,
           pricing, lengths=None, P_fixed=None, D_fixed=None, seed=0, hist=0, block_len=0.0,
-          qcap=None, sli=None, horizon_iters=0) -> SimInputs:
-    """Plan every block and assemble a SimInputs.  Pm/Dm are the class mean lengths the LP uses."""
+          qcap=None, sli=None, horizon_iters=0, nchunks=None) -> SimInputs:
+    """Plan every block and assemble a SimInputs.  Pm/Dm are the class mean lengths the LP uses; nchunks
+    (mean prefill iterations per request) makes the planned prefill rate chunk-aware."""
     lam_blocks = np.atleast_2d(np.asarray(lam_blocks, float))
     nblk, I = lam_blocks.shape
     theta = np.asarray(theta, float)
@@ -67,7 +70,7 @@ def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, 
     values, plans = [], []
     for b in range(nblk):
         plan, Mb, p_solo = _plan_block(lam_blocks[b], Pm, Dm, theta, N, B, C, coeffs, prices,
-                                       pricing == PRICING_SEPARATE, **sli)
+                                       pricing == PRICING_SEPARATE, nchunks=nchunks, **sli)
         M[b] = Mb
         xs[b] = plan.x; nx[b] = N * plan.x; nq[b] = N * plan.qp; ps[b] = p_solo
         values.append(plan.value)
@@ -93,28 +96,29 @@ def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, 
     return inp
 
 
-def _capacity(pi, Pm, Dm, B, C, coeffs):
+def _capacity(pi, Pm, Dm, B, C, coeffs, nchunks=None):
     return _capacity_cached(tuple(map(float, pi)), tuple(map(float, Pm)), tuple(map(float, Dm)), int(B), int(C),
-                            tuple(map(float, coeffs)))
+                            tuple(map(float, coeffs)), None if nchunks is None else tuple(map(float, nchunks)))
 
 
 @functools.lru_cache(maxsize=None)
-def _capacity_cached(pi, Pm, Dm, B, C, coeffs):
+def _capacity_cached(pi, Pm, Dm, B, C, coeffs, nchunks):
     """Fluid capacity: the largest total per-GPU rate s with lambda = s*pi servable without queues, the
     iteration times being those of the batches that this load itself induces (bisection on s)."""
     pi = np.asarray(pi, float)
     coeffs = np.asarray(coeffs, float)
     w = np.asarray(Pm, float) + np.asarray(Dm, float)      # any positive weights: the question is feasibility
+    ck = dict(beta=float(coeffs[1]), nchunks=np.asarray(nchunks, float)) if nchunks is not None else {}
 
     def served_all(s):
         lam = s * pi
         def solve(tm, ts):
-            return lp.solve_plan(lam, Pm, Dm, np.zeros(len(pi)), B, C, tm, ts, 1.0, 1.0)
+            return lp.solve_plan(lam, Pm, Dm, np.zeros(len(pi)), B, C, tm, ts, 1.0, 1.0, **ck)
         _, _, plan = lp.consistent_taus(coeffs, B, C, solve)
         return plan.value >= float(np.dot(lam, w)) * (1.0 - 1e-7)
 
     tm, ts = lp.nominal_taus(coeffs, B, C)
-    lo = lp.fluid_capacity(pi, Pm, Dm, B, C, tm, ts)       # full batches are the slowest: a safe lower bound
+    lo = lp.fluid_capacity(pi, Pm, Dm, B, C, tm, ts, **ck)  # full batches are the slowest: a safe lower bound
     if coeffs[2] == 0.0 and coeffs[4] == 0.0:
         return lo
     hi = lo
@@ -149,9 +153,10 @@ def cfg1(placement=PLACE_LEAST_LOADED, R=1024, horizon_iters=100_000) -> SimInpu
     tabs = _two_class_tables()
     Pm = [table_mean(tabs[i, 0]) for i in range(2)]
     Dm = [table_mean(tabs[i, 1]) for i in range(2)]
+    nch = [table_mean_chunks(tabs[i, 0], 256) for i in range(2)]
     pi = np.array([0.5, 0.5])
-    s = _capacity(pi, Pm, Dm, 128, 256, COEFFS_BENCH)
-    inp = build("cfg1", N=64, R=R, B=128, C=256, Pm=Pm, Dm=Dm, lam_blocks=0.9 * s * pi, theta=[0.0, 0.0],
+    s = _capacity(pi, Pm, Dm, 128, 256, COEFFS_BENCH, nch)
+    inp = build("cfg1", N=64, R=R, B=128, C=256, Pm=Pm, Dm=Dm, nchunks=nch, lam_blocks=0.9 * s * pi, theta=[0.0, 0.0],
                 prices=[0.5, 1.5], coeffs=COEFFS_BENCH, gate=GATE_PRIORITY, router=ROUTER_SOLO_FIRST,
                 placement=placement, pricing=PRICING_SEPARATE, lengths=tabs, seed=1, qcap=4096,
                 horizon_iters=horizon_iters)
@@ -176,15 +181,16 @@ def _four_class():
     tabs = lognormal_tables([((math.log(a), 0.7), (math.log(b), 0.7)) for a, b in zip(_IN_MED, _OUT_MED)])
     Pm = [table_mean(tabs[i, 0]) for i in range(4)]
     Dm = [table_mean(tabs[i, 1]) for i in range(4)]
+    nch = [table_mean_chunks(tabs[i, 0], 256) for i in range(4)]
     tabs.setflags(write=False)
-    return tabs, Pm, Dm
+    return tabs, Pm, Dm, nch
 
 
 def cfg2(N=512, placement=PLACE_LEAST_LOADED, R=4096, horizon_iters=100_000) -> SimInputs:
     """Four lognormal classes at 1.05 of fluid capacity (patience 0.1/s so the excess leaves), bundled."""
-    tabs, Pm, Dm = _four_class()
-    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH)
-    inp = build("cfg2", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, lam_blocks=1.05 * s * _MIX4,
+    tabs, Pm, Dm, nch = _four_class()
+    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH, nch)
+    inp = build("cfg2", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, nchunks=nch, lam_blocks=1.05 * s * _MIX4,
                 theta=[0.1] * 4, prices=[1.0, 2.0], coeffs=COEFFS_BENCH, gate=GATE_OCCUPANCY,
                 router=ROUTER_SOLO_FIRST, placement=placement, pricing=PRICING_BUNDLED, lengths=tabs,
                 seed=2, horizon_iters=horizon_iters)
@@ -194,10 +200,10 @@ def cfg2(N=512, placement=PLACE_LEAST_LOADED, R=4096, horizon_iters=100_000) -> 
 
 def cfg3(N=1024, placement=PLACE_LEAST_LOADED, R=2048, block_len=3600.0, nblk=24) -> SimInputs:
     """Time-varying demand: 24 blocks, sinusoid of amplitude 0.5 around 0.95 of capacity, per-block LP tables."""
-    tabs, Pm, Dm = _four_class()
-    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH)
+    tabs, Pm, Dm, nch = _four_class()
+    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH, nch)
     lam = np.array([s * _MIX4 * (0.95 + 0.5 * math.sin(2.0 * math.pi * b / 24.0)) for b in range(nblk)])
-    inp = build("cfg3", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, lam_blocks=lam, theta=[0.1] * 4,
+    inp = build("cfg3", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, nchunks=nch, lam_blocks=lam, theta=[0.1] * 4,
                 prices=[0.5, 1.5], coeffs=COEFFS_BENCH, gate=GATE_PRIORITY, router=ROUTER_SOLO_FIRST,
                 placement=placement, pricing=PRICING_SEPARATE, lengths=tabs, seed=3, hist=1,
                 block_len=block_len)
@@ -208,9 +214,9 @@ def cfg3(N=1024, placement=PLACE_LEAST_LOADED, R=2048, block_len=3600.0, nblk=24
 
 def cfg4(N=1024, placement=PLACE_LEAST_LOADED, R=8192, horizon_iters=100_000) -> SimInputs:
     """cfg2 workload under constrained-LP targets with the SLI-aware randomized router."""
-    tabs, Pm, Dm = _four_class()
-    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH)
-    inp = build(f"cfg4_N{N}", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, lam_blocks=1.05 * s * _MIX4,
+    tabs, Pm, Dm, nch = _four_class()
+    s = _capacity(_MIX4, Pm, Dm, 256, 256, COEFFS_BENCH, nch)
+    inp = build(f"cfg4_N{N}", N=N, R=R, B=256, C=256, Pm=Pm, Dm=Dm, nchunks=nch, lam_blocks=1.05 * s * _MIX4,
                 theta=[0.1] * 4, prices=[1.0, 2.0], coeffs=COEFFS_BENCH, gate=GATE_OCCUPANCY,
                 router=ROUTER_SLI, placement=placement, pricing=PRICING_BUNDLED, lengths=tabs, seed=4,
                 hist=1, sli=dict(qd_zero=True, min_admit_ratio=0.8, max_prefill_wait=2.0),
