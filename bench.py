@@ -1,0 +1,285 @@
+#!/usr/bin/env python
+"""Benchmark: simulated GPU-server-iterations per second on the two-class lognormal workload (cfg1).
+
+One step = one pass of the whole hot path (arrivals, next-event selection, iteration completion,
+accounting, decode routing, prefill gate, abandonment clocks, iteration starts, state staging) over one
+batch: all R = 1024 replications of N = 64 simulated GPUs advance by 10^5 iterations of horizon.  Steps
+continue the same simulation, so the timed steps run in steady state.
+
+    python bench.py --gpus N --steps K --warmup W          (N > 1: launched under torchrun, one rank per GPU)
+    python bench.py --impl reference ...                   (the CPU oracle, timed on the host cores)
+
+Prints one JSON line.  `value` is timed with CUDA events around qsim_run with all state resident in HBM;
+`e2e` is the same metric through qsim_simulate with host buffers (tables copied in, statistics copied out,
+device memory allocated and freed inside the timed region).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "simulated GPU-server-iterations/sec"
+UNIT = "server-iterations/s"
+JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
+                           # decode-buffer pass, each written and read once at 32-byte sector granularity
+HORIZON = 100_000          # iterations of horizon per step (cfg1)
+R_PER_GPU = 1024
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "200"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_throughput(inp, horizon_iters: int, n_reps: int, n_threads: int):
+    """The CPU oracle as it stands, one replication per thread (the C code runs without the GIL)."""
+    from oracle import OracleSim, build_oracle
+    build_oracle()
+    iters = [0] * n_reps
+    nxt = [0]
+    lock = threading.Lock()
+
+    def work():
+        while True:
+            with lock:
+                r = nxt[0]
+                nxt[0] += 1
+            if r >= n_reps:
+                return
+            sim = OracleSim(inp.with_(R=1, rep_offset=inp.rep_offset + r))
+            sim.run(horizon_iters)
+            st = sim.stats()
+            iters[r] = int(st["iters_mixed"].sum() + st["iters_solo"].sum())
+            sim.close()
+
+    t0 = time.perf_counter()
+    threads = [threading.Thread(target=work) for _ in range(min(n_threads, n_reps))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    dt = time.perf_counter() - t0
+    return sum(iters) / dt, sum(iters), dt
+
+
+def run_reference(args, workload):
+    from qsim_inputs import presets
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    inp = presets.cfg1(R=R_PER_GPU)
+    # bounded sample of the workload per step: one replication per core, 2000 iterations of horizon each
+    h_sample, n_reps = 2000, cores
+    vals, ms = [], []
+    for s in range(args.warmup + args.steps):
+        v, iters, dt = oracle_throughput(inp.with_(rep_offset=s * n_reps), h_sample, n_reps, cores)
+        if s >= args.warmup:
+            vals.append(v); ms.append(dt * 1e3)
+    value = sum(vals) / len(vals)
+    sample = f"{n_reps} replications x {h_sample} iterations of horizon of {workload} per step, one per thread"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sum(ms) / len(ms), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="qsim", choices=["qsim", "reference"])
+    ap.add_argument("--horizon", type=int, default=HORIZON, help="iterations of horizon per step")
+    ap.add_argument("--reps", type=int, default=R_PER_GPU, help="replications per GPU")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    workload = (f"cfg1: 2 lognormal classes, N=64 GPUs, B=128, C=256, separate pricing, priority gate, solo-first "
+                f"router, least-loaded placement, R={args.reps} replications per GPU, {args.horizon} iterations "
+                f"of horizon per step")
+    if args.impl == "reference":
+        run_reference(args, workload)
+        return
+    if args.warmup < 3:
+        args.warmup = 3
+
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02987_b200 import QSim, simulate_host
+    from qsim_inputs import presets
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the simulator has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # replications are independent: rank k simulates global replications [k R, (k+1) R)  (weak scaling)
+    inp = presets.cfg1(R=args.reps).with_(rep_offset=rank * args.reps)
+    sim = QSim(inp, device=f"cuda:{local}")
+    for _ in range(args.warmup):
+        sim.run(args.horizon)
+    it0, ev0, tot0 = sim.totals()
+    jobs0 = sum(int(tot0.cls[i].done_mixed + tot0.cls[i].done_solo) for i in range(inp.I))
+    launches0 = sim.launch_count()
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_wall0 = time.perf_counter()
+    for a, b in evs:
+        a.record()
+        sim.run(args.horizon)
+        b.record()
+    barrier()
+    wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    it1, ev1, tot1 = sim.totals()
+    jobs1 = sum(int(tot1.cls[i].done_mixed + tot1.cls[i].done_solo) for i in range(inp.I))
+    launches = sim.launch_count() - launches0
+    overflow = sum(int(tot1.cls[i].overflow + tot1.cls[i].overflow_d) for i in range(inp.I))
+    my = torch.tensor([sum(step_ms), float(it1 - it0), float(ev1 - ev0), float(jobs1 - jobs0), float(launches),
+                       float(overflow)], dtype=torch.float64, device="cuda")
+    tmax = my[:1].clone()
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        dist.all_reduce(my[1:], op=dist.ReduceOp.SUM)
+    total_ms = float(tmax[0])
+    iters, events, jobs, n_launch, ovf = (float(x) for x in my[1:])
+    value = iters / (total_ms * 1e-3)
+
+    # end to end through the host-buffer entry point (fresh system each step)
+    e2e = None
+    if not args.no_e2e:
+        e_iters, e_t = 0.0, 0.0
+        h2d = int(inp.lengths.nbytes + inp.rates.nbytes + 8 * 6 + 8 * 2 + inp.nblk * 264 + inp.I * 24 + 80)
+        d2h = 0
+        simulate_host(inp.with_(R=8), 200)   # warm the context and allocator paths
+        barrier()
+        for _ in range(args.steps):
+            t0 = time.perf_counter()
+            st = simulate_host(inp, args.horizon)
+            e_t += time.perf_counter() - t0
+            e_iters += float(st["iters_mixed"].sum() + st["iters_solo"].sum())
+            d2h = int(sim.workspace_bytes * 0) + inp.R * 4224
+        ev = torch.tensor([e_t, e_iters], dtype=torch.float64, device="cuda")
+        tm = ev[:1].clone()
+        if world > 1:
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            dist.all_reduce(ev[1:], op=dist.ReduceOp.SUM)
+        e2e = {"value": float(ev[1]) / float(tm[0]), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h}
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        # algorithmic HBM bytes of one launch of the dominant kernel (qsim_run_kernel): the server state is
+        # resident in shared memory, so what must move is the request life cycle plus the state staging
+        stage = 2.0 * inp.R * (4224 + 48 * ((inp.N + 31) // 32 * 32))
+        alg_bytes_per_launch = (JOB_BYTES * jobs / world + stage * args.steps) / max(n_launch / world, 1.0)
+        kernel_ms = total_ms / max(n_launch / world, 1.0)
+        achieved = alg_bytes_per_launch / (kernel_ms * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload, "l2": "state larger than L2 (workspace %.0f MB per GPU)" % (sim.workspace_bytes / 1e6),
+                       "events_per_iteration": events / iters, "requests_per_iteration": jobs / iters,
+                       "queue_overflow": ovf},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_kind": peak_kind,
+                         "bytes_per_iteration": JOB_BYTES * jobs / iters,
+                         "note": "latency/issue-bound event chain; HBM fraction is the contract figure"},
+            "clocks": clocks, "gpu_launches": int(n_launch), "wall_s": wall,
+        }
+        if e2e:
+            out["e2e"] = e2e
+        if not args.no_cpu_baseline and world == 1:
+            cores = os.cpu_count() or 1
+            h_s = 3000
+            v, it_s, dt = oracle_throughput(inp, h_s, 2 * cores, cores)
+            out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                   "sample": f"{2 * cores} replications x {h_s} iterations of horizon of cfg1, one per thread, {dt:.1f} s"}
+        print(json.dumps(out))
+    sim.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
