@@ -179,6 +179,34 @@ int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const doubl
                   const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
                   qsim_rep_stats *per_rep);
 
+/*
+ * The same simulation as qsim_simulate for callers that must not allocate.  (The paper has no
+ * counterpart: this is a packaging variant of the library, not part of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin inside a serving process whose
+ * own allocator has already reserved the whole card, so a fresh cudaMalloc would fail or evict; a
+ * latency-critical section that cannot afford the device-wide synchronisation cudaMalloc / cudaFree
+ * imply; a host that forbids allocation after start-up.  This entry point calls no cudaMalloc, cudaFree,
+ * cudaMallocHost or any other allocating routine.  All simulation state, the rate/target table and
+ * the length tables live in one array that is compiled into the library: 32 MiB of device memory on
+ * every GPU that loads libqsim.so, held until the process exits.
+ *
+ * Arguments as in qsim_simulate ([host] inputs, [host] totals / per_rep[R] outputs, either may be NULL),
+ * plus cuda_stream (a cudaStream_t, NULL = default stream) on which the copies and kernels are ordered;
+ * the call returns after the stream has finished.  Histograms are not recorded (cfg.hist is ignored) and
+ * nblk must be <= 64.  If the problem needs more than the 32 MiB (state grows with R, N*B and qcap) the
+ * call fails with QSIM_EWORKSPACE and a message that states the bytes needed.
+ *
+ * The first call on each device looks up the array's device address; make that first call with the
+ * device current and outside any stream capture.  Every call on a device shares the one array: calls
+ * must not overlap on the GPU (two host threads, or two streams) or they corrupt each other.  Nothing
+ * needs clearing by the caller - each call re-initialises the state it uses.
+ */
+int qsim_simulate_static(const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                         const uint32_t *lengths, const double *prices, const double *iter_time_coeffs,
+                         const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
+                         qsim_rep_stats *per_rep, void *cuda_stream);
+
 /* Kernel launches issued by this handle so far (for accounting in benchmarks). */
 int qsim_launch_count(const qsim_t *h, uint64_t *launches);
 

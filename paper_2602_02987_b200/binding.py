@@ -18,7 +18,7 @@ _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_
 
 EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
-           "qsim_launch_count", "qsim_destroy", "qsim_last_error")
+           "qsim_simulate_static", "qsim_launch_count", "qsim_destroy", "qsim_last_error")
 
 
 class QSimError(RuntimeError):
@@ -77,6 +77,8 @@ def load_library():
         L.qsim_server_state.argtypes = [vp, C.c_uint32, vp, vp, vp, vp]
         L.qsim_simulate.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
                                     C.POINTER(qsim_targets), C.c_uint64, vp, vp]
+        L.qsim_simulate_static.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
+                                           C.POINTER(qsim_targets), C.c_uint64, vp, vp, vp]
         L.qsim_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.qsim_destroy.argtypes = [vp]
         L.qsim_last_error.restype = C.c_char_p
@@ -235,6 +237,22 @@ def simulate_host(inp, horizon_iters: int) -> dict:
     tot = qsim_rep_stats()
     _check(L.qsim_simulate(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
                            int(horizon_iters), C.byref(tot), per))
+    out = _unpack(per, inp.R, inp.I)
+    out["_totals"] = _unpack((tot,), 1, inp.I)
+    return out
+
+
+def simulate_static(inp, horizon_iters: int, stream=None) -> dict:
+    """qsim_simulate_static: like simulate_host, but the library allocates nothing; its state lives in a
+    32 MiB array built into libqsim.so, so only small problems fit (a QSimError names the bytes needed).
+    Meant for callers that may not call cudaMalloc; calls must not overlap on one GPU."""
+    L = load_library()
+    cfg, classes, rates, lengths, prices, coeffs, tg = marshal(inp)
+    per = (qsim_rep_stats * inp.R)()
+    tot = qsim_rep_stats()
+    sp = C.c_void_p(stream.cuda_stream) if stream is not None else None
+    _check(L.qsim_simulate_static(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
+                                  int(horizon_iters), C.byref(tot), per, sp))
     out = _unpack(per, inp.R, inp.I)
     out["_totals"] = _unpack((tot,), 1, inp.I)
     return out

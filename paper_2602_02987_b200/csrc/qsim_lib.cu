@@ -448,3 +448,122 @@ int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const doubl
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------
+// qsim_simulate_static: the whole simulation with no device or pinned-memory allocation at all.
+// State, tables and the completion flag live in one file-scope device array.  Host code never uses the
+// array's name as a pointer: its device address is asked for once per device (cudaGetSymbolAddress).
+// ---------------------------------------------------------------------------------------------------
+#define QSIM_STATIC_SCRATCH_BYTES (32u << 20)
+static __device__ __align__(256) unsigned char g_static_scratch[QSIM_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_ptr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                                    const uint32_t *lengths, const double *prices, const double *coef,
+                                    const qsim_targets *tg, uint64_t horizon_iters, qsim_rep_stats *totals,
+                                    qsim_rep_stats *per_rep, void *cuda_stream)
+{
+    int rc = validate(cfg, classes, rates, lengths, prices, coef, tg);
+    if (rc != QSIM_OK) return rc;
+    if (cfg->nblk > 64) return fail(QSIM_EINVAL, "qsim_simulate_static supports at most 64 blocks");
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(QSIM_EINVAL, "device index out of range");
+    if (!g_static_ptr[dev]) {
+        // first call on this device: resolve the device address of the array (the current device is `dev`)
+        void *ptr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        g_static_ptr[dev] = ptr;
+    }
+    char *base = static_cast<char *>(g_static_ptr[dev]);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    qsim h;   // a handle that owns nothing: no table allocation, no pinned flag
+    h.cfg = *cfg;
+    h.cfg.hist = 0;
+    std::memcpy(h.cls, classes, cfg->I * sizeof(qsim_class));
+    h.prices[0] = prices[0];
+    h.prices[1] = prices[1];
+    h.device = dev;
+    h.stream = stream;
+    Params &p = h.par;
+    p.I = cfg->I; p.N = cfg->N; p.Npad = (cfg->N + 31u) & ~31u; p.R = cfg->R; p.B = cfg->B; p.C = cfg->C;
+    p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
+    p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = 0;
+    p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
+    p.event_budget = 1ull << 40;
+    for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
+    for (uint32_t i = 0; i < cfg->I; ++i) {
+        p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
+        p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
+    }
+    h.lay = smem_layout(p.Npad);
+    p.srv_bytes = h.lay.srv_bytes;
+    if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
+    qsim_config nohist = *cfg;
+    nohist.hist = 0;
+    h.sec = layout_sections(nohist, p.srv_bytes);
+    // scratch = [state sections | block table | length tables]
+    const size_t off_blocks = h.sec.total;
+    const size_t off_lengths = align256(off_blocks + (size_t)cfg->nblk * sizeof(BlockPar));
+    const size_t len_bytes = cfg->length_mode == QSIM_LENGTH_TABLE ? (size_t)cfg->I * 2 * QSIM_LMAX * 4 : 0;
+    const size_t need = off_lengths + len_bytes;
+    if (need > QSIM_STATIC_SCRATCH_BYTES)
+        return fail(QSIM_EWORKSPACE, "qsim_simulate_static: this problem needs " + std::to_string(need) +
+                                         " bytes of state but the built-in scratch holds " +
+                                         std::to_string((size_t)QSIM_STATIC_SCRATCH_BYTES) +
+                                         "; reduce R, N*B or qcap, or use qsim_create/qsim_bind with your own workspace");
+    BlockPar blocks[64];
+    std::memset(blocks, 0, sizeof blocks);
+    for (uint32_t b = 0; b < cfg->nblk; ++b) {
+        blocks[b].M = tg[b].M;
+        for (uint32_t i = 0; i < cfg->I; ++i) {
+            blocks[b].xstar[i] = tg[b].xstar[i]; blocks[b].nx[i] = tg[b].n_xstar[i]; blocks[b].nq[i] = tg[b].n_qpstar[i];
+            blocks[b].ps[i] = tg[b].p_solo[i]; blocks[b].rate[i] = rates[(size_t)b * cfg->I + i];
+        }
+    }
+    // pageable sources: these copies have returned from the host buffers when the calls return
+    CUDA_TRY(cudaMemcpyAsync(base + off_blocks, blocks, (size_t)cfg->nblk * sizeof(BlockPar), cudaMemcpyHostToDevice, stream));
+    if (len_bytes) CUDA_TRY(cudaMemcpyAsync(base + off_lengths, lengths, len_bytes, cudaMemcpyHostToDevice, stream));
+    p.blocks = reinterpret_cast<const BlockPar *>(base + off_blocks);
+    p.lengths = len_bytes ? reinterpret_cast<const uint32_t *>(base + off_lengths) : nullptr;
+    p.hdr = reinterpret_cast<RepHeader *>(base + h.sec.hdr);
+    p.srv = base + h.sec.srv;
+    p.slot_fin = reinterpret_cast<uint32_t *>(base + h.sec.fin);
+    p.slot_tpf = reinterpret_cast<double *>(base + h.sec.tpf);
+    p.slot_pk = reinterpret_cast<uint32_t *>(base + h.sec.pk);
+    p.pq = reinterpret_cast<QEntry *>(base + h.sec.pq);
+    p.dq = reinterpret_cast<QEntry *>(base + h.sec.dq);
+    p.hist_mem = nullptr;
+    p.not_done = reinterpret_cast<uint32_t *>(base + h.sec.flag);
+    if (h.lay.total > 48u * 1024u) {
+        CUDA_TRY(cudaFuncSetAttribute(qsim_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.lay.total));
+        CUDA_TRY(cudaFuncSetAttribute(qsim_init_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.lay.total));
+    }
+    // the array keeps the previous call's contents: the init kernel rewrites every header and GPU image;
+    // queue rings and slot lists are never read before they are written, the flag is cleared per launch
+    qsim_init_kernel<<<cfg->R, 32, h.lay.total, stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    bool advance = true;
+    for (;;) {
+        Params q = p;
+        q.advance = advance ? 1u : 0u;
+        q.horizon_iters = advance ? horizon_iters : 0;
+        CUDA_TRY(cudaMemsetAsync(q.not_done, 0, 4, stream));
+        qsim_run_kernel<<<cfg->R, 32, h.lay.total, stream>>>(q);
+        CUDA_TRY(cudaGetLastError());
+        uint32_t left = 0;
+        CUDA_TRY(cudaMemcpyAsync(&left, q.not_done, 4, cudaMemcpyDeviceToHost, stream));
+        CUDA_TRY(cudaStreamSynchronize(stream));
+        if (left == 0) break;
+        advance = false;
+    }
+    h.bound = true;
+    rc = qsim_stats(&h, totals, per_rep, nullptr, nullptr);
+    h.bound = false;
+    return rc;
+}
