@@ -143,8 +143,9 @@ int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
  */
 int qsim_run(qsim_t *h, uint64_t horizon_iters);
 
-/* Upper bound on events one replication processes per kernel launch (default 2^40, i.e. one launch per
- * qsim_run); a replication that reaches it is continued by further launches with identical results. */
+/* Upper bound on the rounds (one non-local event plus the iteration ends before it) one replication
+ * processes per kernel launch (default 2^28); a replication that reaches it is continued by further
+ * launches with identical results. */
 int qsim_set_event_budget(qsim_t *h, uint64_t events_per_launch);
 
 /* Wait until all work queued on the handle's stream has finished; reports sticky replication errors. */

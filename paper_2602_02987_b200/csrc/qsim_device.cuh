@@ -1,4 +1,16 @@
-// Device side of qsim: one warp simulates one replication, event by event.
+// Device side of qsim: one warp simulates one replication.
+//
+// Look-ahead.  The end of an iteration on a simulated GPU touches nothing outside that GPU unless a request
+// finishes its prefill there (it must be routed, and the gate admits the next one) or a decode ends while
+// requests wait in a decode buffer (the freed slot must be refilled).  All other iteration ends are
+// "local".  A request placed on a running GPU only joins at that GPU's next iteration boundary, and no
+// iteration is shorter than tau_min = min(alpha_m, alpha_s).  So in every round the warp finds the next
+// non-local event (time T_int) and the earliest running iteration end T_min, and every lane finishes, in
+// parallel, the local iteration ends of its own GPUs that come before min(T_int, T_min + tau_min, T_end):
+// each GPU has at most one such end, and nothing that happens in that window can change another GPU's
+// batch.  Decode completions found on the way are then retired by the whole warp, GPU by GPU, and only
+// after that is the non-local event handled by the warp-wide path.  The outcome is event for event that of
+// the one-at-a-time order; only the order in which some sums are accumulated differs.
 //
 // Ownership inside the warp (no two lanes ever write the same word, so the only synchronisation is a
 // few __syncwarp per event):
@@ -45,7 +57,8 @@ struct ClassState {
     unsigned long long adraw, sli_ord;
     uint32_t ablk, nextP, nextD, pq_head, pq_n, X, Ym, Ys, Qd0, Qd1;
     AbClock abp, abd0, abd1;
-    Area aQp, aX, aQd, aYm, aYs;
+    Area aQp, aX, aQd;
+    double sYm_in, sYm_out, sYs_in, sYs_out;   // sums of (placement / completion time - T_reset): integral of Y = out - in + Y (T - T_reset)
     unsigned long long arrivals, admitted, prefill_done, placed_mixed, placed_solo, done_mixed, done_solo,
         abandoned_p, abandoned_d, overflow, overflow_d, tok_in_pf, tok_in_done, tok_out_done;
     double sum_ttft, sum_tpot;
@@ -240,7 +253,7 @@ struct Sim {
     QEntry *pq, *dq;
     uint32_t *hist;
     // replicated scalars
-    double t, T_end, T_blk_next;
+    double t, T_end, T_blk_next, T_reset, tau_min;
     uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
     unsigned long long place_ord, events;
     bool drain_dirty, gate_dirty, touch_all;
@@ -471,8 +484,9 @@ struct Sim {
             ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd - 1, t);
             area_touch(c.aQd, c.Qd0 + c.Qd1, t);
             if (pool) c.Qd1--; else c.Qd0--;
-            if (mixed) { area_touch(c.aYm, c.Ym, t); c.Ym++; c.placed_mixed++; }
-            else       { area_touch(c.aYs, c.Ys, t); c.Ys++; c.placed_solo++; }
+            const double rel = __dsub_rn(t, T_reset);
+            if (mixed) { c.sYm_in = __dadd_rn(c.sYm_in, rel); c.Ym++; c.placed_mixed++; }
+            else       { c.sYs_in = __dadd_rn(c.sYs_in, rel); c.Ys++; c.placed_solo++; }
         }
         if (lane == (int)(g & 31u)) {
             const uint32_t sl = ndec[g];
@@ -540,23 +554,28 @@ struct Sim {
         touch_server(g);
     }
 
-    __device__ __forceinline__ void start_if_needed(uint32_t g)
+    // Called by the owner: a GPU with work that is between iterations starts one at time ts.  The batch
+    // (prefill chunk, decodes) is frozen here for the whole iteration, and with it what its end will bring:
+    // bit 14 of nact = some decode emits its last token, bit 15 = the prefill finishes.
+    __device__ __forceinline__ void start_at(uint32_t g, double ts)
     {
-        // called by the owner: a GPU with work that is between iterations starts one now;
-        // the batch (prefill chunk, decodes) is frozen here for the whole iteration
         if (!(tnext[g] < dinf())) {
             const uint32_t nd = ndec[g];
             const uint32_t pj = pfjob[g];
             if (nd > 0 || (pj >> 31)) {
-                const uint32_t Kg = K[g] + Kpend[g];
-                K[g] = Kg; Kpend[g] = 0;
-                nact[g] = (uint16_t)nd;
-                const uint32_t pc = (pj >> 31) ? min(p.C, pfrem[g]) : 0u;
+                uint32_t Kg = 0;
+                if (p.coef[5] != 0.0) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
+                const uint32_t rem = pfrem[g];
+                const uint32_t pc = (pj >> 31) ? min(p.C, rem) : 0u;
                 pfcur[g] = (uint16_t)pc;
-                tnext[g] = __dadd_rn(t, iter_time(p, pc, nd, Kg));
+                uint32_t fl = (nfin[g] == it[g] + 1u) ? 0x4000u : 0u;
+                if (pc > 0 && pc == rem) fl |= 0x8000u;
+                nact[g] = (uint16_t)(nd | fl);
+                tnext[g] = __dadd_rn(ts, iter_time(p, pc, nd, Kg));
             }
         }
     }
+    __device__ __forceinline__ void start_if_needed(uint32_t g) { start_at(g, t); }
 
     __device__ void dispatch()
     {
@@ -616,7 +635,58 @@ struct Sim {
         touch_all = false;
     }
 
-    // --- end of an iteration on GPU g ------------------------------------------------------------
+    // Some decode on GPU g emitted its last token in the iteration that ended at te (its it-th): the whole
+    // warp scans the GPU's slot list from the tail, accounts every finished request and closes the gaps.
+    __device__ void retire_decodes(uint32_t g, uint32_t itg, uint32_t nd, double te)
+    {
+        const int owner = (int)(g & 31u);
+        uint32_t n = nd, newmin = NONE32, Kdrop = 0;
+        const size_t base = (size_t)g * p.B;
+        for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
+            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
+            const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
+            const bool hit = f == itg;
+            if (!hit) newmin = min(newmin, f);
+            uint32_t hits = __ballot_sync(FULL, hit);
+            while (hits) {
+                const int hl = 31 - __clz(hits);
+                hits &= ~(1u << hl);
+                const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
+                const double tpf = s_tpf[base + h];
+                const uint32_t pk = s_pk[base + h];
+                const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
+                if (lane == (int)i) {
+                    ClassState &c = cs[i];
+                    const double rel = __dsub_rn(te, T_reset);
+                    if (job_flag(pk)) { c.sYm_out = __dadd_rn(c.sYm_out, rel); c.Ym--; c.done_mixed++; }
+                    else              { c.sYs_out = __dadd_rn(c.sYs_out, rel); c.Ys--; c.done_solo++; }
+                    c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
+                    c.tok_out_done += D;
+                    const double tpot = __ddiv_rn(__dsub_rn(te, tpf), (double)D);
+                    c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
+                    if (hist) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
+                }
+                Kdrop += P + D;
+                const uint32_t last = n - 1;
+                __syncwarp();
+                if (lane == 0 && h != last) {
+                    s_fin[base + h] = s_fin[base + last];
+                    s_tpf[base + h] = s_tpf[base + last];
+                    s_pk[base + h] = s_pk[base + last];
+                }
+                n = last;
+            }
+        }
+        newmin = __reduce_min_sync(FULL, newmin);
+        if (lane == owner) {
+            ndec[g] = (uint16_t)n;
+            nfin[g] = newmin;
+            K[g] -= Kdrop;
+        }
+        __syncwarp();
+    }
+
+    // --- end of an iteration on GPU g (warp-wide path: the end is not local) ----------------------
     __device__ void on_server(uint32_t g)
     {
         const int owner = (int)(g & 31u);
@@ -624,7 +694,7 @@ struct Sim {
         if (lane == owner) {
             itg = it[g] + 1;
             it[g] = itg;
-            const uint32_t na = nact[g], pc = pfcur[g], Kg = K[g];
+            const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = K[g];
             const double tau = iter_time(p, pc, na, Kg);
             if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
@@ -641,51 +711,9 @@ struct Sim {
         }
         flags = __shfl_sync(FULL, flags, owner);
         if (flags & 1u) {
-            // some decode emitted its last token: scan the GPU's slot list from the tail, close the gaps
             itg = __shfl_sync(FULL, itg, owner);
             nd = __shfl_sync(FULL, nd, owner);
-            uint32_t n = nd, newmin = NONE32, Kdrop = 0;
-            const size_t base = (size_t)g * p.B;
-            for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
-                const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
-                const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
-                const bool hit = f == itg;
-                if (!hit) newmin = min(newmin, f);
-                uint32_t hits = __ballot_sync(FULL, hit);
-                while (hits) {
-                    const int hl = 31 - __clz(hits);
-                    hits &= ~(1u << hl);
-                    const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
-                    const double tpf = s_tpf[base + h];
-                    const uint32_t pk = s_pk[base + h];
-                    const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
-                    if (lane == (int)i) {
-                        ClassState &c = cs[i];
-                        if (job_flag(pk)) { area_touch(c.aYm, c.Ym, t); c.Ym--; c.done_mixed++; }
-                        else              { area_touch(c.aYs, c.Ys, t); c.Ys--; c.done_solo++; }
-                        c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
-                        c.tok_out_done += D;
-                        const double tpot = __ddiv_rn(__dsub_rn(t, tpf), (double)D);
-                        c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
-                        if (hist) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
-                    }
-                    Kdrop += P + D;
-                    const uint32_t last = n - 1;
-                    __syncwarp();
-                    if (lane == 0 && h != last) {
-                        s_fin[base + h] = s_fin[base + last];
-                        s_tpf[base + h] = s_tpf[base + last];
-                        s_pk[base + h] = s_pk[base + last];
-                    }
-                    n = last;
-                }
-            }
-            newmin = __reduce_min_sync(FULL, newmin);
-            if (lane == owner) {
-                ndec[g] = (uint16_t)n;
-                nfin[g] = newmin;
-                K[g] -= Kdrop;
-            }
+            retire_decodes(g, itg, nd, t);
             drain_dirty = true;
             gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
         }
@@ -741,15 +769,37 @@ struct Sim {
         touch_server(g);
     }
 
-    // --- event loop ----------------------------------------------------------------------------------
+    // --- local end of an iteration (owner lane only) ----------------------------------------------------
+    // The iteration of GPU g ends at te and nothing outside g depends on it.  Returns true when a decode
+    // finished: the GPU then waits for retire_decodes before it starts its next iteration.
+    __device__ __forceinline__ bool local_end(uint32_t g, double te)
+    {
+        const uint32_t itg = it[g] + 1u;
+        it[g] = itg;
+        const uint32_t na_raw = nact[g], na = na_raw & 0x3fffu, pc = pfcur[g];
+        uint32_t Kg = 0;
+        if (p.coef[5] != 0.0) { Kg = K[g]; K[g] = Kg + na; }
+        const double tau = iter_time(p, pc, na, Kg);
+        if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] -= pc; }
+        else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
+        pfcur[g] = 0;
+        tnext[g] = dinf();
+        if (na_raw & 0x4000u) return true;
+        start_at(g, te);
+        return false;
+    }
+
+    // --- round loop ----------------------------------------------------------------------------------
     __device__ bool run()
     {
         const uint32_t rows = p.Npad >> 5;
+        const unsigned long long INF = 0x7ff0000000000000ull;
+        const unsigned long long tend_bits = (unsigned long long)__double_as_longlong(T_end);
         unsigned long long budget = p.event_budget;
         for (;;) {
             __syncwarp();
-            // earliest source of this lane; scanning in id order with '<' keeps the tie order
-            unsigned long long bt = 0x7ff0000000000000ull;
+            // next non-local event of this lane (sources scanned in id order with '<' keep the tie order)
+            unsigned long long bt = INF, tmin = INF;
             uint32_t bs = NONE32;
             if (lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
             if (lane < (int)p.I) {
@@ -763,40 +813,93 @@ struct Sim {
                 v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
                 if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
             }
+            const bool buffered = (dq_n0 | dq_n1) != 0;
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-                if (v < bt) { bt = v; bs = SRC_SERVER + g; }
+                if (v < INF) {
+                    tmin = min(tmin, v);
+                    if (!is_local(g, buffered) && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                }
             }
-            // warp argmin of (time bits, source id)
+            // warp argmin of (time bits, source id) over non-local events; warp min over all iteration ends
             const uint32_t hi = (uint32_t)(bt >> 32), lo = (uint32_t)bt;
             const uint32_t mhi = __reduce_min_sync(FULL, hi);
             const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : NONE32);
             const uint32_t src = __reduce_min_sync(FULL, (hi == mhi && lo == mlo) ? bs : NONE32);
-            const double te = __longlong_as_double((long long)(((unsigned long long)mhi << 32) | mlo));
-            if (src == NONE32 || te > T_end) return true;
+            const unsigned long long tint = ((unsigned long long)mhi << 32) | mlo;
+            const uint32_t th = (uint32_t)(tmin >> 32);
+            const uint32_t tmh = __reduce_min_sync(FULL, th);
+            const uint32_t tml = __reduce_min_sync(FULL, th == tmh ? (uint32_t)tmin : NONE32);
+            const unsigned long long tmin_all = ((unsigned long long)tmh << 32) | tml;
+            if (tint > tend_bits && tmin_all > tend_bits) return true;     // nothing left up to T_end
             if (budget == 0) return false;
             --budget;
-            ++events;
-            t = te;
-            if (src >= SRC_SERVER) {
-                on_server(src - SRC_SERVER);
-            } else if (src >= SRC_ABD1) {
-                on_abandon_d(1, src - SRC_ABD1);
-            } else if (src >= SRC_ABD0) {
-                on_abandon_d(0, src - SRC_ABD0);
-            } else if (src >= SRC_ABP) {
-                on_abandon_p(src - SRC_ABP);
-            } else if (src >= SRC_ARRIVAL) {
-                on_arrival(src - SRC_ARRIVAL);
-            } else {
-                load_block(blk + 1);
-                drain_dirty = true;
-                gate_dirty = true;
+            // no iteration that starts in this round can end before T_min + tau_min
+            unsigned long long wt = INF;
+            if (tmin_all < INF)
+                wt = (unsigned long long)__double_as_longlong(__dadd_rn(__longlong_as_double((long long)tmin_all), tau_min));
+            // local ends strictly before the limit key min{(T_int, src), (W, 0), (T_end, max)}
+            unsigned long long lim_t = tint;
+            uint32_t lim_s = src;
+            if (wt <= lim_t) { lim_t = wt; lim_s = 0; }
+            if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
+            uint32_t any_retire = 0;
+            bool progressed = false;
+            for (uint32_t k = 0; k < rows; ++k) {
+                const uint32_t g = (k << 5) + (uint32_t)lane;
+                const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+                bool retire = false;
+                if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+                    retire = local_end(g, __longlong_as_double((long long)v));
+                    progressed = true;
+                }
+                uint32_t need = __ballot_sync(FULL, retire);
+                any_retire |= need;
+                __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
+                // decode completions found in this row: retired by the whole warp, GPU by GPU
+                while (need) {
+                    const int l = __ffs((int)need) - 1;
+                    need &= need - 1;
+                    const uint32_t gg = (k << 5) + (uint32_t)l;
+                    const unsigned long long vv = __shfl_sync(FULL, v, l);
+                    const double te = __longlong_as_double((long long)vv);
+                    retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
+                    if (lane == l) start_at(gg, te);
+                }
             }
-            if (err) return true;
-            dispatch();
+            (void)any_retire;
+            // the non-local event, if it comes before anything a new iteration could bring
+            if (tint < wt && tint <= tend_bits) {
+                t = __longlong_as_double((long long)tint);
+                if (src >= SRC_SERVER) {
+                    on_server(src - SRC_SERVER);
+                } else {
+                    ++events;
+                    if (src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
+                    else if (src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
+                    else if (src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
+                    else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
+                    else { load_block(blk + 1); drain_dirty = true; gate_dirty = true; }
+                }
+                if (err) return true;
+                dispatch();
+            } else if (!__any_sync(FULL, progressed)) {
+                err = ERR_INTERNAL;     // a round that neither ended an iteration nor handled an event: never spin
+                return true;
+            }
         }
+    }
+
+    // Is the end of the running iteration of GPU g local?  Not when its prefill finishes, nor when a decode
+    // finishes while requests wait in a decode buffer or while the GPU (moved into the mixed group by a block
+    // switch) holds a full solo batch and could take a prefill afterwards.
+    __device__ __forceinline__ bool is_local(uint32_t g, bool buffered) const
+    {
+        const uint32_t na = nact[g];
+        if (na & 0x8000u) return false;
+        if ((na & 0x4000u) && (buffered || (g < M && ndec[g] > p.B - 1))) return false;
+        return true;
     }
 };
 
@@ -929,6 +1032,8 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         const unsigned long long H_total = h.H_total + (p.advance ? p.horizon_iters : 0ull);
         if (p.advance) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
         s.T_end = T_end;
+        s.T_reset = h.T_reset;
+        s.tau_min = fmin(p.coef[0], p.coef[3]);
         s.t = 0.0;
         s.load_block(h.blk);
         s.dq_head0 = h.dq_head0; s.dq_head1 = h.dq_head1; s.dq_n0 = h.dq_n0; s.dq_n1 = h.dq_n1;
@@ -973,8 +1078,9 @@ __global__ void qsim_reset_kernel(Params p)
     for (int l = 0; l < 32; ++l) { h.iters_mixed[l] = 0; h.iters_solo[l] = 0; h.busy_mixed[l] = 0.0; h.busy_solo[l] = 0.0; }
     for (uint32_t i = 0; i < MAXI; ++i) {
         ClassState &c = h.cs[i];
-        Area *as[5] = { &c.aQp, &c.aX, &c.aQd, &c.aYm, &c.aYs };
-        for (int k = 0; k < 5; ++k) { as[k]->area = 0.0; as[k]->t_last = T; }
+        Area *as[3] = { &c.aQp, &c.aX, &c.aQd };
+        for (int k = 0; k < 3; ++k) { as[k]->area = 0.0; as[k]->t_last = T; }
+        c.sYm_in = c.sYm_out = c.sYs_in = c.sYs_out = 0.0;
         c.arrivals = c.admitted = c.prefill_done = c.placed_mixed = c.placed_solo = c.done_mixed = c.done_solo = 0;
         c.abandoned_p = c.abandoned_d = c.overflow = c.overflow_d = c.tok_in_pf = c.tok_in_done = c.tok_out_done = 0;
         c.sum_ttft = 0.0; c.sum_tpot = 0.0;

@@ -163,7 +163,7 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
     p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = cfg->hist;
     p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
-    p.event_budget = 1ull << 40;
+    p.event_budget = 1ull << 28;
     for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
     for (uint32_t i = 0; i < cfg->I; ++i) {
         p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
@@ -312,13 +312,13 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
         std::memset(&st, 0, sizeof st);
         const double T = H.T_end;
         st.T_elapsed = T - H.T_reset;
-        st.events = H.events;
         for (int l = 0; l < 32; ++l) {
             st.iters_mixed += H.iters_mixed[l];
             st.iters_solo += H.iters_solo[l];
             st.busy_mixed = st.busy_mixed + H.busy_mixed[l];
             st.busy_solo = st.busy_solo + H.busy_solo[l];
         }
+        st.events = H.events + st.iters_mixed + st.iters_solo;   // H.events counts everything but iteration ends
         for (uint32_t i = 0; i < I; ++i) {
             const ClassState &c = H.cs[i];
             qsim_class_stats &o = st.cls[i];
@@ -333,8 +333,8 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
             o.area_Qp = c.aQp.area + (double)c.pq_n * (T - c.aQp.t_last);
             o.area_X = c.aX.area + (double)c.X * (T - c.aX.t_last);
             o.area_Qd = c.aQd.area + (double)Qd * (T - c.aQd.t_last);
-            o.area_Ym = c.aYm.area + (double)c.Ym * (T - c.aYm.t_last);
-            o.area_Ys = c.aYs.area + (double)c.Ys * (T - c.aYs.t_last);
+            o.area_Ym = (c.sYm_out - c.sYm_in) + (double)c.Ym * (T - H.T_reset);
+            o.area_Ys = (c.sYs_out - c.sYs_in) + (double)c.Ys * (T - H.T_reset);
             o.sum_ttft = c.sum_ttft; o.sum_tpot = c.sum_tpot;
         }
         if (per_rep) per_rep[r] = st;
@@ -495,7 +495,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
     p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = 0;
     p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
-    p.event_budget = 1ull << 40;
+    p.event_budget = 1ull << 28;
     for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
     for (uint32_t i = 0; i < cfg->I; ++i) {
         p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;

@@ -106,9 +106,15 @@ def test_resumable_and_event_budget_do_not_change_results():
     a, _ = gpu_run(inp, 3000)
     b, _ = gpu_run(inp, 3000, chunks=[700, 1300, 1000])
     c, _ = gpu_run(inp, 3000, budget=5000)
+    # integer statistics are identical; fp64 sums may be accumulated in another order when the look-ahead
+    # windows are cut at different places
     for k in a:
-        assert np.array_equal(a[k], b[k]), ("chunks", k)
-        assert np.array_equal(a[k], c[k]), ("budget", k)
+        if a[k].dtype.kind == "f":
+            assert np.allclose(a[k], b[k], rtol=1e-12, atol=0), ("chunks", k)
+            assert np.allclose(a[k], c[k], rtol=1e-12, atol=0), ("budget", k)
+        else:
+            assert np.array_equal(a[k], b[k]), ("chunks", k)
+            assert np.array_equal(a[k], c[k]), ("budget", k)
 
 
 def test_replication_offset_shards_compose():
