@@ -208,6 +208,10 @@ int qsim_simulate_static(const qsim_config *cfg, const qsim_class *classes, cons
                          const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
                          qsim_rep_stats *per_rep, void *cuda_stream);
 
+/* Diagnostic: look-ahead rounds executed since the last reset, summed over replications (a round handles at
+ * most one non-local event and every local iteration end before it).  Synchronises the stream. */
+int qsim_round_count(qsim_t *h, uint64_t *rounds);
+
 /* Kernel launches issued by this handle so far (for accounting in benchmarks). */
 int qsim_launch_count(const qsim_t *h, uint64_t *launches);
 

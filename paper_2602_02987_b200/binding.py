@@ -18,7 +18,7 @@ _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_
 
 EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
-           "qsim_simulate_static", "qsim_launch_count", "qsim_destroy", "qsim_last_error")
+           "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_destroy", "qsim_last_error")
 
 
 class QSimError(RuntimeError):
@@ -80,6 +80,7 @@ def load_library():
         L.qsim_simulate_static.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
                                            C.POINTER(qsim_targets), C.c_uint64, vp, vp, vp]
         L.qsim_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.qsim_round_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.qsim_destroy.argtypes = [vp]
         L.qsim_last_error.restype = C.c_char_p
         for n in EXPORTS:
@@ -180,6 +181,11 @@ class QSim:
     def launch_count(self) -> int:
         n = C.c_uint64()
         _check(self.L.qsim_launch_count(self.h, C.byref(n)))
+        return int(n.value)
+
+    def round_count(self) -> int:
+        n = C.c_uint64()
+        _check(self.L.qsim_round_count(self.h, C.byref(n)))
         return int(n.value)
 
     def stats(self, with_totals=False) -> dict:

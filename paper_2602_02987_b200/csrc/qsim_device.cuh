@@ -66,7 +66,7 @@ struct ClassState {
 
 struct RepHeader {
     double T_end, T_reset;
-    unsigned long long place_ord, events, H_total, pad64;
+    unsigned long long place_ord, events, H_total, rounds;
     uint32_t blk, done, err, pad;
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
     unsigned long long iters_mixed[32], iters_solo[32];
@@ -255,7 +255,7 @@ struct Sim {
     // replicated scalars
     double t, T_end, T_blk_next, T_reset, tau_min;
     uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
-    unsigned long long place_ord, events;
+    unsigned long long place_ord, events, rounds;
     bool drain_dirty, gate_dirty, touch_all;
     // per-lane partial sums
     unsigned long long it_mixed, it_solo;
@@ -835,6 +835,7 @@ struct Sim {
             if (tint > tend_bits && tmin_all > tend_bits) return true;     // nothing left up to T_end
             if (budget == 0) return false;
             --budget;
+            ++rounds;
             // no iteration that starts in this round can end before T_min + tau_min
             unsigned long long wt = INF;
             if (tmin_all < INF)
@@ -1037,7 +1038,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.t = 0.0;
         s.load_block(h.blk);
         s.dq_head0 = h.dq_head0; s.dq_head1 = h.dq_head1; s.dq_n0 = h.dq_n0; s.dq_n1 = h.dq_n1;
-        s.place_ord = h.place_ord; s.events = h.events;
+        s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
         s.n_touch = 0; s.touch_all = false; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
         s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
@@ -1058,7 +1059,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         if (lane == 0) {
             h.T_end = T_end; h.H_total = H_total; h.blk = s.blk;
             h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
-            h.place_ord = s.place_ord; h.events = s.events; h.err = s.err;
+            h.place_ord = s.place_ord; h.events = s.events; h.rounds = s.rounds; h.err = s.err;
             h.done = finished ? 1u : 0u;
             if (!finished) atomicAdd(p.not_done, 1u);
         }
@@ -1075,6 +1076,7 @@ __global__ void qsim_reset_kernel(Params p)
     const double T = h.T_end;
     h.T_reset = T;
     h.events = 0;
+    h.rounds = 0;
     for (int l = 0; l < 32; ++l) { h.iters_mixed[l] = 0; h.iters_solo[l] = 0; h.busy_mixed[l] = 0.0; h.busy_solo[l] = 0.0; }
     for (uint32_t i = 0; i < MAXI; ++i) {
         ClassState &c = h.cs[i];

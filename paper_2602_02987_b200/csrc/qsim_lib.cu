@@ -285,6 +285,19 @@ int qsim_launch_count(const qsim_t *h, uint64_t *launches)
     return QSIM_OK;
 }
 
+int qsim_round_count(qsim_t *h, uint64_t *rounds)
+{
+    if (!h || !rounds) return fail(QSIM_EINVAL, "null argument");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_round_count before qsim_bind");
+    std::vector<RepHeader> hdr(h->cfg.R);
+    CUDA_TRY(cudaMemcpyAsync(hdr.data(), h->par.hdr, hdr.size() * sizeof(RepHeader), cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    uint64_t n = 0;
+    for (const RepHeader &H : hdr) n += H.rounds;
+    *rounds = n;
+    return QSIM_OK;
+}
+
 int qsim_reset_stats(qsim_t *h)
 {
     if (!h) return fail(QSIM_EINVAL, "null handle");
