@@ -77,6 +77,7 @@ struct RepHeader {
 static_assert(sizeof(ClassState) % 8 == 0 && (sizeof(ClassState) * MAXI) % 16 == 0, "ClassState is copied in 16-byte words");
 static_assert(sizeof(RepHeader) % 16 == 0 && offsetof(RepHeader, cs) % 16 == 0, "RepHeader layout");
 
+struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential and packed lengths
 struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
 
 struct ClassPar { double theta; uint32_t P, D, prio, pad; };
@@ -183,20 +184,6 @@ __device__ __forceinline__ uint32_t hist_bin(double x)
     return (uint32_t)b;
 }
 
-// Cooperative table look-up: 1 + #{j < LMAX-1 : thr[j] <= w} in three 32-way probes (8192 = 32*32*8).
-__device__ __forceinline__ uint32_t table_length(const uint32_t *thr, uint32_t w, int lane)
-{
-    uint32_t idx = (uint32_t)lane * 256u + 255u;
-    bool ok = idx < LMAX - 1 && __ldg(thr + idx) <= w;
-    uint32_t base = (uint32_t)__popc(__ballot_sync(FULL, ok)) * 256u;
-    idx = base + (uint32_t)lane * 8u + 7u;
-    ok = idx < LMAX - 1 && __ldg(thr + idx) <= w;
-    base += (uint32_t)__popc(__ballot_sync(FULL, ok)) * 8u;
-    idx = base + (uint32_t)lane;
-    ok = lane < 8 && idx < LMAX - 1 && __ldg(thr + idx) <= w;
-    return 1u + base + (uint32_t)__popc(__ballot_sync(FULL, ok));
-}
-
 __device__ __forceinline__ uint32_t pack_job(uint32_t P, uint32_t D, uint32_t cls, uint32_t flag)
 {
     return (P - 1u) | ((D - 1u) << 13) | (cls << 26) | (flag << 31);
@@ -230,6 +217,36 @@ __device__ __forceinline__ void ab_change(AbClock &c, double theta, uint32_t Q_o
     }
 }
 
+// 1 + #{j < LMAX-1 : thr[j] <= w} by binary search
+__device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, uint32_t w)
+{
+    uint32_t lo = 0, hi = LMAX - 1;          // the count lies in [lo, hi]
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(thr + mid) <= w) lo = mid + 1; else hi = mid;
+    }
+    return 1u + lo;
+}
+
+// Arrival draw `index` of class i: one Philox block gives the unit exponential and both lengths.
+// (Arguments by value: a reference to the kernel parameters would force a local copy of them.)
+__device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long long global_rep, uint32_t i,
+                                        unsigned long long index, const uint32_t *tables, uint32_t P, uint32_t D)
+{
+    uint32_t w0, w1, w2, w3;
+    philox((uint32_t)index, (uint32_t)(index >> 32), (STREAM_ARRIVAL << 8) | i, (uint32_t)global_rep, (uint32_t)seed,
+           (uint32_t)(seed >> 32), w0, w1, w2, w3);
+    ADraw d;
+    d.E = -qlog(u53(w0, w1));
+    if (tables) {
+        P = table_lookup(tables + ((size_t)i * 2 + 0) * LMAX, w2);
+        D = table_lookup(tables + ((size_t)i * 2 + 1) * LMAX, w3);
+    }
+    d.pk = pack_job(P, D, i, 0);
+    d.pad = 0;
+    return d;
+}
+
 // ---------------------------------------------------------------------------------------------
 // the per-warp simulator
 // ---------------------------------------------------------------------------------------------
@@ -255,11 +272,17 @@ struct Sim {
     // replicated scalars
     double t, T_end, T_blk_next, T_reset, tau_min;
     uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
+    uint32_t n_idle_pf;          // mixed GPUs whose prefill slot is idle (and that may take a prefill)
     unsigned long long place_ord, events, rounds;
     bool drain_dirty, gate_dirty, touch_all;
     // per-lane partial sums
     unsigned long long it_mixed, it_solo;
     double busy_mixed, busy_solo;
+    // pre-generated arrival draws of this lane's class (ring in shared memory) and a pending scheduling request
+    ADraw *aring;
+    uint32_t ring_n, ring_pos;
+    bool sched_pending;
+    double t0_pending;
     // block parameters of the current block (lane i holds class i)
     double b_xstar, b_nx, b_nq, b_ps;
 
@@ -280,63 +303,90 @@ struct Sim {
     }
 
     // --- arrivals ------------------------------------------------------------------------------
-    // Next class-i arrival after t0 (all lanes compute the same draw; lane i stores the result).
-    // A candidate at or past the end of its block is discarded and drawn again from the boundary under
-    // the next block's rate (memorylessness of the Poisson process).
-    __device__ void schedule_arrival(uint32_t i, double t0)
+    // Arrival draws do not depend on the simulation: draw k of class i is one Philox block that gives a unit
+    // exponential E_k (words 0,1) and the two lengths (words 2,3).  The warp produces 32 consecutive draws
+    // of a class at a time, one per lane, into a ring in shared memory; the class lane consumes them in
+    // order.  Draws left in the ring at the end of a launch are given back (adraw is rewound).
+
+    __device__ __forceinline__ void refill(uint32_t i)
     {
-        unsigned long long k = __shfl_sync(FULL, cs[lane & 7].adraw, i);
-        uint32_t b = __shfl_sync(FULL, cs[lane & 7].ablk, i);
-        double ta = dinf();
-        uint32_t nP = p.cls[i].P, nD = p.cls[i].D;
+        const unsigned long long base = __shfl_sync(FULL, cs[lane & 7].adraw, i);
+        aring[i * 32 + lane] = make_draw(p.seed, p.rep_offset + rep, i, base + (unsigned long long)lane,
+                                         p.length_mode == 1 ? p.lengths : nullptr, p.cls[i].P, p.cls[i].D);
+        __syncwarp();
+        if (lane == (int)i) {
+            cs[i].adraw = base + 32ull;
+            ring_pos = 0;
+            ring_n = 32;
+            if (sched_pending) { sched_pending = false; schedule_from(t0_pending); }
+        }
+        __syncwarp();
+    }
+
+    // Class lane only: next arrival of this lane's class after t0.  A candidate at or past the end of its
+    // block is discarded and drawn again from the boundary under the next block's rate (memorylessness).
+    __device__ void schedule_from(double t0)
+    {
+        ClassState &c = cs[lane];
+        uint32_t b = c.ablk;
         for (;;) {
-            const double Lam = __dmul_rn((double)p.N, p.blocks[b].rate[i]);
+            const double Lam = __dmul_rn((double)p.N, p.blocks[b].rate[lane]);
             const bool has_next = b + 1 < p.nblk;
             if (!(Lam > 0.0)) {
-                if (!has_next) break;
+                if (!has_next) { c.ta = dinf(); c.ablk = b; return; }
                 ++b; t0 = block_start(b);
                 continue;
             }
-            uint32_t w0, w1, w2, w3;
-            draw(p, rep, (STREAM_ARRIVAL << 8) | i, k++, w0, w1, w2, w3);
-            const double E = -qlog(u53(w0, w1));
-            const double cand = __dadd_rn(t0, __ddiv_rn(E, Lam));
+            if (ring_n == 0) {          // out of draws: the warp refills at the top of the next round
+                sched_pending = true; t0_pending = t0; c.ablk = b; c.ta = dinf();
+                return;
+            }
+            const ADraw d = aring[lane * 32 + ring_pos];
+            ring_pos++; ring_n--;
+            const double cand = __dadd_rn(t0, __ddiv_rn(d.E, Lam));
             if (has_next && cand >= block_start(b + 1)) {
                 ++b; t0 = block_start(b);
                 continue;
             }
-            ta = cand;
-            if (p.length_mode == 1) {
-                nP = table_length(p.lengths + ((size_t)i * 2 + 0) * LMAX, w2, lane);
-                nD = table_length(p.lengths + ((size_t)i * 2 + 1) * LMAX, w3, lane);
-            }
-            break;
-        }
-        if (lane == (int)i) {
-            ClassState &c = cs[i];
-            c.ta = ta; c.adraw = k; c.ablk = b; c.nextP = nP; c.nextD = nD;
+            c.ta = cand; c.ablk = b; c.nextP = job_P(d.pk); c.nextD = job_D(d.pk);
+            return;
         }
     }
 
+    // Class lane only: the arrival scheduled at c.ta happens; nothing outside the class is touched.
+    __device__ void arrival_local()
+    {
+        const uint32_t i = (uint32_t)lane;
+        ClassState &c = cs[i];
+        const double ta = c.ta;
+        c.arrivals++;
+        if (c.pq_n >= p.qcap) {
+            c.overflow++;
+        } else {
+            ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n + 1, ta);
+            area_touch(c.aQp, c.pq_n, ta);
+            uint32_t pos = c.pq_head + c.pq_n;
+            if (pos >= p.qcap) pos -= p.qcap;
+            QEntry e; e.t = ta; e.pk = pack_job(c.nextP, c.nextD, i, 0); e.cls = i;
+            pq[(size_t)i * p.qcap + pos] = e;
+            c.pq_n++;
+        }
+        schedule_from(ta);
+    }
+
+    // warp-wide path: an arrival while some prefill slot is idle (the gate may admit it at once)
     __device__ void on_arrival(uint32_t i)
     {
-        if (lane == (int)i) {
-            ClassState &c = cs[i];
-            c.arrivals++;
-            if (c.pq_n >= p.qcap) {
-                c.overflow++;
-            } else {
-                ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n + 1, t);
-                area_touch(c.aQp, c.pq_n, t);
-                uint32_t pos = c.pq_head + c.pq_n;
-                if (pos >= p.qcap) pos -= p.qcap;
-                QEntry e; e.t = t; e.pk = pack_job(c.nextP, c.nextD, i, 0); e.cls = i;
-                pq[(size_t)i * p.qcap + pos] = e;
-                c.pq_n++;
-            }
-        }
-        schedule_arrival(i, t);
+        if (lane == (int)i) arrival_local();
         gate_dirty = true;
+    }
+
+    __device__ uint32_t count_idle_pf()
+    {
+        uint32_t cnt = 0;
+        for (uint32_t k = 0; k < (p.Npad >> 5); ++k)
+            cnt += (uint32_t)__popc(__ballot_sync(FULL, eligible((k << 5) + (uint32_t)lane, WANT_PREFILL)));
+        return cnt;
     }
 
     // --- abandonment ---------------------------------------------------------------------------
@@ -546,6 +596,7 @@ struct Sim {
             c.X++;
             c.admitted++;
         }
+        n_idle_pf--;
         if (lane == (int)(g & 31u)) {
             pfjob[g] = e.pk | 0x80000000u;
             pfrem[g] = job_P(e.pk);
@@ -691,6 +742,7 @@ struct Sim {
     {
         const int owner = (int)(g & 31u);
         uint32_t flags = 0, itg = 0, nd = 0;
+        bool recount_idle = false;
         if (lane == owner) {
             itg = it[g] + 1;
             it[g] = itg;
@@ -716,6 +768,7 @@ struct Sim {
             retire_decodes(g, itg, nd, t);
             drain_dirty = true;
             gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
+            recount_idle = true;
         }
         if (flags & 2u) {
             // prefill finished: account, then hand the request to the decode stage
@@ -765,7 +818,9 @@ struct Sim {
             if (lane == owner) pfjob[g] = 0;
             drain_dirty = true;
             gate_dirty = true;
+            recount_idle = true;
         }
+        if (recount_idle) { __syncwarp(); n_idle_pf = count_idle_pf(); }
         touch_server(g);
     }
 
@@ -798,14 +853,19 @@ struct Sim {
         unsigned long long budget = p.event_budget;
         for (;;) {
             __syncwarp();
-            // next non-local event of this lane (sources scanned in id order with '<' keep the tie order)
+            // classes that ran out of arrival draws get 32 new ones
+            for (uint32_t need = __ballot_sync(FULL, sched_pending); need; need &= need - 1)
+                refill((uint32_t)__ffs((int)need) - 1u);
+            // next non-local event of this lane (sources scanned in id order with '<' keep the tie order);
+            // an arrival is local while no prefill slot is idle: it only joins its class queue
             unsigned long long bt = INF, tmin = INF;
             uint32_t bs = NONE32;
             if (lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
             if (lane < (int)p.I) {
                 const ClassState &c = cs[lane];
                 unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
-                if (v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
+                tmin = v;
+                if (n_idle_pf > 0 && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
                 v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
                 if (v < bt) { bt = v; bs = SRC_ABP + lane; }
                 v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
@@ -847,6 +907,18 @@ struct Sim {
             if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
             uint32_t any_retire = 0;
             bool progressed = false;
+            if (lane < (int)p.I && n_idle_pf == 0) {
+                // local arrivals of this lane's class, in time order, up to the limit and up to the class's own
+                // next abandonment (which each arrival moves)
+                ClassState &c = cs[lane];
+                for (int guard = 0; guard < 64; ++guard) {
+                    const unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
+                    if (!(v < lim_t || (v == lim_t && SRC_ARRIVAL + (uint32_t)lane < lim_s))) break;
+                    if (v > (unsigned long long)__double_as_longlong(c.abp.t_ab)) break;
+                    arrival_local();
+                    progressed = true;
+                }
+            }
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
@@ -876,12 +948,11 @@ struct Sim {
                 if (src >= SRC_SERVER) {
                     on_server(src - SRC_SERVER);
                 } else {
-                    ++events;
                     if (src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
                     else if (src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
                     else if (src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
                     else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
-                    else { load_block(blk + 1); drain_dirty = true; gate_dirty = true; }
+                    else { ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true; n_idle_pf = count_idle_pf(); }
                 }
                 if (err) return true;
                 dispatch();
@@ -907,7 +978,7 @@ struct Sim {
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
     uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
-        off_pfcur, srv_bytes, off_touch, off_gate, off_cs, total;
+        off_pfcur, srv_bytes, off_touch, off_gate, off_cs, off_ring, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
@@ -932,6 +1003,8 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
     L.off_gate = o; o += (8 + 8 + 4) * MAXI;
     o = (o + 15u) & ~15u;
     L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
+    o = (o + 15u) & ~15u;
+    L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * MAXI;
     L.total = (o + 15u) & ~15u;
     return L;
 }
@@ -954,6 +1027,8 @@ __device__ __forceinline__ void bind_pointers(Sim &s, char *sm, const SmemLayout
     s.gate_dq = s.gate_xi + MAXI;
     s.gate_ok = reinterpret_cast<uint32_t *>(s.gate_dq + MAXI);
     s.cs = reinterpret_cast<ClassState *>(sm + L.off_cs);
+    s.aring = reinterpret_cast<ADraw *>(sm + L.off_ring);
+    s.ring_n = 0; s.ring_pos = 0; s.sched_pending = false; s.t0_pending = 0.0;
     const Params &p = s.p;
     const size_t r = s.rep;
     s.s_fin = p.slot_fin + r * (size_t)p.N * p.B;
@@ -990,7 +1065,16 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
             }
         }
         __syncwarp();
-        for (uint32_t i = 0; i < p.I; ++i) { s.schedule_arrival(i, 0.0); __syncwarp(); }
+        // first arrival of every class: ask for draws, let the warp fill the rings, give the unused draws back
+        s.sched_pending = lane < (int)p.I;
+        s.t0_pending = 0.0;
+        for (int guard = 0; guard < 64; ++guard) {
+            uint32_t need = __ballot_sync(FULL, s.sched_pending);
+            if (!need) break;
+            for (; need; need &= need - 1) s.refill((uint32_t)__ffs((int)need) - 1u);
+        }
+        if (lane < (int)p.I) s.cs[lane].adraw -= s.ring_n;
+        __syncwarp();
         // write everything out
         RepHeader &h = p.hdr[rep];
         for (uint32_t o = lane * 4; o < sizeof(RepHeader); o += 128)
@@ -1041,9 +1125,11 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
         s.n_touch = 0; s.touch_all = false; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
+        s.n_idle_pf = s.count_idle_pf();
         s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
         s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
         const bool finished = s.err ? true : s.run();
+        if (lane < (int)p.I) s.cs[lane].adraw -= s.ring_n;     // unused arrival draws are produced again next time
         __syncwarp();
         // stage back
         char *out = p.srv + (size_t)rep * p.srv_bytes;

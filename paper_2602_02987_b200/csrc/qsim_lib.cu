@@ -331,7 +331,7 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
             st.busy_mixed = st.busy_mixed + H.busy_mixed[l];
             st.busy_solo = st.busy_solo + H.busy_solo[l];
         }
-        st.events = H.events + st.iters_mixed + st.iters_solo;   // H.events counts everything but iteration ends
+        st.events = H.events + st.iters_mixed + st.iters_solo;   // H.events counts block switches; class events are added below
         for (uint32_t i = 0; i < I; ++i) {
             const ClassState &c = H.cs[i];
             qsim_class_stats &o = st.cls[i];
@@ -349,6 +349,7 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
             o.area_Ym = (c.sYm_out - c.sYm_in) + (double)c.Ym * (T - H.T_reset);
             o.area_Ys = (c.sYs_out - c.sYs_in) + (double)c.Ys * (T - H.T_reset);
             o.sum_ttft = c.sum_ttft; o.sum_tpot = c.sum_tpot;
+            st.events += c.arrivals + c.abandoned_p + c.abandoned_d;
         }
         if (per_rep) per_rep[r] = st;
         tot.iters_mixed += st.iters_mixed; tot.iters_solo += st.iters_solo; tot.events += st.events;
