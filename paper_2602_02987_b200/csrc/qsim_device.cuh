@@ -942,6 +942,14 @@ struct Sim {
                 }
             }
             (void)any_retire;
+            // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
+            // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
+            bool redo = sched_pending;
+            if (lane < (int)p.I) {
+                const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
+                redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
+            }
+            if (__any_sync(FULL, redo)) continue;
             // the non-local event, if it comes before anything a new iteration could bring
             if (tint < wt && tint <= tend_bits) {
                 t = __longlong_as_double((long long)tint);
