@@ -41,6 +41,12 @@ constexpr unsigned FULL = 0xffffffffu;
 constexpr uint32_t NONE32 = 0xffffffffu;
 constexpr int TOUCH_CAP = 48;
 
+// Compile-time specialisation of the run kernel.  With F_GENERIC every mode is read from the parameters at
+// run time; otherwise the set bits say which features the instance contains and everything else is
+// compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
+constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
+                   F_OCC = 128;
+
 // source ids: smaller id wins an exact tie in time
 constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
 
@@ -84,7 +90,7 @@ struct ClassPar { double theta; uint32_t P, D, prio, pad; };
 struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI]; };
 
 struct Params {
-    uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance;
+    uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance, any_theta;
     unsigned long long seed, rep_offset, horizon_iters, event_budget;
     double block_len;
     double coef[6];
@@ -163,7 +169,7 @@ __device__ __forceinline__ double qlog(double x)
 }
 
 // iteration time of a batch with pf prefill tokens, d decodes, K resident KV tokens (Eq. (1)-(3))
-__device__ __forceinline__ double iter_time(const Params &p, uint32_t pf, uint32_t d, uint32_t K)
+__device__ __forceinline__ double iter_time(const Params &p, uint32_t pf, uint32_t d, uint32_t K, bool kappa = true)
 {
     double t;
     if (pf > 0) {
@@ -172,7 +178,7 @@ __device__ __forceinline__ double iter_time(const Params &p, uint32_t pf, uint32
     } else {
         t = __dadd_rn(p.coef[3], __dmul_rn(p.coef[4], (double)d));
     }
-    if (p.coef[5] != 0.0)
+    if (kappa && p.coef[5] != 0.0)
         t = __dadd_rn(t, __dmul_rn(p.coef[5], (double)K));
     return t;
 }
@@ -251,7 +257,17 @@ __device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long l
 // the per-warp simulator
 // ---------------------------------------------------------------------------------------------
 
+template <int SPL, uint32_t F>
 struct Sim {
+    __device__ __forceinline__ bool f_abandon() const { return (F & F_GENERIC) ? p.any_theta != 0 : (F & F_ABANDON) != 0; }
+    __device__ __forceinline__ bool f_sli() const { return (F & F_GENERIC) ? p.router == 1 : (F & F_SLI) != 0; }
+    __device__ __forceinline__ bool f_kappa() const { return (F & F_GENERIC) ? p.coef[5] != 0.0 : (F & F_KAPPA) != 0; }
+    __device__ __forceinline__ bool f_hist() const { return (F & F_GENERIC) ? hist != nullptr : (F & F_HIST) != 0; }
+    __device__ __forceinline__ bool f_blocks() const { return (F & F_GENERIC) ? p.nblk > 1 : (F & F_BLOCKS) != 0; }
+    __device__ __forceinline__ bool f_random() const { return (F & F_GENERIC) ? p.placement == 0 : (F & F_RANDOM) != 0; }
+    __device__ __forceinline__ bool f_occ() const { return (F & F_GENERIC) ? p.gate == 0 : (F & F_OCC) != 0; }
+    __device__ __forceinline__ uint32_t n_rows() const { return SPL > 0 ? (uint32_t)SPL : (p.Npad >> 5); }
+
     const Params &p;
     const int lane;
     const uint32_t rep;
@@ -299,7 +315,7 @@ struct Sim {
         if (lane < (int)p.I) {
             b_xstar = bp.xstar[lane]; b_nx = bp.nx[lane]; b_nq = bp.nq[lane]; b_ps = bp.ps[lane];
         }
-        T_blk_next = (b + 1 < p.nblk) ? block_start(b + 1) : dinf();
+        T_blk_next = (f_blocks() && b + 1 < p.nblk) ? block_start(b + 1) : dinf();
     }
 
     // --- arrivals ------------------------------------------------------------------------------
@@ -331,7 +347,7 @@ struct Sim {
         uint32_t b = c.ablk;
         for (;;) {
             const double Lam = __dmul_rn((double)p.N, p.blocks[b].rate[lane]);
-            const bool has_next = b + 1 < p.nblk;
+            const bool has_next = f_blocks() && b + 1 < p.nblk;
             if (!(Lam > 0.0)) {
                 if (!has_next) { c.ta = dinf(); c.ablk = b; return; }
                 ++b; t0 = block_start(b);
@@ -363,7 +379,7 @@ struct Sim {
         if (c.pq_n >= p.qcap) {
             c.overflow++;
         } else {
-            ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n + 1, ta);
+            if (f_abandon()) ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n + 1, ta);
             area_touch(c.aQp, c.pq_n, ta);
             uint32_t pos = c.pq_head + c.pq_n;
             if (pos >= p.qcap) pos -= p.qcap;
@@ -384,7 +400,8 @@ struct Sim {
     __device__ uint32_t count_idle_pf()
     {
         uint32_t cnt = 0;
-        for (uint32_t k = 0; k < (p.Npad >> 5); ++k)
+#pragma unroll
+        for (uint32_t k = 0; k < n_rows(); ++k)
             cnt += (uint32_t)__popc(__ballot_sync(FULL, eligible((k << 5) + (uint32_t)lane, WANT_PREFILL)));
         return cnt;
     }
@@ -483,9 +500,10 @@ struct Sim {
     // uniformly at random among the eligible GPUs (k-th in index order) or least loaded, lowest index
     __device__ uint32_t choose_server(int want)
     {
-        const uint32_t rows = p.Npad >> 5;
-        if (p.placement == 1) {
+        const uint32_t rows = n_rows();
+        if (!f_random()) {
             uint32_t best = NONE32;
+#pragma unroll
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 if (eligible(g, want)) best = min(best, ((uint32_t)ndec[g] << 16) | g);
@@ -531,7 +549,7 @@ struct Sim {
         if (lane == (int)i) {
             ClassState &c = cs[i];
             const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
-            ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd - 1, t);
+            if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd - 1, t);
             area_touch(c.aQd, c.Qd0 + c.Qd1, t);
             if (pool) c.Qd1--; else c.Qd0--;
             const double rel = __dsub_rn(t, T_reset);
@@ -549,7 +567,7 @@ struct Sim {
             s_pk[o] = pack_job(P, D, i, mixed ? 1u : 0u);
             ndec[g] = (uint16_t)(sl + 1);
             nfin[g] = min(nfin[g], fin);
-            Kpend[g] += P;
+            if (f_kappa()) Kpend[g] += P;
         }
         touch_server(g);
     }
@@ -557,7 +575,7 @@ struct Sim {
     // --- prefill gate ------------------------------------------------------------------------------
     __device__ uint32_t gate_class()
     {
-        if (p.gate == 1) {
+        if (!f_occ()) {
             // Prioritize-and-Route: largest D_i/P_i among waiting classes = smallest static rank
             uint32_t key = NONE32;
             if (lane < (int)p.I && cs[lane].pq_n > 0) key = (p.cls[lane].prio << 8) | (uint32_t)lane;
@@ -588,7 +606,7 @@ struct Sim {
         const QEntry e = pq[(size_t)i * p.qcap + head];
         if (lane == (int)i) {
             ClassState &c = cs[i];
-            ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n - 1, t);
+            if (f_abandon()) ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n - 1, t);
             area_touch(c.aQp, c.pq_n, t);
             c.pq_n--;
             c.pq_head = (head + 1 == p.qcap) ? 0 : head + 1;
@@ -615,14 +633,14 @@ struct Sim {
             const uint32_t pj = pfjob[g];
             if (nd > 0 || (pj >> 31)) {
                 uint32_t Kg = 0;
-                if (p.coef[5] != 0.0) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
+                if (f_kappa()) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
                 const uint32_t rem = pfrem[g];
                 const uint32_t pc = (pj >> 31) ? min(p.C, rem) : 0u;
                 pfcur[g] = (uint16_t)pc;
                 uint32_t fl = (nfin[g] == it[g] + 1u) ? 0x4000u : 0u;
                 if (pc > 0 && pc == rem) fl |= 0x8000u;
                 nact[g] = (uint16_t)(nd | fl);
-                tnext[g] = __dadd_rn(ts, iter_time(p, pc, nd, Kg));
+                tnext[g] = __dadd_rn(ts, iter_time(p, pc, nd, Kg, f_kappa()));
             }
         }
     }
@@ -633,7 +651,7 @@ struct Sim {
         __syncwarp();   // queue entries and GPU state written by the event handler are visible to every lane
         // decode routing: buffered jobs first (FCFS), solo GPUs before mixed ones
         if (drain_dirty && (dq_n0 | dq_n1)) {
-            if (p.router == 0) {
+            if (!f_sli()) {
                 while (dq_n0 > 0) {
                     uint32_t g = choose_server(WANT_SOLO);
                     if (g == NONE32) g = choose_server(WANT_MIX);
@@ -672,7 +690,7 @@ struct Sim {
         // start the next iteration on every GPU that was touched and is between iterations
         __syncwarp();
         if (touch_all) {
-            for (uint32_t k = 0; k < (p.Npad >> 5); ++k) {
+            for (uint32_t k = 0; k < n_rows(); ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 if (g < p.N) start_if_needed(g);
             }
@@ -715,7 +733,7 @@ struct Sim {
                     c.tok_out_done += D;
                     const double tpot = __ddiv_rn(__dsub_rn(te, tpf), (double)D);
                     c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
-                    if (hist) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
+                    if (f_hist()) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
                 }
                 Kdrop += P + D;
                 const uint32_t last = n - 1;
@@ -732,7 +750,7 @@ struct Sim {
         if (lane == owner) {
             ndec[g] = (uint16_t)n;
             nfin[g] = newmin;
-            K[g] -= Kdrop;
+            if (f_kappa()) K[g] -= Kdrop;
         }
         __syncwarp();
     }
@@ -746,11 +764,11 @@ struct Sim {
         if (lane == owner) {
             itg = it[g] + 1;
             it[g] = itg;
-            const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = K[g];
-            const double tau = iter_time(p, pc, na, Kg);
+            const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
+            const double tau = iter_time(p, pc, na, Kg, f_kappa());
             if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
-            K[g] = Kg + na;
+            if (f_kappa()) K[g] = Kg + na;
             tnext[g] = dinf();
             nd = ndec[g];
             if (nfin[g] == itg) flags |= 1u;
@@ -776,7 +794,7 @@ struct Sim {
             const double tarr = pf_tarr[g];
             const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
             uint32_t pool = 0;
-            if (p.router == 1) {
+            if (f_sli()) {
                 // SLI-aware router: one uniform per finished prefill decides the pool
                 const unsigned long long ord = __shfl_sync(FULL, cs[lane & 7].sli_ord, i);
                 const double ps = __shfl_sync(FULL, b_ps, i);
@@ -794,13 +812,13 @@ struct Sim {
                 c.tok_in_pf += P;                  // separate charging credits the prompt here, Eq. (23)
                 const double ttft = __dsub_rn(t, tarr);
                 c.sum_ttft = __dadd_rn(c.sum_ttft, ttft);
-                if (hist) hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)]++;
-                if (p.router == 1) c.sli_ord++;
+                if (f_hist()) hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)]++;
+                if (f_sli()) c.sli_ord++;
                 if (full) {
                     c.overflow_d++;
                 } else {
                     const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
-                    ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd + 1, t);
+                    if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd + 1, t);
                     area_touch(c.aQd, c.Qd0 + c.Qd1, t);
                     if (pool) c.Qd1++; else c.Qd0++;
                 }
@@ -833,8 +851,8 @@ struct Sim {
         it[g] = itg;
         const uint32_t na_raw = nact[g], na = na_raw & 0x3fffu, pc = pfcur[g];
         uint32_t Kg = 0;
-        if (p.coef[5] != 0.0) { Kg = K[g]; K[g] = Kg + na; }
-        const double tau = iter_time(p, pc, na, Kg);
+        if (f_kappa()) { Kg = K[g]; K[g] = Kg + na; }
+        const double tau = iter_time(p, pc, na, Kg, f_kappa());
         if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] -= pc; }
         else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
         pfcur[g] = 0;
@@ -847,7 +865,7 @@ struct Sim {
     // --- round loop ----------------------------------------------------------------------------------
     __device__ bool run()
     {
-        const uint32_t rows = p.Npad >> 5;
+        const uint32_t rows = n_rows();
         const unsigned long long INF = 0x7ff0000000000000ull;
         const unsigned long long tend_bits = (unsigned long long)__double_as_longlong(T_end);
         unsigned long long budget = p.event_budget;
@@ -860,20 +878,23 @@ struct Sim {
             // an arrival is local while no prefill slot is idle: it only joins its class queue
             unsigned long long bt = INF, tmin = INF;
             uint32_t bs = NONE32;
-            if (lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
+            if (f_blocks() && lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
             if (lane < (int)p.I) {
                 const ClassState &c = cs[lane];
                 unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
                 tmin = v;
                 if (n_idle_pf > 0 && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
-                v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABP + lane; }
-                v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABD0 + lane; }
-                v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
+                if (f_abandon()) {
+                    v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABP + lane; }
+                    v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABD0 + lane; }
+                    v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
+                }
             }
             const bool buffered = (dq_n0 | dq_n1) != 0;
+#pragma unroll
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
@@ -914,11 +935,12 @@ struct Sim {
                 for (int guard = 0; guard < 64; ++guard) {
                     const unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
                     if (!(v < lim_t || (v == lim_t && SRC_ARRIVAL + (uint32_t)lane < lim_s))) break;
-                    if (v > (unsigned long long)__double_as_longlong(c.abp.t_ab)) break;
+                    if (f_abandon() && v > (unsigned long long)__double_as_longlong(c.abp.t_ab)) break;
                     arrival_local();
                     progressed = true;
                 }
             }
+#pragma unroll
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
@@ -945,7 +967,7 @@ struct Sim {
             // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
             // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
             bool redo = sched_pending;
-            if (lane < (int)p.I) {
+            if (f_abandon() && lane < (int)p.I) {
                 const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
                 redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
             }
@@ -956,9 +978,9 @@ struct Sim {
                 if (src >= SRC_SERVER) {
                     on_server(src - SRC_SERVER);
                 } else {
-                    if (src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
-                    else if (src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
-                    else if (src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
+                    if (f_abandon() && src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
+                    else if (f_abandon() && src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
+                    else if (f_abandon() && src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
                     else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
                     else { ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true; n_idle_pf = count_idle_pf(); }
                 }
@@ -1017,7 +1039,8 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
     return L;
 }
 
-__device__ __forceinline__ void bind_pointers(Sim &s, char *sm, const SmemLayout &L)
+template <int SPL, uint32_t F>
+__device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const SmemLayout &L)
 {
     s.tnext = reinterpret_cast<double *>(sm + L.off_tnext);
     s.pf_tarr = reinterpret_cast<double *>(sm + L.off_tarr);
@@ -1050,11 +1073,13 @@ __device__ __forceinline__ void bind_pointers(Sim &s, char *sm, const SmemLayout
 // Empty system at t = 0: idle GPUs, first arrival of every class scheduled, abandonment levels drawn.
 __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
 {
+    constexpr int SPLT = 0;
+    constexpr uint32_t FT = F_GENERIC;
     extern __shared__ __align__(16) char sm[];
     const int lane = threadIdx.x;
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         const SmemLayout L = smem_layout(p.Npad);
-        Sim s(p, lane, rep);
+        Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();
         for (uint32_t o = lane * 4; o < L.total; o += 128) *reinterpret_cast<uint32_t *>(sm + o) = 0;
@@ -1099,6 +1124,7 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
 }
 
 // Advance replications to their new end time (or until the per-launch event budget runs out).
+template <int SPLT, uint32_t FT>
 __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
 {
     extern __shared__ __align__(16) char sm[];
@@ -1107,7 +1133,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
         const SmemLayout L = smem_layout(p.Npad);
-        Sim s(p, lane, rep);
+        Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();
         // stage state: server arrays (coalesced 16-byte copies) and the class records

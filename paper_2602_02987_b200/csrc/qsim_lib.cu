@@ -55,6 +55,7 @@ struct qsim {
     bool bound = false;
     uint64_t launches = 0;
     int device = 0;
+    void (*run_fn)(qsimdev::Params) = nullptr;
 };
 
 namespace {
@@ -122,13 +123,83 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
     return QSIM_OK;
 }
 
+// Instances of the run kernel: (GPUs per lane, feature set).  A problem runs on the smallest instance that
+// contains its features; the fully generic instance takes everything else.
+using RunKernel = void (*)(Params);
+struct RunVariant { int spl; uint32_t feat; RunKernel fn; };
+
+template <int SPL>
+void add_variants(std::vector<RunVariant> &v)
+{
+    v.push_back({SPL, 0u, qsim_run_kernel<SPL, 0u>});
+    v.push_back({SPL, F_OCC, qsim_run_kernel<SPL, F_OCC>});
+    v.push_back({SPL, F_OCC | F_ABANDON, qsim_run_kernel<SPL, F_OCC | F_ABANDON>});
+    v.push_back({SPL, F_OCC | F_ABANDON | F_RANDOM, qsim_run_kernel<SPL, F_OCC | F_ABANDON | F_RANDOM>});
+    v.push_back({SPL, F_GENERIC, qsim_run_kernel<SPL, F_GENERIC>});
+}
+
+const std::vector<RunVariant> &run_variants()
+{
+    static const std::vector<RunVariant> table = [] {
+        std::vector<RunVariant> v;
+        add_variants<1>(v);
+        add_variants<2>(v);
+        add_variants<4>(v);
+        v.push_back({0, F_GENERIC, qsim_run_kernel<0, F_GENERIC>});
+        return v;
+    }();
+    return table;
+}
+
+qsim_config nohist_features(qsim_config c) { c.hist = 0; return c; }
+
+uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *coef)
+{
+    uint32_t f = 0;
+    for (uint32_t i = 0; i < c.I; ++i)
+        if (cls[i].theta > 0.0) f |= F_ABANDON;
+    if (c.router == QSIM_ROUTER_SLI) f |= F_SLI;
+    if (coef[5] != 0.0) f |= F_KAPPA;
+    if (c.hist) f |= F_HIST;
+    if (c.nblk > 1) f |= F_BLOCKS;
+    if (c.placement == QSIM_PLACE_RANDOM) f |= F_RANDOM;
+    if (c.gate == QSIM_GATE_OCCUPANCY) f |= F_OCC;
+    return f;
+}
+
+RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
+{
+    const int rows = (int)((N + 31u) / 32u);
+    const RunVariant *generic = nullptr, *best = nullptr;
+    // QSIM_KERNEL=generic forces the run-time-configured instance (for cross-checking the specialised ones)
+    const char *force = std::getenv("QSIM_KERNEL");
+    if (force && std::strcmp(force, "generic") == 0) feat = ~0u;
+    int best_bits = 99;
+    for (const RunVariant &v : run_variants()) {
+        if (v.spl != 0 && v.spl < rows) continue;          // too few GPUs per lane
+        if (v.spl == 0 && !generic) generic = &v;
+        if (v.spl == 0) continue;
+        // smallest row count that fits; among those the feature set with the fewest extras
+        int spl_fit = rows <= 1 ? 1 : (rows <= 2 ? 2 : 4);
+        if (v.spl != spl_fit) continue;
+        if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
+        // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits
+        // (abandonment, KV slope, blocks) may be present without being used
+        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_HIST;
+        if (feat == ~0u || (feat & MODES) != (v.feat & MODES) || (feat & ~v.feat) != 0) continue;
+        const int extra = __builtin_popcount(v.feat & ~feat);
+        if (extra < best_bits) { best = &v; best_bits = extra; }
+    }
+    return best ? *best : *generic;
+}
+
 int launch_run(qsim *h, bool advance, uint64_t horizon)
 {
     Params p = h->par;
     p.advance = advance ? 1u : 0u;
     p.horizon_iters = horizon;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    qsim_run_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
+    h->run_fn<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
@@ -169,6 +240,14 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
         p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
         p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
     }
+    p.any_theta = 0;
+    for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
+    {
+        // the per-GPU arrays are padded to the unrolled row count of the chosen instance
+        const RunVariant v = pick_run_kernel(cfg->N, features_of(*cfg, classes, coef));
+        h->run_fn = v.fn;
+        if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
+    }
     h->lay = smem_layout(p.Npad);
     p.srv_bytes = h->lay.srv_bytes;
     if (h->lay.total > 227u * 1024u) {
@@ -195,7 +274,7 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     }
     if (e == cudaSuccess) e = cudaMallocHost(&h->h_flag, 256);
     if (e == cudaSuccess && h->lay.total > 48u * 1024u) {
-        e = cudaFuncSetAttribute(qsim_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total);
+        e = cudaFuncSetAttribute(reinterpret_cast<const void *>(h->run_fn), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(qsim_init_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total);
     }
@@ -515,6 +594,13 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
         p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
         p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
     }
+    p.any_theta = 0;
+    for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
+    {
+        const RunVariant v = pick_run_kernel(cfg->N, features_of(nohist_features(*cfg), classes, coef));
+        h.run_fn = v.fn;
+        if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
+    }
     h.lay = smem_layout(p.Npad);
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
@@ -555,7 +641,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.hist_mem = nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h.sec.flag);
     if (h.lay.total > 48u * 1024u) {
-        CUDA_TRY(cudaFuncSetAttribute(qsim_run_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.lay.total));
+        CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void *>(h.run_fn), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.lay.total));
         CUDA_TRY(cudaFuncSetAttribute(qsim_init_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.lay.total));
     }
     // the array keeps the previous call's contents: the init kernel rewrites every header and GPU image;
@@ -568,7 +654,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
         q.advance = advance ? 1u : 0u;
         q.horizon_iters = advance ? horizon_iters : 0;
         CUDA_TRY(cudaMemsetAsync(q.not_done, 0, 4, stream));
-        qsim_run_kernel<<<cfg->R, 32, h.lay.total, stream>>>(q);
+        h.run_fn<<<cfg->R, 32, h.lay.total, stream>>>(q);
         CUDA_TRY(cudaGetLastError());
         uint32_t left = 0;
         CUDA_TRY(cudaMemcpyAsync(&left, q.not_done, 4, cudaMemcpyDeviceToHost, stream));
