@@ -289,6 +289,7 @@ struct Sim {
     double t, T_end, T_blk_next, T_reset, tau_min;
     uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
     uint32_t n_idle_pf;          // mixed GPUs whose prefill slot is idle (and that may take a prefill)
+    uint32_t idle_hint;          // when n_idle_pf == 1: that GPU if known, else NONE32
     unsigned long long place_ord, events, rounds;
     bool drain_dirty, gate_dirty, touch_all;
     // per-lane partial sums
@@ -498,6 +499,24 @@ struct Sim {
     }
 
     // uniformly at random among the eligible GPUs (k-th in index order) or least loaded, lowest index
+    // Solo-first target of a decode under least-loaded placement in one reduction: key = tier, load, index.
+    __device__ __forceinline__ uint32_t choose_solo_first()
+    {
+        uint32_t best = NONE32;
+#pragma unroll
+        for (uint32_t k = 0; k < n_rows(); ++k) {
+            const uint32_t g = (k << 5) + (uint32_t)lane;
+            if (g < p.N) {
+                const uint32_t nd = ndec[g];
+                const bool mix = g < M;
+                const uint32_t cap = (mix || (pfjob[g] >> 31)) ? p.B - 1 : p.B;
+                if (nd < cap) best = min(best, (mix ? 0x40000000u : 0u) | (nd << 16) | g);
+            }
+        }
+        best = __reduce_min_sync(FULL, best);
+        return best == NONE32 ? NONE32 : (best & 0xffffu);
+    }
+
     __device__ uint32_t choose_server(int want)
     {
         const uint32_t rows = n_rows();
@@ -538,20 +557,28 @@ struct Sim {
     }
 
     // --- decode placement ------------------------------------------------------------------------
+    // head of the pool's buffer goes to GPU g
     __device__ void place_decode(uint32_t pool, uint32_t g)
     {
         const uint32_t head = pool ? dq_head1 : dq_head0;
         const QEntry e = dq[(size_t)pool * p.qcap + head];
-        const uint32_t i = e.cls, P = job_P(e.pk), D = job_D(e.pk);
         if (pool) { dq_head1 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n1--; }
         else      { dq_head0 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n0--; }
+        place_job(pool, g, e.cls, job_P(e.pk), job_D(e.pk), e.t, true);
+    }
+
+    // A request of class i whose prefill ended at tpf starts decoding on GPU g.  from_buffer: it waited in
+    // the pool's buffer; otherwise it passes through the (empty) buffer at this very instant, which
+    // leaves the buffer's count, integral and abandonment clock as one touch at time t would.
+    __device__ void place_job(uint32_t pool, uint32_t g, uint32_t i, uint32_t P, uint32_t D, double tpf, bool from_buffer)
+    {
         const bool mixed = g < M;
         if (lane == (int)i) {
             ClassState &c = cs[i];
             const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
-            if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd - 1, t);
+            if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, from_buffer ? Qd - 1 : Qd, t);
             area_touch(c.aQd, c.Qd0 + c.Qd1, t);
-            if (pool) c.Qd1--; else c.Qd0--;
+            if (from_buffer) { if (pool) c.Qd1--; else c.Qd0--; }
             const double rel = __dsub_rn(t, T_reset);
             if (mixed) { c.sYm_in = __dadd_rn(c.sYm_in, rel); c.Ym++; c.placed_mixed++; }
             else       { c.sYs_in = __dadd_rn(c.sYs_in, rel); c.Ys++; c.placed_solo++; }
@@ -563,7 +590,7 @@ struct Sim {
             const uint32_t fin = it[g] + (running ? 1u : 0u) + D;
             const size_t o = (size_t)g * p.B + sl;
             s_fin[o] = fin;
-            s_tpf[o] = e.t;
+            s_tpf[o] = tpf;
             s_pk[o] = pack_job(P, D, i, mixed ? 1u : 0u);
             ndec[g] = (uint16_t)(sl + 1);
             nfin[g] = min(nfin[g], fin);
@@ -615,6 +642,7 @@ struct Sim {
             c.admitted++;
         }
         n_idle_pf--;
+        idle_hint = NONE32;
         if (lane == (int)(g & 31u)) {
             pfjob[g] = e.pk | 0x80000000u;
             pfrem[g] = job_P(e.pk);
@@ -653,8 +681,13 @@ struct Sim {
         if (drain_dirty && (dq_n0 | dq_n1)) {
             if (!f_sli()) {
                 while (dq_n0 > 0) {
-                    uint32_t g = choose_server(WANT_SOLO);
-                    if (g == NONE32) g = choose_server(WANT_MIX);
+                    uint32_t g;
+                    if (!f_random()) {
+                        g = choose_solo_first();
+                    } else {
+                        g = choose_server(WANT_SOLO);
+                        if (g == NONE32) g = choose_server(WANT_MIX);
+                    }
                     if (g == NONE32) break;
                     place_decode(0, g);
                     __syncwarp();
@@ -677,10 +710,11 @@ struct Sim {
         drain_dirty = false;
         // prefill gate on mixed GPUs whose prefill slot is idle
         if (gate_dirty) {
-            for (;;) {
+            while (n_idle_pf > 0) {
                 const uint32_t i = gate_class();
                 if (i == NONE32) break;
-                const uint32_t g = choose_server(WANT_PREFILL);
+                // a single idle slot whose GPU is known needs no search (and draws nothing: one candidate)
+                const uint32_t g = (n_idle_pf == 1 && idle_hint != NONE32) ? idle_hint : choose_server(WANT_PREFILL);
                 if (g == NONE32) break;
                 admit(i, g);
                 __syncwarp();
@@ -802,8 +836,6 @@ struct Sim {
                 draw(p, rep, (STREAM_SLI << 8) | i, ord, w0, w1, w2, w3);
                 pool = (u53(w0, w1) <= ps) ? 0u : 1u;
             }
-            const uint32_t n = pool ? dq_n1 : dq_n0;
-            const bool full = n >= p.qcap;
             if (lane == (int)i) {
                 ClassState &c = cs[i];
                 area_touch(c.aX, c.X, t);
@@ -814,31 +846,57 @@ struct Sim {
                 c.sum_ttft = __dadd_rn(c.sum_ttft, ttft);
                 if (f_hist()) hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)]++;
                 if (f_sli()) c.sli_ord++;
-                if (full) {
-                    c.overflow_d++;
-                } else {
-                    const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
-                    if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd + 1, t);
-                    area_touch(c.aQd, c.Qd0 + c.Qd1, t);
-                    if (pool) c.Qd1++; else c.Qd0++;
-                }
-            }
-            if (!full) {
-                uint32_t pos = (pool ? dq_head1 : dq_head0) + n;
-                if (pos >= p.qcap) pos -= p.qcap;
-                if (lane == 0) {
-                    QEntry e; e.t = t; e.pk = pack_job(P, D, i, 0); e.cls = i;
-                    dq[(size_t)pool * p.qcap + pos] = e;
-                }
-                if (pool) dq_n1++; else dq_n0++;
             }
             __syncwarp();   // every lane has read the finished job before its owner clears it
             if (lane == owner) pfjob[g] = 0;
-            drain_dirty = true;
+            __syncwarp();
+            // the prefill slot of g is idle again
+            if (!recount_idle && g < M && ndec[g] <= p.B - 1) {
+                n_idle_pf++;
+                idle_hint = (n_idle_pf == 1) ? g : NONE32;
+            }
+            // Decode stage.  With an empty buffer the request is its head at once: place it if a slot is free.
+            const uint32_t n = pool ? dq_n1 : dq_n0;
+            bool placed = false;
+            if (n == 0) {
+                uint32_t h;
+                if (f_sli()) {
+                    h = choose_server(pool == 0 ? WANT_SOLO : WANT_MIX);
+                } else if (!f_random()) {
+                    h = choose_solo_first();
+                } else {
+                    h = choose_server(WANT_SOLO);
+                    if (h == NONE32) h = choose_server(WANT_MIX);
+                }
+                if (h != NONE32) { place_job(pool, h, i, P, D, t, false); placed = true; }
+            }
+            if (!placed) {
+                const bool full = n >= p.qcap;
+                if (lane == (int)i) {
+                    ClassState &c = cs[i];
+                    if (full) {
+                        c.overflow_d++;
+                    } else {
+                        const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
+                        if (f_abandon()) ab_change(pool ? c.abd1 : c.abd0, p.cls[i].theta, Qd, Qd + 1, t);
+                        area_touch(c.aQd, c.Qd0 + c.Qd1, t);
+                        if (pool) c.Qd1++; else c.Qd0++;
+                    }
+                }
+                if (!full) {
+                    uint32_t pos = (pool ? dq_head1 : dq_head0) + n;
+                    if (pos >= p.qcap) pos -= p.qcap;
+                    if (lane == 0) {
+                        QEntry e; e.t = t; e.pk = pack_job(P, D, i, 0); e.cls = i;
+                        dq[(size_t)pool * p.qcap + pos] = e;
+                    }
+                    if (pool) dq_n1++; else dq_n0++;
+                }
+                drain_dirty = true;
+            }
             gate_dirty = true;
-            recount_idle = true;
         }
-        if (recount_idle) { __syncwarp(); n_idle_pf = count_idle_pf(); }
+        if (recount_idle) { __syncwarp(); n_idle_pf = count_idle_pf(); idle_hint = NONE32; }
         touch_server(g);
     }
 
@@ -982,7 +1040,7 @@ struct Sim {
                     else if (f_abandon() && src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
                     else if (f_abandon() && src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
                     else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
-                    else { ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true; n_idle_pf = count_idle_pf(); }
+                    else { ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true; n_idle_pf = count_idle_pf(); idle_hint = NONE32; }
                 }
                 if (err) return true;
                 dispatch();
@@ -1160,6 +1218,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.n_touch = 0; s.touch_all = false; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
         s.n_idle_pf = s.count_idle_pf();
+        s.idle_hint = NONE32;
         s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
         s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
         const bool finished = s.err ? true : s.run();
