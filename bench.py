@@ -189,7 +189,9 @@ def main():
         torch.cuda.synchronize()
 
     # replications are independent: rank k simulates global replications [k R, (k+1) R)  (weak scaling)
-    inp = presets.cfg1(R=args.reps).with_(rep_offset=rank * args.reps)
+    from paper_2602_02987_b200.sharding import shard
+    count, offset = shard(args.reps * world, world, rank)
+    inp = presets.cfg1(R=count).with_(rep_offset=offset)
     sim = QSim(inp, device=f"cuda:{local}")
     for _ in range(args.warmup):
         sim.run(args.horizon)

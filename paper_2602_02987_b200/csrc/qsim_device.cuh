@@ -290,6 +290,7 @@ struct Sim {
     uint32_t blk, M, dq_head0, dq_head1, dq_n0, dq_n1, n_touch, err;
     uint32_t n_idle_pf;          // mixed GPUs whose prefill slot is idle (and that may take a prefill)
     uint32_t idle_hint;          // when n_idle_pf == 1: that GPU if known, else NONE32
+    uint32_t need_start;         // per lane: rows of own GPUs touched by the current event
     unsigned long long place_ord, events, rounds;
     bool drain_dirty, gate_dirty, touch_all;
     // per-lane partial sums
@@ -550,9 +551,11 @@ struct Sim {
         return NONE32;
     }
 
+    // GPU g may have to start an iteration at the end of this event: noted in its owner's row mask
     __device__ __forceinline__ void touch_server(uint32_t g)
     {
-        if (n_touch < TOUCH_CAP) { if (lane == 0) touch[n_touch] = g; n_touch++; }
+        if (SPL > 0) { if (lane == (int)(g & 31u)) need_start |= 1u << (g >> 5); }
+        else if (n_touch < TOUCH_CAP) { if (lane == 0) touch[n_touch] = g; n_touch++; }
         else touch_all = true;
     }
 
@@ -723,7 +726,13 @@ struct Sim {
         gate_dirty = false;
         // start the next iteration on every GPU that was touched and is between iterations
         __syncwarp();
-        if (touch_all) {
+        if (SPL > 0) {
+            // every owner starts its touched GPUs; different lanes work in parallel
+#pragma unroll
+            for (uint32_t k = 0; k < (uint32_t)(SPL > 0 ? SPL : 1); ++k)
+                if (need_start & (1u << k)) start_if_needed((k << 5) + (uint32_t)lane);
+            need_start = 0;
+        } else if (touch_all) {
             for (uint32_t k = 0; k < n_rows(); ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 if (g < p.N) start_if_needed(g);
@@ -1215,7 +1224,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.load_block(h.blk);
         s.dq_head0 = h.dq_head0; s.dq_head1 = h.dq_head1; s.dq_n0 = h.dq_n0; s.dq_n1 = h.dq_n1;
         s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
-        s.n_touch = 0; s.touch_all = false; s.err = h.err;
+        s.n_touch = 0; s.touch_all = false; s.need_start = 0; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
         s.n_idle_pf = s.count_idle_pf();
         s.idle_hint = NONE32;
