@@ -45,7 +45,7 @@ constexpr int TOUCH_CAP = 48;
 // run time; otherwise the set bits say which features the instance contains and everything else is
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
-                   F_OCC = 128;
+                   F_OCC = 128, F_SLOTS = 256;
 
 // source ids: smaller id wins an exact tie in time
 constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
@@ -90,7 +90,7 @@ struct ClassPar { double theta; uint32_t P, D, prio, pad; };
 struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI]; };
 
 struct Params {
-    uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance, any_theta;
+    uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance, any_theta, slots_smem;
     unsigned long long seed, rep_offset, horizon_iters, event_budget;
     double block_len;
     double coef[6];
@@ -266,6 +266,8 @@ struct Sim {
     __device__ __forceinline__ bool f_blocks() const { return (F & F_GENERIC) ? p.nblk > 1 : (F & F_BLOCKS) != 0; }
     __device__ __forceinline__ bool f_random() const { return (F & F_GENERIC) ? p.placement == 0 : (F & F_RANDOM) != 0; }
     __device__ __forceinline__ bool f_occ() const { return (F & F_GENERIC) ? p.gate == 0 : (F & F_OCC) != 0; }
+    // finish stamps and slot occupancy of every simulated GPU live in shared memory (small N*B only)
+    __device__ __forceinline__ bool f_slots() const { return (F & F_GENERIC) ? p.slots_smem != 0 : (F & F_SLOTS) != 0; }
     __device__ __forceinline__ uint32_t n_rows() const { return SPL > 0 ? (uint32_t)SPL : (p.Npad >> 5); }
 
     const Params &p;
@@ -275,6 +277,8 @@ struct Sim {
     double *tnext, *pf_tarr;
     uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
     uint16_t *ndec, *nact, *pfcur;
+    uint16_t *sfin16;            // [Npad][B]  low 16 bits of each slot's finish iteration (f_slots)
+    uint32_t *socc;              // [Npad][ceil(B/32)]  slot occupancy bits; bits past B are set for good
     uint32_t *touch;
     double *gate_xi, *gate_dq;
     uint32_t *gate_ok;
@@ -591,8 +595,26 @@ struct Sim {
             const bool running = tnext[g] < dinf();
             // joins the iteration that starts next: a running iteration first finishes as it+1
             const uint32_t fin = it[g] + (running ? 1u : 0u) + D;
-            const size_t o = (size_t)g * p.B + sl;
-            s_fin[o] = fin;
+            size_t o;
+            if (f_slots()) {
+                // first free slot of the GPU's occupancy words
+                const uint32_t bw = (p.B + 31u) >> 5;
+                uint32_t slot = 0;
+                for (uint32_t w = 0; w < bw; ++w) {
+                    const uint32_t word = socc[g * bw + w];
+                    if (word != 0xffffffffu) {
+                        const uint32_t b = (uint32_t)__ffs((int)~word) - 1u;
+                        socc[g * bw + w] = word | (1u << b);
+                        slot = (w << 5) + b;
+                        break;
+                    }
+                }
+                sfin16[g * p.B + slot] = (uint16_t)fin;
+                o = (size_t)g * p.B + slot;
+            } else {
+                o = (size_t)g * p.B + sl;
+                s_fin[o] = fin;
+            }
             s_tpf[o] = tpf;
             s_pk[o] = pack_job(P, D, i, mixed ? 1u : 0u);
             ndec[g] = (uint16_t)(sl + 1);
@@ -749,8 +771,66 @@ struct Sim {
 
     // Some decode on GPU g emitted its last token in the iteration that ended at te (its it-th): the whole
     // warp scans the GPU's slot list from the tail, accounts every finished request and closes the gaps.
+    // Accounting of one finished request (uniform arguments; the class lane does the work).
+    __device__ __forceinline__ void account_done(uint32_t pk, double tpf, double te)
+    {
+        const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
+        if (lane == (int)i) {
+            ClassState &c = cs[i];
+            const double rel = __dsub_rn(te, T_reset);
+            if (job_flag(pk)) { c.sYm_out = __dadd_rn(c.sYm_out, rel); c.Ym--; c.done_mixed++; }
+            else              { c.sYs_out = __dadd_rn(c.sYs_out, rel); c.Ys--; c.done_solo++; }
+            c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
+            c.tok_out_done += D;
+            const double tpot = __ddiv_rn(__dsub_rn(te, tpf), (double)D);
+            c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
+            if (f_hist()) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
+        }
+    }
+
+    // retire_decodes when stamps and occupancy are in shared memory: every lane checks one slot per word of
+    // occupancy; the lanes that hit fetch their request records at the same time.
+    __device__ void retire_slots(uint32_t g, uint32_t itg, uint32_t nd, double te)
+    {
+        const int owner = (int)(g & 31u);
+        const uint32_t bw = (p.B + 31u) >> 5, it16 = itg & 0xffffu;
+        uint32_t newmin = NONE32, done = 0, Kdrop = 0;
+        for (uint32_t w = 0; w < bw; ++w) {
+            const uint32_t occ = socc[g * bw + w];
+            const uint32_t j = (w << 5) + (uint32_t)lane;
+            const bool live = ((occ >> lane) & 1u) != 0 && j < p.B;
+            const uint32_t dist = live ? (((uint32_t)sfin16[g * p.B + j] - it16) & 0xffffu) : NONE32;
+            const bool hit = live && dist == 0;
+            if (live && !hit) newmin = min(newmin, dist);
+            uint32_t hits = __ballot_sync(FULL, hit);
+            if (hits) {
+                double tpf = 0.0;
+                uint32_t pk = 0;
+                if (hit) { tpf = s_tpf[(size_t)g * p.B + j]; pk = s_pk[(size_t)g * p.B + j]; }
+                if (lane == owner) socc[g * bw + w] = occ & ~hits;
+                done += (uint32_t)__popc(hits);
+                while (hits) {
+                    const int hl = __ffs((int)hits) - 1;
+                    hits &= hits - 1;
+                    const uint32_t pkh = __shfl_sync(FULL, pk, hl);
+                    const double tpfh = __shfl_sync(FULL, tpf, hl);
+                    account_done(pkh, tpfh, te);
+                    Kdrop += job_P(pkh) + job_D(pkh);
+                }
+            }
+        }
+        newmin = __reduce_min_sync(FULL, newmin);
+        if (lane == owner) {
+            ndec[g] = (uint16_t)(nd - done);
+            nfin[g] = newmin == NONE32 ? NONE32 : itg + newmin;
+            if (f_kappa()) K[g] -= Kdrop;
+        }
+        __syncwarp();
+    }
+
     __device__ void retire_decodes(uint32_t g, uint32_t itg, uint32_t nd, double te)
     {
+        if (f_slots()) { retire_slots(g, itg, nd, te); return; }
         const int owner = (int)(g & 31u);
         uint32_t n = nd, newmin = NONE32, Kdrop = 0;
         const size_t base = (size_t)g * p.B;
@@ -766,18 +846,8 @@ struct Sim {
                 const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
                 const double tpf = s_tpf[base + h];
                 const uint32_t pk = s_pk[base + h];
-                const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
-                if (lane == (int)i) {
-                    ClassState &c = cs[i];
-                    const double rel = __dsub_rn(te, T_reset);
-                    if (job_flag(pk)) { c.sYm_out = __dadd_rn(c.sYm_out, rel); c.Ym--; c.done_mixed++; }
-                    else              { c.sYs_out = __dadd_rn(c.sYs_out, rel); c.Ys--; c.done_solo++; }
-                    c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
-                    c.tok_out_done += D;
-                    const double tpot = __ddiv_rn(__dsub_rn(te, tpf), (double)D);
-                    c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
-                    if (f_hist()) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
-                }
+                account_done(pk, tpf, te);
+                const uint32_t P = job_P(pk), D = job_D(pk);
                 Kdrop += P + D;
                 const uint32_t last = n - 1;
                 __syncwarp();
@@ -1075,10 +1145,10 @@ struct Sim {
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
     uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
-        off_pfcur, srv_bytes, off_touch, off_gate, off_cs, off_ring, total;
+        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
+__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem)
 {
     SmemLayout L;
     uint32_t o = 0;
@@ -1093,6 +1163,10 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad)
     L.off_ndec = o; o += 2 * Npad;
     L.off_nact = o; o += 2 * Npad;
     L.off_pfcur = o; o += 2 * Npad;
+    o = (o + 15u) & ~15u;
+    L.off_sfin16 = o; if (slots_smem) o += 2 * Npad * B;
+    o = (o + 15u) & ~15u;
+    L.off_socc = o; if (slots_smem) o += 4 * Npad * ((B + 31u) >> 5);
     o = (o + 15u) & ~15u;
     L.srv_bytes = o;
     L.off_touch = o; o += 4 * TOUCH_CAP;
@@ -1120,6 +1194,8 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.ndec = reinterpret_cast<uint16_t *>(sm + L.off_ndec);
     s.nact = reinterpret_cast<uint16_t *>(sm + L.off_nact);
     s.pfcur = reinterpret_cast<uint16_t *>(sm + L.off_pfcur);
+    s.sfin16 = reinterpret_cast<uint16_t *>(sm + L.off_sfin16);
+    s.socc = reinterpret_cast<uint32_t *>(sm + L.off_socc);
     s.touch = reinterpret_cast<uint32_t *>(sm + L.off_touch);
     s.gate_xi = reinterpret_cast<double *>(sm + L.off_gate);
     s.gate_dq = s.gate_xi + MAXI;
@@ -1145,13 +1221,17 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
     extern __shared__ __align__(16) char sm[];
     const int lane = threadIdx.x;
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
-        const SmemLayout L = smem_layout(p.Npad);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem);
         Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();
         for (uint32_t o = lane * 4; o < L.total; o += 128) *reinterpret_cast<uint32_t *>(sm + o) = 0;
         __syncwarp();
         for (uint32_t g = lane; g < p.Npad; g += 32) { s.tnext[g] = dinf(); s.nfin[g] = NONE32; }
+        if (p.slots_smem && (p.B & 31u)) {
+            const uint32_t bw = (p.B + 31u) >> 5;
+            for (uint32_t g = lane; g < p.Npad; g += 32) s.socc[g * bw + bw - 1] = ~0u << (p.B & 31u);
+        }
         if (lane < MAXI) {
             ClassState &c = s.cs[lane];
             c.ta = dinf();
@@ -1199,7 +1279,7 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
-        const SmemLayout L = smem_layout(p.Npad);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem);
         Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();

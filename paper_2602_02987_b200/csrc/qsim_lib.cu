@@ -131,10 +131,10 @@ struct RunVariant { int spl; uint32_t feat; RunKernel fn; };
 template <int SPL>
 void add_variants(std::vector<RunVariant> &v)
 {
-    v.push_back({SPL, 0u, qsim_run_kernel<SPL, 0u>});
-    v.push_back({SPL, F_OCC, qsim_run_kernel<SPL, F_OCC>});
-    v.push_back({SPL, F_OCC | F_ABANDON, qsim_run_kernel<SPL, F_OCC | F_ABANDON>});
-    v.push_back({SPL, F_OCC | F_ABANDON | F_RANDOM, qsim_run_kernel<SPL, F_OCC | F_ABANDON | F_RANDOM>});
+    v.push_back({SPL, F_SLOTS, qsim_run_kernel<SPL, F_SLOTS>});
+    v.push_back({SPL, F_SLOTS | F_OCC, qsim_run_kernel<SPL, F_SLOTS | F_OCC>});
+    v.push_back({SPL, F_SLOTS | F_OCC | F_ABANDON, qsim_run_kernel<SPL, F_SLOTS | F_OCC | F_ABANDON>});
+    v.push_back({SPL, F_SLOTS | F_OCC | F_ABANDON | F_RANDOM, qsim_run_kernel<SPL, F_SLOTS | F_OCC | F_ABANDON | F_RANDOM>});
     v.push_back({SPL, F_GENERIC, qsim_run_kernel<SPL, F_GENERIC>});
 }
 
@@ -185,7 +185,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
         if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
         // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits
         // (abandonment, KV slope, blocks) may be present without being used
-        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_HIST;
+        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_HIST | F_SLOTS;
         if (feat == ~0u || (feat & MODES) != (v.feat & MODES) || (feat & ~v.feat) != 0) continue;
         const int extra = __builtin_popcount(v.feat & ~feat);
         if (extra < best_bits) { best = &v; best_bits = extra; }
@@ -244,11 +244,15 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
     {
         // the per-GPU arrays are padded to the unrolled row count of the chosen instance
-        const RunVariant v = pick_run_kernel(cfg->N, features_of(*cfg, classes, coef));
-        h->run_fn = v.fn;
+        uint32_t feat = features_of(*cfg, classes, coef);
+        RunVariant v = pick_run_kernel(cfg->N, feat);
         if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
+        // finish stamps + occupancy bits go to shared memory when the whole block state stays small
+        p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
+        if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
+        h->run_fn = v.fn;
     }
-    h->lay = smem_layout(p.Npad);
+    h->lay = smem_layout(p.Npad, p.B, p.slots_smem);
     p.srv_bytes = h->lay.srv_bytes;
     if (h->lay.total > 227u * 1024u) {
         delete h;
@@ -597,11 +601,14 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.any_theta = 0;
     for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
     {
-        const RunVariant v = pick_run_kernel(cfg->N, features_of(nohist_features(*cfg), classes, coef));
-        h.run_fn = v.fn;
+        uint32_t feat = features_of(nohist_features(*cfg), classes, coef);
+        RunVariant v = pick_run_kernel(cfg->N, feat);
         if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
+        p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
+        if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
+        h.run_fn = v.fn;
     }
-    h.lay = smem_layout(p.Npad);
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem);
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     qsim_config nohist = *cfg;
