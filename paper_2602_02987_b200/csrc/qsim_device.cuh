@@ -274,7 +274,7 @@ struct Sim {
     const int lane;
     const uint32_t rep;
     // shared memory (lane-owned entries)
-    double *tnext, *pf_tarr;
+    double *tnext, *pf_tarr, *taucur;      // taucur: duration of the running iteration
     uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
     uint16_t *ndec, *nact, *pfcur;
     uint16_t *sfin16;            // [Npad][B]  low 16 bits of each slot's finish iteration (f_slots)
@@ -693,7 +693,9 @@ struct Sim {
                 uint32_t fl = (nfin[g] == it[g] + 1u) ? 0x4000u : 0u;
                 if (pc > 0 && pc == rem) fl |= 0x8000u;
                 nact[g] = (uint16_t)(nd | fl);
-                tnext[g] = __dadd_rn(ts, iter_time(p, pc, nd, Kg, f_kappa()));
+                const double tau = iter_time(p, pc, nd, Kg, f_kappa());
+                taucur[g] = tau;
+                tnext[g] = __dadd_rn(ts, tau);
             }
         }
     }
@@ -878,7 +880,7 @@ struct Sim {
             itg = it[g] + 1;
             it[g] = itg;
             const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
-            const double tau = iter_time(p, pc, na, Kg, f_kappa());
+            const double tau = taucur[g];
             if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
             if (f_kappa()) K[g] = Kg + na;
@@ -986,16 +988,29 @@ struct Sim {
     {
         const uint32_t itg = it[g] + 1u;
         it[g] = itg;
-        const uint32_t na_raw = nact[g], na = na_raw & 0x3fffu, pc = pfcur[g];
-        uint32_t Kg = 0;
-        if (f_kappa()) { Kg = K[g]; K[g] = Kg + na; }
-        const double tau = iter_time(p, pc, na, Kg, f_kappa());
-        if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] -= pc; }
+        const uint32_t na_raw = nact[g], pc = pfcur[g];
+        const double tau = taucur[g];
+        if (f_kappa()) K[g] += na_raw & 0x3fffu;
+        uint32_t rem = 0;
+        if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); rem = pfrem[g] - pc; pfrem[g] = rem; }
         else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
-        pfcur[g] = 0;
-        tnext[g] = dinf();
-        if (na_raw & 0x4000u) return true;
-        start_at(g, te);
+        if (na_raw & 0x4000u) { pfcur[g] = 0; tnext[g] = dinf(); return true; }
+        // restart at te with what the GPU holds now (requests placed meanwhile join here)
+        const uint32_t nd = ndec[g];
+        const uint32_t pj = pfjob[g];
+        const bool has_pf = (pj >> 31) != 0;
+        if (nd == 0 && !has_pf) { pfcur[g] = 0; tnext[g] = dinf(); return false; }
+        if (has_pf && pc == 0) rem = pfrem[g];
+        uint32_t Kg = 0;
+        if (f_kappa()) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
+        const uint32_t pc2 = has_pf ? min(p.C, rem) : 0u;
+        uint32_t fl = (nfin[g] == itg + 1u) ? 0x4000u : 0u;
+        if (pc2 > 0 && pc2 == rem) fl |= 0x8000u;
+        const double tau2 = iter_time(p, pc2, nd, Kg, f_kappa());
+        pfcur[g] = (uint16_t)pc2;
+        nact[g] = (uint16_t)(nd | fl);
+        taucur[g] = tau2;
+        tnext[g] = __dadd_rn(te, tau2);
         return false;
     }
 
@@ -1031,13 +1046,18 @@ struct Sim {
                 }
             }
             const bool buffered = (dq_n0 | dq_n1) != 0;
+            constexpr int NC = SPL > 0 ? SPL : 1;       // per-row values kept in registers when the rows unroll
+            unsigned long long vrow[NC];
+            bool lrow[NC];
 #pragma unroll
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
                 const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+                const bool loc = v < INF && is_local(g, buffered);
+                if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
                 if (v < INF) {
                     tmin = min(tmin, v);
-                    if (!is_local(g, buffered) && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                    if (!loc && v < bt) { bt = v; bs = SRC_SERVER + g; }
                 }
             }
             // warp argmin of (time bits, source id) over non-local events; warp min over all iteration ends
@@ -1077,27 +1097,52 @@ struct Sim {
                     progressed = true;
                 }
             }
+            // pass 1: every lane ends the local iterations of its own GPUs (straight-line over the rows)
+            uint32_t retire_rows = 0;
 #pragma unroll
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
-                const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-                bool retire = false;
-                if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
-                    retire = local_end(g, __longlong_as_double((long long)v));
+                unsigned long long v;
+                bool loc;
+                if (SPL > 0) { v = vrow[k]; loc = lrow[k]; }
+                else { v = (unsigned long long)__double_as_longlong(tnext[g]); loc = v < INF && is_local(g, buffered); }
+                if (loc && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+                    if (local_end(g, __longlong_as_double((long long)v))) retire_rows |= 1u << (k & 31u);
                     progressed = true;
                 }
-                uint32_t need = __ballot_sync(FULL, retire);
-                any_retire |= need;
-                __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
-                // decode completions found in this row: retired by the whole warp, GPU by GPU
-                while (need) {
-                    const int l = __ffs((int)need) - 1;
-                    need &= need - 1;
-                    const uint32_t gg = (k << 5) + (uint32_t)l;
-                    const unsigned long long vv = __shfl_sync(FULL, v, l);
-                    const double te = __longlong_as_double((long long)vv);
-                    retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
-                    if (lane == l) start_at(gg, te);
+                if (SPL == 0) {
+                    // run-time row count: retire per row (the row mask has only 32 bits)
+                    uint32_t need = __ballot_sync(FULL, retire_rows != 0);
+                    any_retire |= need;
+                    __syncwarp();
+                    while (need) {
+                        const int l = __ffs((int)need) - 1;
+                        need &= need - 1;
+                        const uint32_t gg = (k << 5) + (uint32_t)l;
+                        const double te = __longlong_as_double((long long)__shfl_sync(FULL, v, l));
+                        retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
+                        if (lane == l) start_at(gg, te);
+                    }
+                    retire_rows = 0;
+                }
+            }
+            if (SPL > 0) {
+                // pass 2: decode completions found in pass 1, retired by the whole warp, GPU by GPU
+                any_retire = __ballot_sync(FULL, retire_rows != 0);
+                if (any_retire) {
+                    __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
+#pragma unroll
+                    for (uint32_t k = 0; k < rows; ++k) {
+                        uint32_t need = __ballot_sync(FULL, (retire_rows >> k) & 1u);
+                        while (need) {
+                            const int l = __ffs((int)need) - 1;
+                            need &= need - 1;
+                            const uint32_t gg = (k << 5) + (uint32_t)l;
+                            const double te = __longlong_as_double((long long)__shfl_sync(FULL, vrow[k], l));
+                            retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
+                            if (lane == l) start_at(gg, te);
+                        }
+                    }
                 }
             }
             (void)any_retire;
@@ -1144,7 +1189,7 @@ struct Sim {
 
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
-    uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
+    uint32_t off_tnext, off_tarr, off_tau, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
         off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, total;
 };
 
@@ -1154,6 +1199,7 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     uint32_t o = 0;
     L.off_tnext = o; o += 8 * Npad;
     L.off_tarr = o; o += 8 * Npad;
+    L.off_tau = o; o += 8 * Npad;
     L.off_it = o; o += 4 * Npad;
     L.off_nfin = o; o += 4 * Npad;
     L.off_pfrem = o; o += 4 * Npad;
@@ -1185,6 +1231,7 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
 {
     s.tnext = reinterpret_cast<double *>(sm + L.off_tnext);
     s.pf_tarr = reinterpret_cast<double *>(sm + L.off_tarr);
+    s.taucur = reinterpret_cast<double *>(sm + L.off_tau);
     s.it = reinterpret_cast<uint32_t *>(sm + L.off_it);
     s.nfin = reinterpret_cast<uint32_t *>(sm + L.off_nfin);
     s.pfrem = reinterpret_cast<uint32_t *>(sm + L.off_pfrem);
