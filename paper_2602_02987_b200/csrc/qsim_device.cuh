@@ -83,6 +83,8 @@ struct RepHeader {
 static_assert(sizeof(ClassState) % 8 == 0 && (sizeof(ClassState) * MAXI) % 16 == 0, "ClassState is copied in 16-byte words");
 static_assert(sizeof(RepHeader) % 16 == 0 && offsetof(RepHeader, cs) % 16 == 0, "RepHeader layout");
 
+struct SlotRec { double tpf; uint32_t pk; uint32_t pad; };  // request in a decode slot: prefill end time, packed lengths/class/group
+constexpr int STAGE_CAP = 64;                                 // finished-request records waiting for their accounting
 struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential and packed lengths
 struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
 
@@ -101,8 +103,7 @@ struct Params {
     RepHeader *hdr;
     char *srv;                   // per replication: server structure-of-arrays image, srv_bytes each
     uint32_t *slot_fin;          // [R][N][B]
-    double *slot_tpf;            // [R][N][B]
-    uint32_t *slot_pk;           // [R][N][B]
+    SlotRec *slot_rec;           // [R][N][B]
     QEntry *pq;                  // [R][I][qcap]
     QEntry *dq;                  // [R][2][qcap]
     uint32_t *hist_mem;          // [R][I][2][NBIN] or null
@@ -223,6 +224,14 @@ __device__ __forceinline__ void ab_change(AbClock &c, double theta, uint32_t Q_o
     }
 }
 
+// 16-byte asynchronous copy global -> shared (L2 only), and the wait for this thread's copies
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+
 // 1 + #{j < LMAX-1 : thr[j] <= w} by binary search
 __device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, uint32_t w)
 {
@@ -285,8 +294,12 @@ struct Sim {
     ClassState *cs;
     // global memory of this replication
     uint32_t *s_fin;
-    double *s_tpf;
-    uint32_t *s_pk;
+    SlotRec *s_rec;
+    // shared-memory staging: records of finished requests (copied asynchronously) and queue-head copies
+    SlotRec *st_rec;
+    double *st_te;
+    QEntry *pqh;
+    uint32_t n_pend;
     QEntry *pq, *dq;
     uint32_t *hist;
     // replicated scalars
@@ -391,6 +404,7 @@ struct Sim {
             if (pos >= p.qcap) pos -= p.qcap;
             QEntry e; e.t = ta; e.pk = pack_job(c.nextP, c.nextD, i, 0); e.cls = i;
             pq[(size_t)i * p.qcap + pos] = e;
+            if (c.pq_n == 0) pqh[i] = e;        // it is the head: keep a copy on chip
             c.pq_n++;
         }
         schedule_from(ta);
@@ -442,9 +456,12 @@ struct Sim {
         uint32_t w0, w1, w2, w3;
         draw(p, rep, (STREAM_ABANDON_P << 8) | i, m, w0, w1, w2, w3);
         const uint32_t rank = __umulhi(w2, Q);       // uniformly chosen waiting job, in FCFS rank
+        cp_async_wait_all();
+        __syncwarp();
         ring_remove(pq + (size_t)i * p.qcap, head, Q, rank);
         if (lane == (int)i) {
             ClassState &c = cs[i];
+            if (Q > 1) pqh[i] = pq[(size_t)i * p.qcap + head];     // the head may have changed
             area_touch(c.aQp, Q, t);
             c.pq_n = Q - 1;
             c.abandoned_p++;
@@ -615,8 +632,8 @@ struct Sim {
                 o = (size_t)g * p.B + sl;
                 s_fin[o] = fin;
             }
-            s_tpf[o] = tpf;
-            s_pk[o] = pack_job(P, D, i, mixed ? 1u : 0u);
+            SlotRec r; r.tpf = tpf; r.pk = pack_job(P, D, i, mixed ? 1u : 0u); r.pad = 0;
+            s_rec[o] = r;
             ndec[g] = (uint16_t)(sl + 1);
             nfin[g] = min(nfin[g], fin);
             if (f_kappa()) Kpend[g] += P;
@@ -654,14 +671,19 @@ struct Sim {
 
     __device__ void admit(uint32_t i, uint32_t g)
     {
-        const uint32_t head = __shfl_sync(FULL, cs[lane & 7].pq_head, i);
-        const QEntry e = pq[(size_t)i * p.qcap + head];
+        // the head of the class queue is kept in shared memory (copied there asynchronously after each pop)
+        cp_async_wait_all();
+        __syncwarp();
+        const QEntry e = pqh[i];
+        __syncwarp();
         if (lane == (int)i) {
             ClassState &c = cs[i];
+            const uint32_t head = c.pq_head;
             if (f_abandon()) ab_change(c.abp, p.cls[i].theta, c.pq_n, c.pq_n - 1, t);
             area_touch(c.aQp, c.pq_n, t);
             c.pq_n--;
             c.pq_head = (head + 1 == p.qcap) ? 0 : head + 1;
+            if (c.pq_n > 0) cp_async16(&pqh[i], &pq[(size_t)i * p.qcap + c.pq_head]);
             area_touch(c.aX, c.X, t);
             c.X++;
             c.admitted++;
@@ -790,6 +812,19 @@ struct Sim {
         }
     }
 
+    // Accounting of the finished requests whose records were staged in shared memory.
+    __device__ void flush_done()
+    {
+        cp_async_wait_all();
+        __syncwarp();
+        for (uint32_t e = 0; e < n_pend; ++e) {
+            const SlotRec r = st_rec[e];
+            account_done(r.pk, r.tpf, st_te[e]);
+        }
+        n_pend = 0;
+        __syncwarp();
+    }
+
     // retire_decodes when stamps and occupancy are in shared memory: every lane checks one slot per word of
     // occupancy; the lanes that hit fetch their request records at the same time.
     __device__ void retire_slots(uint32_t g, uint32_t itg, uint32_t nd, double te)
@@ -806,18 +841,28 @@ struct Sim {
             if (live && !hit) newmin = min(newmin, dist);
             uint32_t hits = __ballot_sync(FULL, hit);
             if (hits) {
-                double tpf = 0.0;
-                uint32_t pk = 0;
-                if (hit) { tpf = s_tpf[(size_t)g * p.B + j]; pk = s_pk[(size_t)g * p.B + j]; }
                 if (lane == owner) socc[g * bw + w] = occ & ~hits;
                 done += (uint32_t)__popc(hits);
-                while (hits) {
-                    const int hl = __ffs((int)hits) - 1;
-                    hits &= hits - 1;
-                    const uint32_t pkh = __shfl_sync(FULL, pk, hl);
-                    const double tpfh = __shfl_sync(FULL, tpf, hl);
-                    account_done(pkh, tpfh, te);
-                    Kdrop += job_P(pkh) + job_D(pkh);
+                if (!f_kappa()) {
+                    // the records only feed statistics: copy them on chip asynchronously, account later
+                    if (n_pend + 32u > (uint32_t)STAGE_CAP) flush_done();
+                    if (hit) {
+                        const uint32_t pos = n_pend + (uint32_t)__popc(hits & ((1u << lane) - 1u));
+                        cp_async16(&st_rec[pos], &s_rec[(size_t)g * p.B + j]);
+                        st_te[pos] = te;
+                    }
+                    n_pend += (uint32_t)__popc(hits);
+                } else {
+                    SlotRec r; r.tpf = 0.0; r.pk = 0;
+                    if (hit) r = s_rec[(size_t)g * p.B + j];
+                    while (hits) {
+                        const int hl = __ffs((int)hits) - 1;
+                        hits &= hits - 1;
+                        const uint32_t pkh = __shfl_sync(FULL, r.pk, hl);
+                        const double tpfh = __shfl_sync(FULL, r.tpf, hl);
+                        account_done(pkh, tpfh, te);
+                        Kdrop += job_P(pkh) + job_D(pkh);
+                    }
                 }
             }
         }
@@ -846,8 +891,9 @@ struct Sim {
                 const int hl = 31 - __clz(hits);
                 hits &= ~(1u << hl);
                 const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
-                const double tpf = s_tpf[base + h];
-                const uint32_t pk = s_pk[base + h];
+                const SlotRec rh = s_rec[base + h];
+                const double tpf = rh.tpf;
+                const uint32_t pk = rh.pk;
                 account_done(pk, tpf, te);
                 const uint32_t P = job_P(pk), D = job_D(pk);
                 Kdrop += P + D;
@@ -855,8 +901,7 @@ struct Sim {
                 __syncwarp();
                 if (lane == 0 && h != last) {
                     s_fin[base + h] = s_fin[base + last];
-                    s_tpf[base + h] = s_tpf[base + last];
-                    s_pk[base + h] = s_pk[base + last];
+                    s_rec[base + h] = s_rec[base + last];
                 }
                 n = last;
             }
@@ -1190,7 +1235,7 @@ struct Sim {
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
     uint32_t off_tnext, off_tarr, off_tau, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
-        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, total;
+        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, total;
 };
 
 __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem)
@@ -1222,6 +1267,9 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
     o = (o + 15u) & ~15u;
     L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * MAXI;
+    L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * STAGE_CAP;
+    L.off_stte = o; o += 8 * STAGE_CAP;
+    L.off_pqh = o; o += (uint32_t)sizeof(QEntry) * MAXI;
     L.total = (o + 15u) & ~15u;
     return L;
 }
@@ -1249,12 +1297,15 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.gate_ok = reinterpret_cast<uint32_t *>(s.gate_dq + MAXI);
     s.cs = reinterpret_cast<ClassState *>(sm + L.off_cs);
     s.aring = reinterpret_cast<ADraw *>(sm + L.off_ring);
+    s.st_rec = reinterpret_cast<SlotRec *>(sm + L.off_strec);
+    s.st_te = reinterpret_cast<double *>(sm + L.off_stte);
+    s.pqh = reinterpret_cast<QEntry *>(sm + L.off_pqh);
+    s.n_pend = 0;
     s.ring_n = 0; s.ring_pos = 0; s.sched_pending = false; s.t0_pending = 0.0;
     const Params &p = s.p;
     const size_t r = s.rep;
     s.s_fin = p.slot_fin + r * (size_t)p.N * p.B;
-    s.s_tpf = p.slot_tpf + r * (size_t)p.N * p.B;
-    s.s_pk = p.slot_pk + r * (size_t)p.N * p.B;
+    s.s_rec = p.slot_rec + r * (size_t)p.N * p.B;
     s.pq = p.pq + r * (size_t)p.I * p.qcap;
     s.dq = p.dq + r * (size_t)2 * p.qcap;
     s.hist = p.hist_mem ? p.hist_mem + r * (size_t)p.I * 2 * NBIN : nullptr;
@@ -1355,9 +1406,12 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.drain_dirty = true; s.gate_dirty = true;
         s.n_idle_pf = s.count_idle_pf();
         s.idle_hint = NONE32;
+        if (lane < (int)p.I && s.cs[lane].pq_n > 0) s.pqh[lane] = s.pq[(size_t)lane * p.qcap + s.cs[lane].pq_head];
+        __syncwarp();
         s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
         s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
         const bool finished = s.err ? true : s.run();
+        s.flush_done();
         if (lane < (int)p.I) s.cs[lane].adraw -= s.ring_n;     // unused arrival draws are produced again next time
         __syncwarp();
         // stage back

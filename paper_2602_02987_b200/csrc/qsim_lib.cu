@@ -35,7 +35,7 @@ int fail(int code, const std::string &msg)
 size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 struct Sections {
-    size_t hdr, srv, fin, tpf, pk, pq, dq, hist, flag, total;
+    size_t hdr, srv, fin, rec, pq, dq, hist, flag, total;
 };
 
 }  // namespace
@@ -68,8 +68,7 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
     s.hdr = o; o = align256(o + R * sizeof(RepHeader));
     s.srv = o; o = align256(o + R * (size_t)srv_bytes);
     s.fin = o; o = align256(o + R * NB * 4);
-    s.tpf = o; o = align256(o + R * NB * 8);
-    s.pk = o; o = align256(o + R * NB * 4);
+    s.rec = o; o = align256(o + R * NB * sizeof(SlotRec));
     s.pq = o; o = align256(o + R * (size_t)c.I * c.qcap * sizeof(QEntry));
     s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
     s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
@@ -318,8 +317,7 @@ int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
     p.hdr = reinterpret_cast<RepHeader *>(base + h->sec.hdr);
     p.srv = base + h->sec.srv;
     p.slot_fin = reinterpret_cast<uint32_t *>(base + h->sec.fin);
-    p.slot_tpf = reinterpret_cast<double *>(base + h->sec.tpf);
-    p.slot_pk = reinterpret_cast<uint32_t *>(base + h->sec.pk);
+    p.slot_rec = reinterpret_cast<SlotRec *>(base + h->sec.rec);
     p.pq = reinterpret_cast<QEntry *>(base + h->sec.pq);
     p.dq = reinterpret_cast<QEntry *>(base + h->sec.dq);
     p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
@@ -641,8 +639,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.hdr = reinterpret_cast<RepHeader *>(base + h.sec.hdr);
     p.srv = base + h.sec.srv;
     p.slot_fin = reinterpret_cast<uint32_t *>(base + h.sec.fin);
-    p.slot_tpf = reinterpret_cast<double *>(base + h.sec.tpf);
-    p.slot_pk = reinterpret_cast<uint32_t *>(base + h.sec.pk);
+    p.slot_rec = reinterpret_cast<SlotRec *>(base + h.sec.rec);
     p.pq = reinterpret_cast<QEntry *>(base + h.sec.pq);
     p.dq = reinterpret_cast<QEntry *>(base + h.sec.dq);
     p.hist_mem = nullptr;
