@@ -32,6 +32,10 @@ METRIC = "simulated GPU-server-iterations/sec"
 UNIT = "server-iterations/s"
 JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
                            # decode-buffer pass, each written and read once at 32-byte sector granularity
+# DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from the ncu capture summarised in
+# profiles/qsim_run_kernel_cfg1_lookahead.md (740.6 MB for 1.414e8 iterations; traffic grows with the iterations
+# of a launch, so a full launch is that figure times its iterations)
+NCU_DRAM_BYTES_PER_ITER = 740.6e6 / 1.414e8
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
 R_PER_GPU = 1024
 
@@ -264,7 +268,9 @@ def main():
                        "events_per_iteration": events / iters, "requests_per_iteration": jobs / iters,
                        "queue_overflow": ovf},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None, "peak_kind": peak_kind,
+                         "traffic": NCU_DRAM_BYTES_PER_ITER * iters / world / max(n_launch / world, 1.0),
+                         "traffic_source": "ncu capture of a 2000-iteration launch, scaled by iterations",
+                         "peak_kind": peak_kind,
                          "bytes_per_iteration": JOB_BYTES * jobs / iters,
                          "note": "latency/issue-bound event chain; HBM fraction is the contract figure"},
             "clocks": clocks, "gpu_launches": int(n_launch), "wall_s": wall,
