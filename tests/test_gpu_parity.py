@@ -174,3 +174,50 @@ def test_bad_arguments_are_rejected():
                 good.with_(coeffs=np.array([0.0, 1e-5, 0, 0.005, 0, 0]))):
         with pytest.raises(QSimError):
             QSim(bad)
+
+
+def test_cfg1_full_size_in_the_bench_launch_configuration():
+    """The benchmark's own launch (R = 1024 replications, 10^5 iterations of horizon in one qsim_run): sampled
+    replications against the oracle one by one, and the flow-balance identities (Eq. (15)-(20)) on all of them."""
+    import threading
+    from oracle import OracleSim
+    from paper_2602_02987_b200 import QSim
+    inp = presets.cfg1(R=1024)
+    H = 100_000
+    sim = QSim(inp)
+    sim.run(H)
+    g = sim.stats()
+    sim.close()
+    sample = [0, 517, 1023]
+    ref = {}
+
+    def one(r):
+        o = OracleSim(inp.with_(R=1, rep_offset=r))
+        o.run(H)
+        ref[r] = o.stats()
+        o.close()
+
+    threads = [threading.Thread(target=one, args=(r,)) for r in sample]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    for r in sample:
+        got = {k: v[r:r + 1] for k, v in g.items()}
+        assert_parity(got, ref[r], what=f"cfg1 full size, replication {r}")
+    u = {k: v.astype(np.int64) for k, v in g.items() if v.dtype.kind in "ui"}
+    assert np.array_equal(u["Qp"], u["arrivals"] - u["admitted"] - u["abandoned_p"] - u["overflow"])
+    assert np.array_equal(u["X"], u["admitted"] - u["prefill_done"])
+    assert np.array_equal(u["Qd"], u["prefill_done"] - u["placed_mixed"] - u["placed_solo"] - u["abandoned_d"] - u["overflow_d"])
+    assert np.array_equal(u["Ym"], u["placed_mixed"] - u["done_mixed"])
+    assert np.array_equal(u["Ys"], u["placed_solo"] - u["done_solo"])
+    assert u["overflow"].sum() == 0 and u["overflow_d"].sum() == 0
+    its = (u["iters_mixed"] + u["iters_solo"])
+    assert its.min() > 6_000_000
+    # Poisson arrivals: counts across replications have mean n lambda T and dispersion 1
+    T = g["T_elapsed"][0]
+    for i in range(inp.I):
+        mean = inp.N * inp.rates[0, i] * T
+        a = g["arrivals"][:, i].astype(float)
+        assert abs(a.mean() - mean) < 5.0 * np.sqrt(mean / a.size)
+        assert abs(a.var(ddof=1) / mean - 1.0) < 5.0 * np.sqrt(2.0 / (a.size - 1))
