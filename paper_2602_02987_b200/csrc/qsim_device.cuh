@@ -45,7 +45,14 @@ constexpr int TOUCH_CAP = 48;
 // run time; otherwise the set bits say which features the instance contains and everything else is
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
-                   F_OCC = 128, F_SLOTS = 256;
+                   F_OCC = 128, F_SLOTS = 256, F_MW = 512;
+// F_MW: several warps per replication.  Warp 0 (the master) runs the round loop and every event handler; the
+// other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
+// round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
+enum { MW_SCAN = 1, MW_ENDS = 2, MW_EXIT = 3 };
+struct MwCmd { unsigned long long lim_t; uint32_t op, lim_s, buffered, M; };
+struct MwRes { unsigned long long bt, tmin; uint32_t bs, progressed; };
+constexpr int MW_MAX = 16;
 
 // source ids: smaller id wins an exact tie in time
 constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
@@ -85,6 +92,8 @@ static_assert(sizeof(RepHeader) % 16 == 0 && offsetof(RepHeader, cs) % 16 == 0, 
 
 struct SlotRec { double tpf; uint32_t pk; uint32_t pad; };  // request in a decode slot: prefill end time, packed lengths/class/group
 constexpr int STAGE_CAP = 64;                                 // finished-request records waiting for their accounting
+// Accounting of finished requests, one block per warp (merged into the class records at kernel exit)
+struct WarpClassStats { double sYm_out, sYs_out, sum_tpot; unsigned long long tok_in, tok_out; uint32_t done_mixed, done_solo; };
 struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential and packed lengths
 struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
 
@@ -282,6 +291,10 @@ struct Sim {
     const Params &p;
     const int lane;
     const uint32_t rep;
+    int warp, nwarps;            // position in the block (F_MW); 0 / 1 otherwise
+    MwCmd *cmd;
+    MwRes *res;
+    WarpClassStats *wcs;         // [nwarps][MAXI]
     // shared memory (lane-owned entries)
     double *tnext, *pf_tarr, *taucur;      // taucur: duration of the running iteration
     uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
@@ -321,7 +334,8 @@ struct Sim {
     // block parameters of the current block (lane i holds class i)
     double b_xstar, b_nx, b_nq, b_ps;
 
-    __device__ Sim(const Params &p_, int lane_, uint32_t rep_) : p(p_), lane(lane_), rep(rep_) {}
+    __device__ Sim(const Params &p_, int lane_, uint32_t rep_) : p(p_), lane(lane_), rep(rep_), warp(0), nwarps(1) {}
+    __device__ __forceinline__ void block_sync() const { if (F & F_MW) __syncthreads(); else __syncwarp(); }
 
     __device__ __forceinline__ double block_start(uint32_t b) const { return __dmul_rn((double)b, p.block_len); }
 
@@ -800,15 +814,15 @@ struct Sim {
     {
         const uint32_t i = job_cls(pk), P = job_P(pk), D = job_D(pk);
         if (lane == (int)i) {
-            ClassState &c = cs[i];
+            WarpClassStats &c = wcs[warp * MAXI + (int)i];
             const double rel = __dsub_rn(te, T_reset);
-            if (job_flag(pk)) { c.sYm_out = __dadd_rn(c.sYm_out, rel); c.Ym--; c.done_mixed++; }
-            else              { c.sYs_out = __dadd_rn(c.sYs_out, rel); c.Ys--; c.done_solo++; }
-            c.tok_in_done += P;       // bundled charging credits the request here, Eq. (21)-(22)
-            c.tok_out_done += D;
+            if (job_flag(pk)) { c.sYm_out = __dadd_rn(c.sYm_out, rel); c.done_mixed++; }
+            else              { c.sYs_out = __dadd_rn(c.sYs_out, rel); c.done_solo++; }
+            c.tok_in += P;       // bundled charging credits the request here, Eq. (21)-(22)
+            c.tok_out += D;
             const double tpot = __ddiv_rn(__dsub_rn(te, tpf), (double)D);
             c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
-            if (f_hist()) hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)]++;
+            if (f_hist()) atomicAdd(&hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)], 1u);
         }
     }
 
@@ -1059,6 +1073,105 @@ struct Sim {
         return false;
     }
 
+    // Class lanes of the master: add every warp's accounting of finished requests to the class records.
+    __device__ void merge_warp_stats()
+    {
+        if (warp == 0 && lane < (int)p.I) {
+            ClassState &c = cs[lane];
+            for (int w = 0; w < nwarps; ++w) {
+                const WarpClassStats &a = wcs[w * MAXI + lane];
+                c.sYm_out = __dadd_rn(c.sYm_out, a.sYm_out);
+                c.sYs_out = __dadd_rn(c.sYs_out, a.sYs_out);
+                c.sum_tpot = __dadd_rn(c.sum_tpot, a.sum_tpot);
+                c.tok_in_done += a.tok_in; c.tok_out_done += a.tok_out;
+                c.done_mixed += a.done_mixed; c.done_solo += a.done_solo;
+                c.Ym -= a.done_mixed; c.Ys -= a.done_solo;
+            }
+        }
+    }
+
+    // This warp's share (rows warp, warp + nwarps, ...) of the candidate scan; run-time row count.
+    __device__ void scan_share(bool buffered, unsigned long long &bt, uint32_t &bs, unsigned long long &tmin)
+    {
+        const unsigned long long INF = 0x7ff0000000000000ull;
+        for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
+            const uint32_t g = (k << 5) + (uint32_t)lane;
+            const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+            if (v < INF) {
+                tmin = min(tmin, v);
+                if (!is_local(g, buffered) && v < bt) { bt = v; bs = SRC_SERVER + g; }
+            }
+        }
+    }
+
+    // This warp's share of the local iteration ends below the limit key, with their retirements.
+    __device__ bool ends_share(unsigned long long lim_t, uint32_t lim_s, bool buffered)
+    {
+        const unsigned long long INF = 0x7ff0000000000000ull;
+        bool progressed = false;
+        for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
+            const uint32_t g = (k << 5) + (uint32_t)lane;
+            const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+            bool retire = false;
+            if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+                retire = local_end(g, __longlong_as_double((long long)v));
+                progressed = true;
+            }
+            uint32_t need = __ballot_sync(FULL, retire);
+            __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
+            while (need) {
+                const int l = __ffs((int)need) - 1;
+                need &= need - 1;
+                const uint32_t gg = (k << 5) + (uint32_t)l;
+                const double te = __longlong_as_double((long long)__shfl_sync(FULL, v, l));
+                retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
+                if (lane == l) start_at(gg, te);
+            }
+        }
+        return progressed;
+    }
+
+    // warp-level argmin of (time bits, source) and min of times
+    __device__ __forceinline__ void warp_keys(unsigned long long bt, uint32_t bs, unsigned long long tmin,
+                                              unsigned long long &tint, uint32_t &src, unsigned long long &tmin_all) const
+    {
+        const uint32_t hi = (uint32_t)(bt >> 32), lo = (uint32_t)bt;
+        const uint32_t mhi = __reduce_min_sync(FULL, hi);
+        const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : NONE32);
+        src = __reduce_min_sync(FULL, (hi == mhi && lo == mlo) ? bs : NONE32);
+        tint = ((unsigned long long)mhi << 32) | mlo;
+        const uint32_t th = (uint32_t)(tmin >> 32);
+        const uint32_t tmh = __reduce_min_sync(FULL, th);
+        const uint32_t tml = __reduce_min_sync(FULL, th == tmh ? (uint32_t)tmin : NONE32);
+        tmin_all = ((unsigned long long)tmh << 32) | tml;
+    }
+
+    // Helper warps (F_MW): serve the master's commands until it says stop.  Every command is bracketed by two
+    // block barriers; the master executes the same two.
+    __device__ void helper_loop()
+    {
+        const unsigned long long INF = 0x7ff0000000000000ull;
+        for (;;) {
+            __syncthreads();
+            const uint32_t op = cmd->op;
+            if (op == MW_EXIT) return;
+            const bool buffered = cmd->buffered != 0;
+            M = cmd->M;
+            if (op == MW_SCAN) {
+                unsigned long long bt = INF, tmin = INF, tint, tall;
+                uint32_t bs = NONE32, src;
+                scan_share(buffered, bt, bs, tmin);
+                warp_keys(bt, bs, tmin, tint, src, tall);
+                if (lane == 0) { MwRes r; r.bt = tint; r.bs = src; r.tmin = tall; r.progressed = 0; res[warp] = r; }
+            } else {
+                const bool pr = ends_share(cmd->lim_t, cmd->lim_s, buffered);
+                const uint32_t any = __ballot_sync(FULL, pr);
+                if (lane == 0) res[warp].progressed = any != 0;
+            }
+            __syncthreads();
+        }
+    }
+
     // --- round loop ----------------------------------------------------------------------------------
     __device__ bool run()
     {
@@ -1094,27 +1207,34 @@ struct Sim {
             constexpr int NC = SPL > 0 ? SPL : 1;       // per-row values kept in registers when the rows unroll
             unsigned long long vrow[NC];
             bool lrow[NC];
+            unsigned long long tint, tmin_all;
+            uint32_t src;
+            if (F & F_MW) {
+                // every warp scans its rows; the partial results meet in shared memory
+                if (lane == 0) { cmd->op = MW_SCAN; cmd->buffered = buffered; cmd->M = M; }
+                __syncthreads();
+                scan_share(buffered, bt, bs, tmin);
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
+                if (lane == 0) { MwRes r; r.bt = tint; r.bs = src; r.tmin = tmin_all; r.progressed = 0; res[0] = r; }
+                __syncthreads();
+                bt = INF; bs = NONE32; tmin = INF;
+                if (lane < nwarps) { bt = res[lane].bt; bs = res[lane].bs; tmin = res[lane].tmin; }
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
+            } else {
 #pragma unroll
-            for (uint32_t k = 0; k < rows; ++k) {
-                const uint32_t g = (k << 5) + (uint32_t)lane;
-                const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-                const bool loc = v < INF && is_local(g, buffered);
-                if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
-                if (v < INF) {
-                    tmin = min(tmin, v);
-                    if (!loc && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                for (uint32_t k = 0; k < rows; ++k) {
+                    const uint32_t g = (k << 5) + (uint32_t)lane;
+                    const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+                    const bool loc = v < INF && is_local(g, buffered);
+                    if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
+                    if (v < INF) {
+                        tmin = min(tmin, v);
+                        if (!loc && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                    }
                 }
+                // warp argmin of (time bits, source id) over non-local events; warp min over all pending times
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
             }
-            // warp argmin of (time bits, source id) over non-local events; warp min over all iteration ends
-            const uint32_t hi = (uint32_t)(bt >> 32), lo = (uint32_t)bt;
-            const uint32_t mhi = __reduce_min_sync(FULL, hi);
-            const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : NONE32);
-            const uint32_t src = __reduce_min_sync(FULL, (hi == mhi && lo == mlo) ? bs : NONE32);
-            const unsigned long long tint = ((unsigned long long)mhi << 32) | mlo;
-            const uint32_t th = (uint32_t)(tmin >> 32);
-            const uint32_t tmh = __reduce_min_sync(FULL, th);
-            const uint32_t tml = __reduce_min_sync(FULL, th == tmh ? (uint32_t)tmin : NONE32);
-            const unsigned long long tmin_all = ((unsigned long long)tmh << 32) | tml;
             if (tint > tend_bits && tmin_all > tend_bits) return true;     // nothing left up to T_end
             if (budget == 0) return false;
             --budget;
@@ -1130,6 +1250,10 @@ struct Sim {
             if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
             uint32_t any_retire = 0;
             bool progressed = false;
+            if (F & F_MW) {
+                if (lane == 0) { cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M; }
+                __syncthreads();
+            }
             if (lane < (int)p.I && n_idle_pf == 0) {
                 // local arrivals of this lane's class, in time order, up to the limit and up to the class's own
                 // next abandonment (which each arrival moves)
@@ -1144,31 +1268,25 @@ struct Sim {
             }
             // pass 1: every lane ends the local iterations of its own GPUs (straight-line over the rows)
             uint32_t retire_rows = 0;
-#pragma unroll
-            for (uint32_t k = 0; k < rows; ++k) {
-                const uint32_t g = (k << 5) + (uint32_t)lane;
-                unsigned long long v;
-                bool loc;
-                if (SPL > 0) { v = vrow[k]; loc = lrow[k]; }
-                else { v = (unsigned long long)__double_as_longlong(tnext[g]); loc = v < INF && is_local(g, buffered); }
-                if (loc && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
-                    if (local_end(g, __longlong_as_double((long long)v))) retire_rows |= 1u << (k & 31u);
-                    progressed = true;
+            if (SPL == 0) {
+                // run-time row count (and, with helpers, only this warp's rows): ends and retirements row by row
+                if (ends_share(lim_t, lim_s, buffered)) progressed = true;
+                if (F & F_MW) {
+                    const uint32_t mine = __ballot_sync(FULL, progressed);
+                    if (lane == 0) res[0].progressed = mine != 0;
+                    __syncthreads();
+                    if (lane < nwarps && res[lane].progressed) progressed = true;
                 }
-                if (SPL == 0) {
-                    // run-time row count: retire per row (the row mask has only 32 bits)
-                    uint32_t need = __ballot_sync(FULL, retire_rows != 0);
-                    any_retire |= need;
-                    __syncwarp();
-                    while (need) {
-                        const int l = __ffs((int)need) - 1;
-                        need &= need - 1;
-                        const uint32_t gg = (k << 5) + (uint32_t)l;
-                        const double te = __longlong_as_double((long long)__shfl_sync(FULL, v, l));
-                        retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
-                        if (lane == l) start_at(gg, te);
+            }
+            if (SPL > 0) {
+#pragma unroll
+                for (uint32_t k = 0; k < rows; ++k) {
+                    const uint32_t g = (k << 5) + (uint32_t)lane;
+                    const unsigned long long v = vrow[k];
+                    if (lrow[k] && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+                        if (local_end(g, __longlong_as_double((long long)v))) retire_rows |= 1u << k;
+                        progressed = true;
                     }
-                    retire_rows = 0;
                 }
             }
             if (SPL > 0) {
@@ -1235,10 +1353,10 @@ struct Sim {
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
     uint32_t off_tnext, off_tarr, off_tau, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
-        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, total;
+        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, off_wcs, off_cmd, off_res, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem)
+__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps = 1)
 {
     SmemLayout L;
     uint32_t o = 0;
@@ -1270,6 +1388,11 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * STAGE_CAP;
     L.off_stte = o; o += 8 * STAGE_CAP;
     L.off_pqh = o; o += (uint32_t)sizeof(QEntry) * MAXI;
+    L.off_wcs = o; o += (uint32_t)sizeof(WarpClassStats) * MAXI * nwarps;
+    o = (o + 15u) & ~15u;
+    L.off_cmd = o; o += (uint32_t)sizeof(MwCmd);
+    o = (o + 15u) & ~15u;
+    L.off_res = o; o += (uint32_t)sizeof(MwRes) * MW_MAX;
     L.total = (o + 15u) & ~15u;
     return L;
 }
@@ -1300,6 +1423,9 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.st_rec = reinterpret_cast<SlotRec *>(sm + L.off_strec);
     s.st_te = reinterpret_cast<double *>(sm + L.off_stte);
     s.pqh = reinterpret_cast<QEntry *>(sm + L.off_pqh);
+    s.wcs = reinterpret_cast<WarpClassStats *>(sm + L.off_wcs);
+    s.cmd = reinterpret_cast<MwCmd *>(sm + L.off_cmd);
+    s.res = reinterpret_cast<MwRes *>(sm + L.off_res);
     s.n_pend = 0;
     s.ring_n = 0; s.ring_pos = 0; s.sched_pending = false; s.t0_pending = 0.0;
     const Params &p = s.p;
@@ -1370,27 +1496,32 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
 
 // Advance replications to their new end time (or until the per-launch event budget runs out).
 template <int SPLT, uint32_t FT>
-__global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
+__global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kernel(Params p)
 {
     extern __shared__ __align__(16) char sm[];
-    const int lane = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t nthr = blockDim.x;
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5);
         Sim<SPLT, FT> s(p, lane, rep);
+        s.warp = warp;
+        s.nwarps = (int)(nthr >> 5);
         bind_pointers(s, sm, L);
-        __syncwarp();
-        // stage state: server arrays (coalesced 16-byte copies) and the class records
+        s.block_sync();
+        // stage state: per-GPU arrays (coalesced 16-byte copies) and the class records; clear the per-warp accounting
         const char *img = p.srv + (size_t)rep * p.srv_bytes;
-        for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
+        for (uint32_t o = tid * 16; o < L.srv_bytes; o += nthr * 16)
             *reinterpret_cast<uint4 *>(sm + o) = *reinterpret_cast<const uint4 *>(img + o);
         {
             const uint4 *src = reinterpret_cast<const uint4 *>(h.cs);
             uint4 *dst = reinterpret_cast<uint4 *>(s.cs);
-            for (uint32_t o = lane; o < sizeof(ClassState) * MAXI / 16; o += 32) dst[o] = src[o];
+            for (uint32_t o = tid; o < sizeof(ClassState) * MAXI / 16; o += nthr) dst[o] = src[o];
+            uint32_t *w = reinterpret_cast<uint32_t *>(s.wcs);
+            for (uint32_t o = tid; o < sizeof(WarpClassStats) * MAXI * (nthr >> 5) / 4; o += nthr) w[o] = 0;
         }
-        __syncwarp();
+        s.block_sync();
         // the end time is one rounded product of the cumulative horizon: run(a); run(b) ends where run(a+b) ends
         double T_end = h.T_end;
         const unsigned long long H_total = h.H_total + (p.advance ? p.horizon_iters : 0ull);
@@ -1404,35 +1535,60 @@ __global__ void __launch_bounds__(32) qsim_run_kernel(Params p)
         s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
         s.n_touch = 0; s.touch_all = false; s.need_start = 0; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
-        s.n_idle_pf = s.count_idle_pf();
+        s.n_idle_pf = 0;
         s.idle_hint = NONE32;
-        if (lane < (int)p.I && s.cs[lane].pq_n > 0) s.pqh[lane] = s.pq[(size_t)lane * p.qcap + s.cs[lane].pq_head];
-        __syncwarp();
-        s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
-        s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
-        const bool finished = s.err ? true : s.run();
-        s.flush_done();
-        if (lane < (int)p.I) s.cs[lane].adraw -= s.ring_n;     // unused arrival draws are produced again next time
-        __syncwarp();
+        s.it_mixed = 0; s.it_solo = 0; s.busy_mixed = 0.0; s.busy_solo = 0.0;
+        bool finished = true;
+        if (warp == 0) {
+            s.n_idle_pf = s.count_idle_pf();
+            if (lane < (int)p.I && s.cs[lane].pq_n > 0) s.pqh[lane] = s.pq[(size_t)lane * p.qcap + s.cs[lane].pq_head];
+            __syncwarp();
+            s.it_mixed = h.iters_mixed[lane]; s.it_solo = h.iters_solo[lane];
+            s.busy_mixed = h.busy_mixed[lane]; s.busy_solo = h.busy_solo[lane];
+            finished = s.err ? true : s.run();
+            s.flush_done();
+            if (FT & F_MW) {
+                if (lane == 0) s.cmd->op = MW_EXIT;
+                __syncthreads();
+            }
+        } else {
+            s.helper_loop();
+        }
+        s.block_sync();
+        s.merge_warp_stats();
+        if (warp == 0 && lane < (int)p.I) s.cs[lane].adraw -= s.ring_n;     // unused arrival draws are produced again next time
+        s.block_sync();
         // stage back
         char *out = p.srv + (size_t)rep * p.srv_bytes;
-        for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
+        for (uint32_t o = tid * 16; o < L.srv_bytes; o += nthr * 16)
             *reinterpret_cast<uint4 *>(out + o) = *reinterpret_cast<const uint4 *>(sm + o);
         {
             uint4 *dst = reinterpret_cast<uint4 *>(h.cs);
             const uint4 *src = reinterpret_cast<const uint4 *>(s.cs);
-            for (uint32_t o = lane; o < sizeof(ClassState) * MAXI / 16; o += 32) dst[o] = src[o];
+            for (uint32_t o = tid; o < sizeof(ClassState) * MAXI / 16; o += nthr) dst[o] = src[o];
         }
-        h.iters_mixed[lane] = s.it_mixed; h.iters_solo[lane] = s.it_solo;
-        h.busy_mixed[lane] = s.busy_mixed; h.busy_solo[lane] = s.busy_solo;
-        if (lane == 0) {
+        // per-thread partial sums go to the 32 lane slots, warp after warp (a fixed order)
+        for (int w = 0; w < s.nwarps; ++w) {
+            if (warp == w) {
+                if (w == 0) {
+                    h.iters_mixed[lane] = s.it_mixed; h.iters_solo[lane] = s.it_solo;
+                    h.busy_mixed[lane] = s.busy_mixed; h.busy_solo[lane] = s.busy_solo;
+                } else {
+                    h.iters_mixed[lane] += s.it_mixed; h.iters_solo[lane] += s.it_solo;
+                    h.busy_mixed[lane] = __dadd_rn(h.busy_mixed[lane], s.busy_mixed);
+                    h.busy_solo[lane] = __dadd_rn(h.busy_solo[lane], s.busy_solo);
+                }
+            }
+            if (FT & F_MW) { __threadfence_block(); __syncthreads(); }
+        }
+        if (tid == 0) {
             h.T_end = T_end; h.H_total = H_total; h.blk = s.blk;
             h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
             h.place_ord = s.place_ord; h.events = s.events; h.rounds = s.rounds; h.err = s.err;
             h.done = finished ? 1u : 0u;
             if (!finished) atomicAdd(p.not_done, 1u);
         }
-        __syncwarp();
+        s.block_sync();
     }
 }
 

@@ -56,6 +56,7 @@ struct qsim {
     uint64_t launches = 0;
     int device = 0;
     void (*run_fn)(qsimdev::Params) = nullptr;
+    uint32_t nwarps = 1;          // warps per replication (block size / 32)
 };
 
 namespace {
@@ -145,6 +146,7 @@ const std::vector<RunVariant> &run_variants()
         add_variants<2>(v);
         add_variants<4>(v);
         v.push_back({0, F_GENERIC, qsim_run_kernel<0, F_GENERIC>});
+        v.push_back({-1, F_GENERIC | F_MW, qsim_run_kernel<0, F_GENERIC | F_MW>});     // several warps per replication
         return v;
     }();
     return table;
@@ -166,6 +168,24 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
     return f;
 }
 
+// Large clusters: per-replication shared memory allows only a few blocks per SM, so each replication gets
+// several warps (master + helpers) that share the per-GPU scans.  QSIM_WARPS overrides the choice (1 = off).
+void choose_multiwarp(uint32_t N, Params &p, RunKernel &fn, uint32_t &nwarps)
+{
+    const uint32_t rows = (N + 31u) / 32u;
+    uint32_t W = rows >= 64 ? 16u : (rows >= 8 ? 4u : 1u);
+    if (const char *e = std::getenv("QSIM_WARPS")) {
+        const int v = std::atoi(e);
+        if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
+    }
+    if (W <= 1 || rows < 2) return;
+    for (const RunVariant &v : run_variants())
+        if (v.spl < 0) { fn = v.fn; break; }
+    nwarps = W;
+    p.Npad = rows * 32u;
+    p.slots_smem = 0;       // helpers retire through the global slot lists
+}
+
 RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
 {
     const int rows = (int)((N + 31u) / 32u);
@@ -175,6 +195,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
     if (force && std::strcmp(force, "generic") == 0) feat = ~0u;
     int best_bits = 99;
     for (const RunVariant &v : run_variants()) {
+        if (v.spl < 0) continue;                            // the multi-warp instance is chosen by the caller
         if (v.spl != 0 && v.spl < rows) continue;          // too few GPUs per lane
         if (v.spl == 0 && !generic) generic = &v;
         if (v.spl == 0) continue;
@@ -198,7 +219,7 @@ int launch_run(qsim *h, bool advance, uint64_t horizon)
     p.advance = advance ? 1u : 0u;
     p.horizon_iters = horizon;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    h->run_fn<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
+    h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
@@ -250,8 +271,10 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
         p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
         if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
         h->run_fn = v.fn;
+        h->nwarps = 1;
+        choose_multiwarp(cfg->N, p, h->run_fn, h->nwarps);
     }
-    h->lay = smem_layout(p.Npad, p.B, p.slots_smem);
+    h->lay = smem_layout(p.Npad, p.B, p.slots_smem, h->nwarps);
     p.srv_bytes = h->lay.srv_bytes;
     if (h->lay.total > 227u * 1024u) {
         delete h;
@@ -605,8 +628,10 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
         p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
         if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
         h.run_fn = v.fn;
+        h.nwarps = 1;
+        choose_multiwarp(cfg->N, p, h.run_fn, h.nwarps);
     }
-    h.lay = smem_layout(p.Npad, p.B, p.slots_smem);
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps);
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     qsim_config nohist = *cfg;
@@ -658,7 +683,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
         q.advance = advance ? 1u : 0u;
         q.horizon_iters = advance ? horizon_iters : 0;
         CUDA_TRY(cudaMemsetAsync(q.not_done, 0, 4, stream));
-        h.run_fn<<<cfg->R, 32, h.lay.total, stream>>>(q);
+        h.run_fn<<<cfg->R, 32 * h.nwarps, h.lay.total, stream>>>(q);
         CUDA_TRY(cudaGetLastError());
         uint32_t left = 0;
         CUDA_TRY(cudaMemcpyAsync(&left, q.not_done, 4, cudaMemcpyDeviceToHost, stream));
