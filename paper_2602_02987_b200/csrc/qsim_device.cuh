@@ -1356,7 +1356,8 @@ struct SmemLayout {
         off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, off_wcs, off_cmd, off_res, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps = 1)
+__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps = 1,
+                                                  bool kappa = true)
 {
     SmemLayout L;
     uint32_t o = 0;
@@ -1367,8 +1368,8 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_nfin = o; o += 4 * Npad;
     L.off_pfrem = o; o += 4 * Npad;
     L.off_pfjob = o; o += 4 * Npad;
-    L.off_K = o; o += 4 * Npad;
-    L.off_Kpend = o; o += 4 * Npad;
+    L.off_K = o; if (kappa) o += 4 * Npad;        // KV-token counts exist only when the KV slope is on
+    L.off_Kpend = o; if (kappa) o += 4 * Npad;
     L.off_ndec = o; o += 2 * Npad;
     L.off_nact = o; o += 2 * Npad;
     L.off_pfcur = o; o += 2 * Npad;
@@ -1445,7 +1446,7 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
     extern __shared__ __align__(16) char sm[];
     const int lane = threadIdx.x;
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, 1, p.coef[5] != 0.0);
         Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();
@@ -1504,7 +1505,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kerne
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0);
         Sim<SPLT, FT> s(p, lane, rep);
         s.warp = warp;
         s.nwarps = (int)(nthr >> 5);

@@ -173,7 +173,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
 void choose_multiwarp(uint32_t N, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
-    uint32_t W = rows >= 64 ? 16u : (rows >= 8 ? 4u : 1u);
+    uint32_t W = rows >= 64 ? 16u : (rows >= 16 ? 4u : 1u);
     if (const char *e = std::getenv("QSIM_WARPS")) {
         const int v = std::atoi(e);
         if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
@@ -268,13 +268,13 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
         RunVariant v = pick_run_kernel(cfg->N, feat);
         if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
         // finish stamps + occupancy bits go to shared memory when the whole block state stays small
-        p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
+        p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, p.coef[5] != 0.0).total <= 40u * 1024u ? 1u : 0u;
         if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
         h->run_fn = v.fn;
         h->nwarps = 1;
         choose_multiwarp(cfg->N, p, h->run_fn, h->nwarps);
     }
-    h->lay = smem_layout(p.Npad, p.B, p.slots_smem, h->nwarps);
+    h->lay = smem_layout(p.Npad, p.B, p.slots_smem, h->nwarps, p.coef[5] != 0.0);
     p.srv_bytes = h->lay.srv_bytes;
     if (h->lay.total > 227u * 1024u) {
         delete h;
@@ -625,13 +625,13 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
         uint32_t feat = features_of(nohist_features(*cfg), classes, coef);
         RunVariant v = pick_run_kernel(cfg->N, feat);
         if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
-        p.slots_smem = smem_layout(p.Npad, p.B, 1).total <= 40u * 1024u ? 1u : 0u;
+        p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, p.coef[5] != 0.0).total <= 40u * 1024u ? 1u : 0u;
         if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
         h.run_fn = v.fn;
         h.nwarps = 1;
         choose_multiwarp(cfg->N, p, h.run_fn, h.nwarps);
     }
-    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps);
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, p.coef[5] != 0.0);
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     qsim_config nohist = *cfg;
