@@ -143,6 +143,27 @@ int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
  */
 int qsim_run(qsim_t *h, uint64_t horizon_iters);
 
+/*
+ * Advance every replication to the absolute simulated time T seconds (T not before the end of the previous
+ * call); otherwise like qsim_run.  Meant for controllers that act at fixed epochs (online replanning every
+ * 10 s, Section 6.2).  Do not mix with qsim_run on one handle: the two keep separate notions of the end time.
+ */
+int qsim_run_until(qsim_t *h, double T);
+
+/*
+ * Trace replay (Section 6.2): replace the Poisson source by a list of arrivals, the same for every
+ * replication.  [host] t[n] ascending times in seconds, job[n][3] = {class, P, D}.  Call between qsim_create
+ * and qsim_bind; needs nblk == 1.  The rates of qsim_create are then ignored.
+ */
+int qsim_set_injected(qsim_t *h, const double *t, const uint32_t *job, uint64_t n);
+
+/*
+ * Replace the policy parameters (M, x*, n x*, n q*_p, p_s) from now on, e.g. after re-solving the LP with
+ * re-estimated rates (Eq. (45)-(46)).  Running service is not pre-empted; the new split governs later
+ * placement and admission, exactly like a block switch.  Needs nblk == 1; takes effect at the next run call.
+ */
+int qsim_set_targets(qsim_t *h, const qsim_targets *lp_targets);
+
 /* Upper bound on the rounds (one non-local event plus the iteration ends before it) one replication
  * processes per kernel launch (default 2^28); a replication that reaches it is continued by further
  * launches with identical results. */

@@ -674,6 +674,26 @@ int orc_run(orc_sim *s, uint64_t horizon_iters, uint32_t rep_lo, uint32_t rep_hi
     return 0;
 }
 
+/* Advance to the absolute time T (controllers that act at fixed epochs). */
+int orc_run_until(orc_sim *s, double T, uint32_t rep_lo, uint32_t rep_hi)
+{
+    if (!s || rep_lo > rep_hi || rep_hi > s->cfg.R) return -1;
+    for (uint32_t r = rep_lo; r < rep_hi; ++r) {
+        if (T < s->reps[r].T_end) return -1;
+        run_rep(s, r, T);
+    }
+    return 0;
+}
+
+/* New policy parameters from now on (online replanning, Section 6.2): nothing running is pre-empted, the new
+ * split governs later placement and admission.  Single-block configurations only. */
+int orc_set_targets(orc_sim *s, const orc_targets *tg)
+{
+    if (!s || !tg || s->cfg.nblk != 1 || tg->M > s->cfg.N) return -1;
+    s->tg[0] = *tg;
+    return 0;
+}
+
 int orc_reset_stats(orc_sim *s)
 {
     if (!s) return -1;

@@ -96,6 +96,8 @@ uint64_t orc_trace_count(const orc_sim *s);
 /* Advance replications [rep_lo, rep_hi) by horizon_iters more iterations of horizon: the new end time is
  * (total horizon so far) * tau_ref, tau_ref = one full solo iteration. */
 int orc_run(orc_sim *s, uint64_t horizon_iters, uint32_t rep_lo, uint32_t rep_hi);
+int orc_run_until(orc_sim *s, double T, uint32_t rep_lo, uint32_t rep_hi);
+int orc_set_targets(orc_sim *s, const orc_targets *tg);
 int orc_reset_stats(orc_sim *s);
 /* per_rep: [R]; hist_ttft / hist_tpot: NULL or uint64 [R][I][ORC_NBIN] */
 int orc_stats(const orc_sim *s, orc_rep_stats *per_rep, uint64_t *hist_ttft, uint64_t *hist_tpot);

@@ -87,6 +87,10 @@ def lib():
         L.orc_run.restype = C.c_int
         L.orc_run.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32]
         L.orc_reset_stats.argtypes = [C.c_void_p]
+        L.orc_run_until.restype = C.c_int
+        L.orc_run_until.argtypes = [C.c_void_p, C.c_double, C.c_uint32, C.c_uint32]
+        L.orc_set_targets.restype = C.c_int
+        L.orc_set_targets.argtypes = [C.c_void_p, C.POINTER(Targets)]
         L.orc_stats.restype = C.c_int
         L.orc_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_server_state.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -155,6 +159,20 @@ class OracleSim:
         rc = lib().orc_run(self.h, int(horizon_iters), rep_lo, self.inp.R if rep_hi is None else rep_hi)
         if rc != 0:
             raise RuntimeError(f"orc_run failed: {rc}")
+
+    def run_until(self, T: float) -> None:
+        rc = lib().orc_run_until(self.h, float(T), 0, self.inp.R)
+        if rc != 0:
+            raise RuntimeError(f"orc_run_until failed: {rc}")
+
+    def set_targets(self, M, xstar, n_xstar, n_qpstar, p_solo) -> None:
+        tg = Targets()
+        tg.M = int(M)
+        for i in range(self.inp.I):
+            tg.xstar[i] = float(xstar[i]); tg.n_xstar[i] = float(n_xstar[i])
+            tg.n_qpstar[i] = float(n_qpstar[i]); tg.p_solo[i] = float(p_solo[i])
+        if lib().orc_set_targets(self.h, C.byref(tg)) != 0:
+            raise RuntimeError("orc_set_targets failed")
 
     def reset_stats(self) -> None:
         lib().orc_reset_stats(self.h)

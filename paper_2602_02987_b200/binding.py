@@ -16,7 +16,8 @@ _COUNTERS = ("arrivals", "admitted", "prefill_done", "placed_mixed", "placed_sol
 _STATE = ("Qp", "X", "Qd", "Ym", "Ys")
 _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_tpot")
 
-EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_set_event_budget", "qsim_sync",
+EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_run_until", "qsim_set_injected",
+           "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
            "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_destroy", "qsim_last_error")
 
@@ -69,6 +70,9 @@ def load_library():
         L.qsim_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.qsim_bind.argtypes = [vp, vp, C.c_size_t, vp]
         L.qsim_run.argtypes = [vp, C.c_uint64]
+        L.qsim_run_until.argtypes = [vp, C.c_double]
+        L.qsim_set_injected.argtypes = [vp, vp, vp, C.c_uint64]
+        L.qsim_set_targets.argtypes = [vp, C.POINTER(qsim_targets)]
         L.qsim_set_event_budget.argtypes = [vp, C.c_uint64]
         L.qsim_sync.argtypes = [vp]
         L.qsim_stats.argtypes = [vp, vp, vp, vp, vp]
@@ -102,8 +106,6 @@ def _ptr(a):
 def marshal(inp):
     """SimInputs -> the C structs and arrays of qsim_create (kept alive by the returned tuple)."""
     I, nblk = inp.I, inp.nblk
-    if getattr(inp, "inject_t", None) is not None:
-        raise QSimError("injected arrivals are not supported by the CUDA library")
     cfg = qsim_config(size=C.sizeof(qsim_config), I=I, N=inp.N, R=inp.R, B=inp.B, C=inp.C, nblk=nblk,
                       gate=inp.gate, router=inp.router, placement=inp.placement, pricing=inp.pricing,
                       length_mode=inp.length_mode, qcap=inp.qcap, hist=inp.hist, seed=inp.seed,
@@ -158,6 +160,10 @@ class QSim:
         with torch.cuda.device(self.device):
             _check(self.L.qsim_create(C.byref(self.h), C.byref(cfg), classes, _ptr(rates), _ptr(lengths),
                                       _ptr(prices), _ptr(coeffs), tg))
+            if getattr(inp, "inject_t", None) is not None:
+                it = np.ascontiguousarray(inp.inject_t, np.float64)
+                ij = np.ascontiguousarray(inp.inject_job, np.uint32)
+                _check(self.L.qsim_set_injected(self.h, _ptr(it), _ptr(ij), it.shape[0]))
             nbytes = C.c_size_t()
             _check(self.L.qsim_workspace_bytes(self.h, C.byref(nbytes)))
             self.workspace_bytes = int(nbytes.value)
@@ -171,6 +177,17 @@ class QSim:
 
     def run(self, horizon_iters: int) -> None:
         _check(self.L.qsim_run(self.h, int(horizon_iters)))
+
+    def run_until(self, T: float) -> None:
+        _check(self.L.qsim_run_until(self.h, float(T)))
+
+    def set_targets(self, M, xstar, n_xstar, n_qpstar, p_solo) -> None:
+        tg = qsim_targets()
+        tg.M = int(M)
+        for i in range(self.inp.I):
+            tg.xstar[i] = float(xstar[i]); tg.n_xstar[i] = float(n_xstar[i])
+            tg.n_qpstar[i] = float(n_qpstar[i]); tg.p_solo[i] = float(p_solo[i])
+        _check(self.L.qsim_set_targets(self.h, C.byref(tg)))
 
     def sync(self) -> None:
         _check(self.L.qsim_sync(self.h))

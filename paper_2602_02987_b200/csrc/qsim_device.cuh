@@ -108,6 +108,10 @@ struct Params {
     ClassPar cls[MAXI];
     const BlockPar *blocks;      // [nblk]
     const uint32_t *lengths;     // [I][2][LMAX] or null
+    const double *inject_t;      // injected arrivals (trace replay): times [n_inject], ascending
+    const uint32_t *inject_job;  // [n_inject][3] = class, P, D
+    uint32_t n_inject, pad_inject;
+    double T_abs;                // advance == 2: absolute end time of this run
     // workspace sections (all arrays are [R][...])
     RepHeader *hdr;
     char *srv;                   // per replication: server structure-of-arrays image, srv_bytes each
@@ -377,6 +381,18 @@ struct Sim {
     __device__ void schedule_from(double t0)
     {
         ClassState &c = cs[lane];
+        if ((F & F_GENERIC) && p.n_inject > 0) {
+            // trace replay: the next entry of this class in the injected list (c.ablk is the read position)
+            uint32_t k = c.ablk;
+            while (k < p.n_inject && p.inject_job[3 * k] != (uint32_t)lane) ++k;
+            if (k < p.n_inject) {
+                c.ta = p.inject_t[k]; c.nextP = p.inject_job[3 * k + 1]; c.nextD = p.inject_job[3 * k + 2];
+                c.ablk = k + 1;
+            } else {
+                c.ta = dinf(); c.ablk = k;
+            }
+            return;
+        }
         uint32_t b = c.ablk;
         for (;;) {
             const double Lam = __dmul_rn((double)p.N, p.blocks[b].rate[lane]);
@@ -1471,8 +1487,9 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
         }
         __syncwarp();
         // first arrival of every class: ask for draws, let the warp fill the rings, give the unused draws back
-        s.sched_pending = lane < (int)p.I;
+        s.sched_pending = lane < (int)p.I && p.n_inject == 0;
         s.t0_pending = 0.0;
+        if (p.n_inject > 0 && lane < (int)p.I) s.schedule_from(0.0);
         for (int guard = 0; guard < 64; ++guard) {
             uint32_t need = __ballot_sync(FULL, s.sched_pending);
             if (!need) break;
@@ -1525,8 +1542,9 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kerne
         s.block_sync();
         // the end time is one rounded product of the cumulative horizon: run(a); run(b) ends where run(a+b) ends
         double T_end = h.T_end;
-        const unsigned long long H_total = h.H_total + (p.advance ? p.horizon_iters : 0ull);
-        if (p.advance) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
+        const unsigned long long H_total = h.H_total + (p.advance == 1 ? p.horizon_iters : 0ull);
+        if (p.advance == 1) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
+        if (p.advance == 2) T_end = p.T_abs;
         s.T_end = T_end;
         s.T_reset = h.T_reset;
         s.tau_min = fmin(p.coef[0], p.coef[3]);

@@ -49,6 +49,10 @@ struct qsim {
     Sections sec{};
     BlockPar *d_blocks = nullptr;
     uint32_t *d_lengths = nullptr;
+    double *d_inject_t = nullptr;
+    uint32_t *d_inject_job = nullptr;
+    uint32_t feat = 0;
+    double T_end_abs = 0.0;       // end time reached by qsim_run_until calls
     uint32_t *h_flag = nullptr;   // pinned
     void *ws = nullptr;
     cudaStream_t stream = nullptr;
@@ -213,11 +217,12 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
     return best ? *best : *generic;
 }
 
-int launch_run(qsim *h, bool advance, uint64_t horizon)
+int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
 {
     Params p = h->par;
-    p.advance = advance ? 1u : 0u;
+    p.advance = advance;
     p.horizon_iters = horizon;
+    p.T_abs = T_abs;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
     h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
@@ -356,15 +361,80 @@ int qsim_run(qsim_t *h, uint64_t horizon_iters)
 {
     if (!h) return fail(QSIM_EINVAL, "null handle");
     if (!h->bound) return fail(QSIM_ESTATE, "qsim_run before qsim_bind");
-    int rc = launch_run(h, true, horizon_iters);
+    int rc = launch_run(h, 1u, horizon_iters);
     if (rc != QSIM_OK) return rc;
     // a replication that used up its per-launch event budget is continued by further launches
     for (;;) {
         CUDA_TRY(cudaStreamSynchronize(h->stream));
         if (*h->h_flag == 0) break;
-        rc = launch_run(h, false, 0);
+        rc = launch_run(h, 0u, 0);
         if (rc != QSIM_OK) return rc;
     }
+    return QSIM_OK;
+}
+
+int qsim_run_until(qsim_t *h, double T)
+{
+    if (!h) return fail(QSIM_EINVAL, "null handle");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_run_until before qsim_bind");
+    if (!(T >= h->T_end_abs) || !std::isfinite(T)) return fail(QSIM_EINVAL, "end time must be finite and not before the previous one");
+    h->T_end_abs = T;
+    int rc = launch_run(h, 2u, 0, T);
+    if (rc != QSIM_OK) return rc;
+    for (;;) {
+        CUDA_TRY(cudaStreamSynchronize(h->stream));
+        if (*h->h_flag == 0) break;
+        rc = launch_run(h, 0u, 0);
+        if (rc != QSIM_OK) return rc;
+    }
+    return QSIM_OK;
+}
+
+int qsim_set_injected(qsim_t *h, const double *t, const uint32_t *job, uint64_t n)
+{
+    if (!h || !t || !job || n == 0 || n > 0x7fffffffull) return fail(QSIM_EINVAL, "bad injected arrival list");
+    if (h->bound) return fail(QSIM_ESTATE, "qsim_set_injected must come before qsim_bind");
+    if (h->cfg.nblk != 1) return fail(QSIM_EINVAL, "injected arrivals need nblk == 1");
+    for (uint64_t k = 0; k < n; ++k) {
+        if (!(t[k] >= 0.0) || !std::isfinite(t[k]) || (k > 0 && t[k] < t[k - 1])) return fail(QSIM_EINVAL, "injected times must be ascending and >= 0");
+        if (job[3 * k] >= h->cfg.I || job[3 * k + 1] < 1 || job[3 * k + 1] > QSIM_LMAX || job[3 * k + 2] < 1 || job[3 * k + 2] > QSIM_LMAX)
+            return fail(QSIM_EINVAL, "injected job out of range");
+    }
+    if (h->d_inject_t) { cudaFree(h->d_inject_t); cudaFree(h->d_inject_job); h->d_inject_t = nullptr; h->d_inject_job = nullptr; }
+    CUDA_TRY(cudaMalloc(&h->d_inject_t, n * sizeof(double)));
+    CUDA_TRY(cudaMalloc(&h->d_inject_job, n * 3 * sizeof(uint32_t)));
+    CUDA_TRY(cudaMemcpy(h->d_inject_t, t, n * sizeof(double), cudaMemcpyHostToDevice));
+    CUDA_TRY(cudaMemcpy(h->d_inject_job, job, n * 3 * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    h->par.inject_t = h->d_inject_t;
+    h->par.inject_job = h->d_inject_job;
+    h->par.n_inject = (uint32_t)n;
+    // the trace source lives in the run-time-configured instance
+    RunVariant v = pick_run_kernel(h->cfg.N, ~0u);
+    if (h->nwarps == 1) {
+        h->run_fn = v.fn;
+        if (h->lay.total > 48u * 1024u)
+            CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void *>(h->run_fn), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total));
+    }
+    return QSIM_OK;
+}
+
+int qsim_set_targets(qsim_t *h, const qsim_targets *tg)
+{
+    if (!h || !tg) return fail(QSIM_EINVAL, "null argument");
+    if (h->cfg.nblk != 1) return fail(QSIM_EINVAL, "qsim_set_targets needs nblk == 1");
+    if (tg->M > h->cfg.N) return fail(QSIM_EINVAL, "M must be <= N");
+    BlockPar bp;
+    CUDA_TRY(cudaMemcpyAsync(&bp, h->d_blocks, sizeof bp, cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    bp.M = tg->M;
+    for (uint32_t i = 0; i < h->cfg.I; ++i) {
+        if (!std::isfinite(tg->xstar[i]) || tg->xstar[i] < 0.0 || !std::isfinite(tg->n_xstar[i]) || !std::isfinite(tg->n_qpstar[i]) ||
+            !(tg->p_solo[i] >= 0.0 && tg->p_solo[i] <= 1.0))
+            return fail(QSIM_EINVAL, "LP targets out of range");
+        bp.xstar[i] = tg->xstar[i]; bp.nx[i] = tg->n_xstar[i]; bp.nq[i] = tg->n_qpstar[i]; bp.ps[i] = tg->p_solo[i];
+    }
+    CUDA_TRY(cudaMemcpyAsync(h->d_blocks, &bp, sizeof bp, cudaMemcpyHostToDevice, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
     return QSIM_OK;
 }
 
@@ -537,6 +607,8 @@ int qsim_destroy(qsim_t *h)
     if (h->bound) cudaStreamSynchronize(h->stream);
     if (h->d_blocks) cudaFree(h->d_blocks);
     if (h->d_lengths) cudaFree(h->d_lengths);
+    if (h->d_inject_t) cudaFree(h->d_inject_t);
+    if (h->d_inject_job) cudaFree(h->d_inject_job);
     if (h->h_flag) cudaFreeHost(h->h_flag);
     delete h;
     return QSIM_OK;

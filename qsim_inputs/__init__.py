@@ -5,4 +5,4 @@ workload recipes.  Neither simulator's event arithmetic lives here.
 """
 from .spec import *  # noqa: F401,F403
 from .spec import SimInputs  # noqa: F401
-from . import fluid_lp, lengths, presets  # noqa: F401
+from . import fluid_lp, lengths, online, presets  # noqa: F401

@@ -266,3 +266,34 @@ def single_class(N=1, B=3, C=256, P=512, D=2, lam=1.0, R=1, seed=7, coeffs=COEFF
         job = np.array([[e[1], e[2], e[3]] for e in inject], np.uint32).reshape(-1, 3)
         inp = inp.with_(inject_t=t, inject_job=job)
     return inp
+
+
+def trace_replay(n=10, R=2, T=90.0, seed=42, placement=PLACE_RANDOM, coeffs=COEFFS_PAPER_KV):
+    """Matched synthetic stand-in for the paper's trace replay (Section 6.2; the Azure traces are not
+    redistributable): two classes ("code": long prompts, short outputs; "conversation": the reverse) with
+    lognormal request-level lengths and Poisson timestamps generated here on the host, 10 GPUs, B = 16, C = 256,
+    the KV-slope iteration law of the trace simulator.  Returns (inputs, class mean lengths)."""
+    rng = np.random.default_rng(seed)
+    spec = [(2.4 * n, 7.3, 0.8, 3.3, 0.9), (1.8 * n, 6.6, 0.9, 5.3, 0.7)]   # rate/s, mu_P, s_P, mu_D, s_D (congested)
+    ts, jobs = [], []
+    for cls, (rate, mp, sp, md, sd) in enumerate(spec):
+        t = 0.0
+        while True:
+            t += rng.exponential(1.0 / rate)
+            if t >= T:
+                break
+            P = int(np.clip(np.rint(np.exp(mp + sp * rng.standard_normal())), 1, 8192))
+            D = int(np.clip(np.rint(np.exp(md + sd * rng.standard_normal())), 1, 8192))
+            ts.append(t); jobs.append((cls, P, D))
+    order = np.argsort(ts, kind="stable")
+    ts = np.array(ts)[order]
+    jobs = np.array(jobs, np.uint32)[order]
+    Pm = [float(jobs[jobs[:, 0] == c, 1].mean()) for c in range(2)]
+    Dm = [float(jobs[jobs[:, 0] == c, 2].mean()) for c in range(2)]
+    lam0 = [1e-6, 1e-6]       # cold start: the controller knows nothing yet (lambda_min)
+    inp = build(f"trace_n{n}", N=n, R=R, B=16, C=256, Pm=Pm, Dm=Dm, lam_blocks=lam0, theta=[0.0, 0.0],
+                prices=[0.1, 0.2], coeffs=coeffs, gate=GATE_OCCUPANCY, router=ROUTER_SOLO_FIRST, placement=placement,
+                pricing=PRICING_BUNDLED, P_fixed=[int(round(v)) for v in Pm], D_fixed=[int(round(v)) for v in Dm],
+                seed=seed, qcap=4096)
+    inp = inp.with_(inject_t=np.ascontiguousarray(ts, np.float64), inject_job=np.ascontiguousarray(jobs, np.uint32))
+    return inp, Pm, Dm
