@@ -50,7 +50,7 @@ constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST 
 // other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
 // round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
 enum { MW_SCAN = 1, MW_ENDS = 2, MW_EXIT = 3 };
-struct MwCmd { unsigned long long lim_t; uint32_t op, lim_s, buffered, M; };
+struct MwCmd { unsigned long long lim_t; uint32_t op, lim_s, buffered, M, force, pad; };
 struct MwRes { unsigned long long bt, tmin; uint32_t bs, progressed; };
 constexpr int MW_MAX = 16;
 
@@ -80,7 +80,7 @@ struct ClassState {
 struct RepHeader {
     double T_end, T_reset;
     unsigned long long place_ord, events, H_total, rounds;
-    uint32_t blk, done, err, pad;
+    uint32_t blk, done, err, force;    // force: the next event must be followed by a dispatch (targets were replaced)
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
     unsigned long long iters_mixed[32], iters_solo[32];
     double busy_mixed[32], busy_solo[32];
@@ -110,7 +110,7 @@ struct Params {
     const uint32_t *lengths;     // [I][2][LMAX] or null
     const double *inject_t;      // injected arrivals (trace replay): times [n_inject], ascending
     const uint32_t *inject_job;  // [n_inject][3] = class, P, D
-    uint32_t n_inject, pad_inject;
+    uint32_t n_inject, force_dispatch;   // force_dispatch: the policy parameters changed since the last launch
     double T_abs;                // advance == 2: absolute end time of this run
     // workspace sections (all arrays are [R][...])
     RepHeader *hdr;
@@ -327,6 +327,7 @@ struct Sim {
     uint32_t need_start;         // per lane: rows of own GPUs touched by the current event
     unsigned long long place_ord, events, rounds;
     bool drain_dirty, gate_dirty, touch_all;
+    bool force_nonlocal;         // treat the next event, whatever it is, as non-local (it must end with a dispatch)
     // per-lane partial sums
     unsigned long long it_mixed, it_solo;
     double busy_mixed, busy_solo;
@@ -1173,6 +1174,7 @@ struct Sim {
             if (op == MW_EXIT) return;
             const bool buffered = cmd->buffered != 0;
             M = cmd->M;
+            force_nonlocal = cmd->force != 0;
             if (op == MW_SCAN) {
                 unsigned long long bt = INF, tmin = INF, tint, tall;
                 uint32_t bs = NONE32, src;
@@ -1209,7 +1211,7 @@ struct Sim {
                 const ClassState &c = cs[lane];
                 unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
                 tmin = v;
-                if (n_idle_pf > 0 && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
+                if ((n_idle_pf > 0 || force_nonlocal) && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
                 if (f_abandon()) {
                     v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
                     if (v < bt) { bt = v; bs = SRC_ABP + lane; }
@@ -1227,7 +1229,7 @@ struct Sim {
             uint32_t src;
             if (F & F_MW) {
                 // every warp scans its rows; the partial results meet in shared memory
-                if (lane == 0) { cmd->op = MW_SCAN; cmd->buffered = buffered; cmd->M = M; }
+                if (lane == 0) { cmd->op = MW_SCAN; cmd->buffered = buffered; cmd->M = M; cmd->force = force_nonlocal; }
                 __syncthreads();
                 scan_share(buffered, bt, bs, tmin);
                 warp_keys(bt, bs, tmin, tint, src, tmin_all);
@@ -1267,10 +1269,10 @@ struct Sim {
             uint32_t any_retire = 0;
             bool progressed = false;
             if (F & F_MW) {
-                if (lane == 0) { cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M; }
+                if (lane == 0) { cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M; cmd->force = force_nonlocal; }
                 __syncthreads();
             }
-            if (lane < (int)p.I && n_idle_pf == 0) {
+            if (lane < (int)p.I && n_idle_pf == 0 && !force_nonlocal) {
                 // local arrivals of this lane's class, in time order, up to the limit and up to the class's own
                 // next abandonment (which each arrival moves)
                 ClassState &c = cs[lane];
@@ -1347,6 +1349,7 @@ struct Sim {
                 }
                 if (err) return true;
                 dispatch();
+                force_nonlocal = false;
             } else if (!__any_sync(FULL, progressed)) {
                 err = ERR_INTERNAL;     // a round that neither ended an iteration nor handled an event: never spin
                 return true;
@@ -1359,6 +1362,7 @@ struct Sim {
     // switch) holds a full solo batch and could take a prefill afterwards.
     __device__ __forceinline__ bool is_local(uint32_t g, bool buffered) const
     {
+        if (force_nonlocal) return false;
         const uint32_t na = nact[g];
         if (na & 0x8000u) return false;
         if ((na & 0x4000u) && (buffered || (g < M && ndec[g] > p.B - 1))) return false;
@@ -1554,6 +1558,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kerne
         s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
         s.n_touch = 0; s.touch_all = false; s.need_start = 0; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
+        s.force_nonlocal = p.force_dispatch != 0 || h.force != 0;
         s.n_idle_pf = 0;
         s.idle_hint = NONE32;
         s.it_mixed = 0; s.it_solo = 0; s.busy_mixed = 0.0; s.busy_solo = 0.0;
@@ -1605,6 +1610,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kerne
             h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
             h.place_ord = s.place_ord; h.events = s.events; h.rounds = s.rounds; h.err = s.err;
             h.done = finished ? 1u : 0u;
+            h.force = s.force_nonlocal ? 1u : 0u;
             if (!finished) atomicAdd(p.not_done, 1u);
         }
         s.block_sync();

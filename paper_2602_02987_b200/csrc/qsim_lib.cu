@@ -53,6 +53,7 @@ struct qsim {
     uint32_t *d_inject_job = nullptr;
     uint32_t feat = 0;
     double T_end_abs = 0.0;       // end time reached by qsim_run_until calls
+    bool targets_changed = false; // qsim_set_targets since the last launch
     uint32_t *h_flag = nullptr;   // pinned
     void *ws = nullptr;
     cudaStream_t stream = nullptr;
@@ -223,6 +224,8 @@ int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
     p.advance = advance;
     p.horizon_iters = horizon;
     p.T_abs = T_abs;
+    p.force_dispatch = h->targets_changed ? 1u : 0u;
+    h->targets_changed = false;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
     h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
@@ -435,6 +438,7 @@ int qsim_set_targets(qsim_t *h, const qsim_targets *tg)
     }
     CUDA_TRY(cudaMemcpyAsync(h->d_blocks, &bp, sizeof bp, cudaMemcpyHostToDevice, h->stream));
     CUDA_TRY(cudaStreamSynchronize(h->stream));
+    h->targets_changed = true;
     return QSIM_OK;
 }
 
