@@ -197,6 +197,7 @@ def main():
     count, offset = shard(args.reps * world, world, rank)
     inp = presets.cfg1(R=count).with_(rep_offset=offset)
     sim = QSim(inp, device=f"cuda:{local}")
+    info = sim.layout_info()
     for _ in range(args.warmup):
         sim.run(args.horizon)
     it0, ev0, tot0 = sim.totals()
@@ -243,7 +244,7 @@ def main():
             st = simulate_host(inp, args.horizon)
             e_t += time.perf_counter() - t0
             e_iters += float(st["iters_mixed"].sum() + st["iters_solo"].sum())
-            d2h = int(sim.workspace_bytes * 0) + inp.R * 4224
+            d2h = inp.R * info["header_bytes"]
         ev = torch.tensor([e_t, e_iters], dtype=torch.float64, device="cuda")
         tm = ev[:1].clone()
         if world > 1:
@@ -256,7 +257,7 @@ def main():
         peak, peak_kind = measured_peaks()
         # algorithmic HBM bytes of one launch of the dominant kernel (qsim_run_kernel): the server state is
         # resident in shared memory, so what must move is the request life cycle plus the state staging
-        stage = 2.0 * inp.R * (4224 + 48 * ((inp.N + 31) // 32 * 32))
+        stage = 2.0 * inp.R * (info["header_bytes"] + info["image_bytes"])
         alg_bytes_per_launch = (JOB_BYTES * jobs / world + stage * args.steps) / max(n_launch / world, 1.0)
         kernel_ms = total_ms / max(n_launch / world, 1.0)
         achieved = alg_bytes_per_launch / (kernel_ms * 1e-3) / 1e9

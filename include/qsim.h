@@ -233,6 +233,11 @@ int qsim_simulate_static(const qsim_config *cfg, const qsim_class *classes, cons
  * most one non-local event and every local iteration end before it).  Synchronises the stream. */
 int qsim_round_count(qsim_t *h, uint64_t *rounds);
 
+/* Diagnostic: out[0] = bytes per replication that qsim_stats copies to the host, out[1] = bytes of per-GPU
+ * state staged per replication at kernel entry and exit, out[2] = shared memory per block, out[3] = warps per
+ * replication. */
+int qsim_layout_info(const qsim_t *h, uint64_t out[4]);
+
 /* Kernel launches issued by this handle so far (for accounting in benchmarks). */
 int qsim_launch_count(const qsim_t *h, uint64_t *launches);
 

@@ -19,7 +19,7 @@ _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_
 EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_run_until", "qsim_set_injected",
            "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
-           "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_destroy", "qsim_last_error")
+           "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error")
 
 
 class QSimError(RuntimeError):
@@ -85,6 +85,7 @@ def load_library():
                                            C.POINTER(qsim_targets), C.c_uint64, vp, vp, vp]
         L.qsim_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.qsim_round_count.argtypes = [vp, C.POINTER(C.c_uint64)]
+        L.qsim_layout_info.argtypes = [vp, C.POINTER(C.c_uint64)]
         L.qsim_destroy.argtypes = [vp]
         L.qsim_last_error.restype = C.c_char_p
         for n in EXPORTS:
@@ -199,6 +200,11 @@ class QSim:
         n = C.c_uint64()
         _check(self.L.qsim_launch_count(self.h, C.byref(n)))
         return int(n.value)
+
+    def layout_info(self) -> dict:
+        out = (C.c_uint64 * 4)()
+        _check(self.L.qsim_layout_info(self.h, out))
+        return dict(header_bytes=int(out[0]), image_bytes=int(out[1]), smem_bytes=int(out[2]), warps=int(out[3]))
 
     def round_count(self) -> int:
         n = C.c_uint64()

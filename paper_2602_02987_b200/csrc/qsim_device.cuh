@@ -1266,7 +1266,6 @@ struct Sim {
             uint32_t lim_s = src;
             if (wt <= lim_t) { lim_t = wt; lim_s = 0; }
             if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
-            uint32_t any_retire = 0;
             bool progressed = false;
             if (F & F_MW) {
                 if (lane == 0) { cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M; cmd->force = force_nonlocal; }
@@ -1309,8 +1308,7 @@ struct Sim {
             }
             if (SPL > 0) {
                 // pass 2: decode completions found in pass 1, retired by the whole warp, GPU by GPU
-                any_retire = __ballot_sync(FULL, retire_rows != 0);
-                if (any_retire) {
+                if (__ballot_sync(FULL, retire_rows != 0)) {
                     __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
 #pragma unroll
                     for (uint32_t k = 0; k < rows; ++k) {
@@ -1326,7 +1324,6 @@ struct Sim {
                     }
                 }
             }
-            (void)any_retire;
             // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
             // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
             bool redo = sched_pending;
@@ -1518,7 +1515,7 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
 
 // Advance replications to their new end time (or until the per-launch event budget runs out).
 template <int SPLT, uint32_t FT>
-__global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32) qsim_run_kernel(Params p)
+__global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_kernel(Params p)
 {
     extern __shared__ __align__(16) char sm[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

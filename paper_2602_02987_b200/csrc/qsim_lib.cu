@@ -157,8 +157,6 @@ const std::vector<RunVariant> &run_variants()
     return table;
 }
 
-qsim_config nohist_features(qsim_config c) { c.hist = 0; return c; }
-
 uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *coef)
 {
     uint32_t f = 0;
@@ -218,6 +216,59 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
     return best ? *best : *generic;
 }
 
+// Everything of a handle that needs no device memory: kernel parameters, kernel instance, block shape,
+// shared-memory and workspace layouts.
+int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const double *prices, const double *coef)
+{
+    h.cfg = cfg;
+    std::memcpy(h.cls, classes, cfg.I * sizeof(qsim_class));
+    h.prices[0] = prices[0];
+    h.prices[1] = prices[1];
+    Params &p = h.par;
+    p.I = cfg.I; p.N = cfg.N; p.Npad = (cfg.N + 31u) & ~31u; p.R = cfg.R; p.B = cfg.B; p.C = cfg.C;
+    p.nblk = cfg.nblk; p.gate = cfg.gate; p.router = cfg.router; p.placement = cfg.placement;
+    p.length_mode = cfg.length_mode; p.qcap = cfg.qcap; p.hist = cfg.hist;
+    p.seed = cfg.seed; p.rep_offset = cfg.rep_offset; p.block_len = cfg.block_len;
+    p.event_budget = 1ull << 28;
+    p.any_theta = 0;
+    for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
+    for (uint32_t i = 0; i < cfg.I; ++i) {
+        p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
+        p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
+        if (classes[i].theta > 0.0) p.any_theta = 1;
+    }
+    const bool kappa = coef[5] != 0.0;
+    const uint32_t feat = features_of(cfg, classes, coef);
+    RunVariant v = pick_run_kernel(cfg.N, feat);
+    // the per-GPU arrays are padded to the unrolled row count of the chosen instance
+    if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
+    // finish stamps + occupancy bits go to shared memory when the whole block state stays small
+    p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, kappa).total <= 40u * 1024u ? 1u : 0u;
+    if (p.slots_smem) v = pick_run_kernel(cfg.N, feat | F_SLOTS);
+    h.run_fn = v.fn;
+    h.nwarps = 1;
+    choose_multiwarp(cfg.N, p, h.run_fn, h.nwarps);
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa);
+    p.srv_bytes = h.lay.srv_bytes;
+    if (h.lay.total > 227u * 1024u)
+        return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
+    h.sec = layout_sections(cfg, p.srv_bytes);
+    return QSIM_OK;
+}
+
+void fill_blocks(BlockPar *blocks, const qsim_config &cfg, const double *rates, const qsim_targets *tg)
+{
+    for (uint32_t b = 0; b < cfg.nblk; ++b) {
+        BlockPar &bp = blocks[b];
+        std::memset(&bp, 0, sizeof bp);
+        bp.M = tg[b].M;
+        for (uint32_t i = 0; i < cfg.I; ++i) {
+            bp.xstar[i] = tg[b].xstar[i]; bp.nx[i] = tg[b].n_xstar[i]; bp.nq[i] = tg[b].n_qpstar[i];
+            bp.ps[i] = tg[b].p_solo[i]; bp.rate[i] = rates[(size_t)b * cfg.I + i];
+        }
+    }
+}
+
 int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
 {
     Params p = h->par;
@@ -250,55 +301,16 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     int ndev = 0;
     CUDA_TRY(cudaGetDeviceCount(&ndev));
     if (ndev < 1) return fail(QSIM_ECUDA, "no CUDA device");
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
     qsim *h = new (std::nothrow) qsim();
     if (!h) return fail(QSIM_ENOMEM, "host allocation failed");
-    CUDA_TRY(cudaGetDevice(&h->device));
-    h->cfg = *cfg;
-    std::memcpy(h->cls, classes, cfg->I * sizeof(qsim_class));
-    h->prices[0] = prices[0];
-    h->prices[1] = prices[1];
+    h->device = dev;
+    rc = configure(*h, *cfg, classes, prices, coef);
+    if (rc != QSIM_OK) { delete h; return rc; }
     Params &p = h->par;
-    p.I = cfg->I; p.N = cfg->N; p.Npad = (cfg->N + 31u) & ~31u; p.R = cfg->R; p.B = cfg->B; p.C = cfg->C;
-    p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
-    p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = cfg->hist;
-    p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
-    p.event_budget = 1ull << 28;
-    for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
-    for (uint32_t i = 0; i < cfg->I; ++i) {
-        p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
-        p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
-    }
-    p.any_theta = 0;
-    for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
-    {
-        // the per-GPU arrays are padded to the unrolled row count of the chosen instance
-        uint32_t feat = features_of(*cfg, classes, coef);
-        RunVariant v = pick_run_kernel(cfg->N, feat);
-        if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
-        // finish stamps + occupancy bits go to shared memory when the whole block state stays small
-        p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, p.coef[5] != 0.0).total <= 40u * 1024u ? 1u : 0u;
-        if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
-        h->run_fn = v.fn;
-        h->nwarps = 1;
-        choose_multiwarp(cfg->N, p, h->run_fn, h->nwarps);
-    }
-    h->lay = smem_layout(p.Npad, p.B, p.slots_smem, h->nwarps, p.coef[5] != 0.0);
-    p.srv_bytes = h->lay.srv_bytes;
-    if (h->lay.total > 227u * 1024u) {
-        delete h;
-        return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
-    }
-    h->sec = layout_sections(*cfg, p.srv_bytes);
     std::vector<BlockPar> blocks(cfg->nblk);
-    for (uint32_t b = 0; b < cfg->nblk; ++b) {
-        BlockPar &bp = blocks[b];
-        std::memset(&bp, 0, sizeof bp);
-        bp.M = tg[b].M;
-        for (uint32_t i = 0; i < cfg->I; ++i) {
-            bp.xstar[i] = tg[b].xstar[i]; bp.nx[i] = tg[b].n_xstar[i]; bp.nq[i] = tg[b].n_qpstar[i];
-            bp.ps[i] = tg[b].p_solo[i]; bp.rate[i] = rates[(size_t)b * cfg->I + i];
-        }
-    }
+    fill_blocks(blocks.data(), *cfg, rates, tg);
     cudaError_t e = cudaMalloc(&h->d_blocks, blocks.size() * sizeof(BlockPar));
     if (e == cudaSuccess) e = cudaMemcpy(h->d_blocks, blocks.data(), blocks.size() * sizeof(BlockPar), cudaMemcpyHostToDevice);
     if (e == cudaSuccess && cfg->length_mode == QSIM_LENGTH_TABLE) {
@@ -453,6 +465,16 @@ int qsim_sync(qsim_t *h)
 {
     if (!h) return fail(QSIM_EINVAL, "null handle");
     CUDA_TRY(cudaStreamSynchronize(h->stream));
+    return QSIM_OK;
+}
+
+int qsim_layout_info(const qsim_t *h, uint64_t out[4])
+{
+    if (!h || !out) return fail(QSIM_EINVAL, "null argument");
+    out[0] = sizeof(RepHeader);          // bytes per replication copied to the host by qsim_stats
+    out[1] = h->lay.srv_bytes;           // bytes of per-GPU state staged per replication at kernel entry and exit
+    out[2] = h->lay.total;               // shared memory per block
+    out[3] = h->nwarps;                  // warps per replication
     return QSIM_OK;
 }
 
@@ -677,42 +699,13 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     qsim h;   // a handle that owns nothing: no table allocation, no pinned flag
-    h.cfg = *cfg;
-    h.cfg.hist = 0;
-    std::memcpy(h.cls, classes, cfg->I * sizeof(qsim_class));
-    h.prices[0] = prices[0];
-    h.prices[1] = prices[1];
+    qsim_config nohist = *cfg;
+    nohist.hist = 0;                       // histograms are not recorded here
+    rc = configure(h, nohist, classes, prices, coef);
+    if (rc != QSIM_OK) return rc;
     h.device = dev;
     h.stream = stream;
     Params &p = h.par;
-    p.I = cfg->I; p.N = cfg->N; p.Npad = (cfg->N + 31u) & ~31u; p.R = cfg->R; p.B = cfg->B; p.C = cfg->C;
-    p.nblk = cfg->nblk; p.gate = cfg->gate; p.router = cfg->router; p.placement = cfg->placement;
-    p.length_mode = cfg->length_mode; p.qcap = cfg->qcap; p.hist = 0;
-    p.seed = cfg->seed; p.rep_offset = cfg->rep_offset; p.block_len = cfg->block_len;
-    p.event_budget = 1ull << 28;
-    for (int k = 0; k < 6; ++k) p.coef[k] = coef[k];
-    for (uint32_t i = 0; i < cfg->I; ++i) {
-        p.cls[i].theta = classes[i].theta; p.cls[i].P = classes[i].P; p.cls[i].D = classes[i].D;
-        p.cls[i].prio = classes[i].prio_rank; p.cls[i].pad = 0;
-    }
-    p.any_theta = 0;
-    for (uint32_t i = 0; i < cfg->I; ++i) if (classes[i].theta > 0.0) p.any_theta = 1;
-    {
-        uint32_t feat = features_of(nohist_features(*cfg), classes, coef);
-        RunVariant v = pick_run_kernel(cfg->N, feat);
-        if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
-        p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, p.coef[5] != 0.0).total <= 40u * 1024u ? 1u : 0u;
-        if (p.slots_smem) v = pick_run_kernel(cfg->N, feat | F_SLOTS);
-        h.run_fn = v.fn;
-        h.nwarps = 1;
-        choose_multiwarp(cfg->N, p, h.run_fn, h.nwarps);
-    }
-    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, p.coef[5] != 0.0);
-    p.srv_bytes = h.lay.srv_bytes;
-    if (h.lay.total > 227u * 1024u) return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
-    qsim_config nohist = *cfg;
-    nohist.hist = 0;
-    h.sec = layout_sections(nohist, p.srv_bytes);
     // scratch = [state sections | block table | length tables]
     const size_t off_blocks = h.sec.total;
     const size_t off_lengths = align256(off_blocks + (size_t)cfg->nblk * sizeof(BlockPar));
@@ -724,14 +717,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
                                          std::to_string((size_t)QSIM_STATIC_SCRATCH_BYTES) +
                                          "; reduce R, N*B or qcap, or use qsim_create/qsim_bind with your own workspace");
     BlockPar blocks[64];
-    std::memset(blocks, 0, sizeof blocks);
-    for (uint32_t b = 0; b < cfg->nblk; ++b) {
-        blocks[b].M = tg[b].M;
-        for (uint32_t i = 0; i < cfg->I; ++i) {
-            blocks[b].xstar[i] = tg[b].xstar[i]; blocks[b].nx[i] = tg[b].n_xstar[i]; blocks[b].nq[i] = tg[b].n_qpstar[i];
-            blocks[b].ps[i] = tg[b].p_solo[i]; blocks[b].rate[i] = rates[(size_t)b * cfg->I + i];
-        }
-    }
+    fill_blocks(blocks, *cfg, rates, tg);
     // pageable sources: these copies have returned from the host buffers when the calls return
     CUDA_TRY(cudaMemcpyAsync(base + off_blocks, blocks, (size_t)cfg->nblk * sizeof(BlockPar), cudaMemcpyHostToDevice, stream));
     if (len_bytes) CUDA_TRY(cudaMemcpyAsync(base + off_lengths, lengths, len_bytes, cudaMemcpyHostToDevice, stream));
