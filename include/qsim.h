@@ -53,7 +53,8 @@ enum {
     QSIM_ESTATE = -6       /* call out of order (run before bind, ...) */
 };
 
-enum { QSIM_GATE_OCCUPANCY = 0, QSIM_GATE_PRIORITY = 1 };
+enum { QSIM_GATE_OCCUPANCY = 0, QSIM_GATE_PRIORITY = 1,
+       QSIM_GATE_FCFS = 2 /* oldest waiting request first: the FCFS-and-Route ablation of the paper's EC */ };
 enum { QSIM_ROUTER_SOLO_FIRST = 0, QSIM_ROUTER_SLI = 1 };
 enum { QSIM_PLACE_RANDOM = 0, QSIM_PLACE_LEAST_LOADED = 1 };
 enum { QSIM_PRICING_BUNDLED = 0, QSIM_PRICING_SEPARATE = 1 };

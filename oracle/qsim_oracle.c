@@ -342,6 +342,13 @@ static int gate_class(const orc_sim *s, const rep_t *R)
 {
     const orc_targets *tg = &s->tg[R->blk];
     int best = -1;
+    if (s->cfg.gate == 2) {
+        /* ablation "FCFS-and-Route" (EC, additional ablation studies): no class rule, the oldest waiting request goes first */
+        for (uint32_t i = 0; i < s->cfg.I; ++i)
+            if (R->pq_n[i] > 0 && (best < 0 || R->pq[i][0].t_arr < R->pq[best][0].t_arr))
+                best = (int)i;
+        return best;
+    }
     if (s->cfg.gate == 1) {
         for (uint32_t i = 0; i < s->cfg.I; ++i)
             if (R->pq_n[i] > 0 && (best < 0 || s->cls[i].prio_rank < s->cls[best].prio_rank))

@@ -45,7 +45,7 @@ constexpr int TOUCH_CAP = 48;
 // run time; otherwise the set bits say which features the instance contains and everything else is
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
-                   F_OCC = 128, F_SLOTS = 256, F_MW = 512;
+                   F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024;
 // F_MW: several warps per replication.  Warp 0 (the master) runs the round loop and every event handler; the
 // other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
 // round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
@@ -675,6 +675,20 @@ struct Sim {
     // --- prefill gate ------------------------------------------------------------------------------
     __device__ uint32_t gate_class()
     {
+        if ((F & F_GENERIC) && p.gate == 2) {
+            // FCFS ablation: the class whose head-of-line request arrived first (heads are mirrored on chip)
+            cp_async_wait_all();
+            __syncwarp();
+            uint32_t best = NONE32;
+            double bt = 0.0;
+            for (uint32_t i = 0; i < p.I; ++i) {
+                if (cs[i].pq_n == 0) continue;
+                const double ta = pqh[i].t;
+                if (best == NONE32 || ta < bt) { best = i; bt = ta; }
+            }
+            __syncwarp();
+            return best;
+        }
         if (!f_occ()) {
             // Prioritize-and-Route: largest D_i/P_i among waiting classes = smallest static rank
             uint32_t key = NONE32;
@@ -912,9 +926,16 @@ struct Sim {
         const int owner = (int)(g & 31u);
         uint32_t n = nd, newmin = NONE32, Kdrop = 0;
         const size_t base = (size_t)g * p.B;
-        for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
-            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
-            const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
+        const int nchunks = (int)((nd + 31u) >> 5);
+        // the first 8 chunks of finish stamps are fetched up front so their latencies overlap
+        uint32_t fpre[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const uint32_t j = ((uint32_t)c << 5) + (uint32_t)lane;
+            fpre[c] = (c < nchunks && j < nd) ? s_fin[base + j] : NONE32;
+        }
+        // one chunk: account the requests that finish now and move tail entries into their places
+        auto chunk = [&](int k, uint32_t f) {
             const bool hit = f == itg;
             if (!hit) newmin = min(newmin, f);
             uint32_t hits = __ballot_sync(FULL, hit);
@@ -923,11 +944,8 @@ struct Sim {
                 hits &= ~(1u << hl);
                 const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
                 const SlotRec rh = s_rec[base + h];
-                const double tpf = rh.tpf;
-                const uint32_t pk = rh.pk;
-                account_done(pk, tpf, te);
-                const uint32_t P = job_P(pk), D = job_D(pk);
-                Kdrop += P + D;
+                account_done(rh.pk, rh.tpf, te);
+                Kdrop += job_P(rh.pk) + job_D(rh.pk);
                 const uint32_t last = n - 1;
                 __syncwarp();
                 if (lane == 0 && h != last) {
@@ -936,7 +954,14 @@ struct Sim {
                 }
                 n = last;
             }
+        };
+        for (int k = nchunks - 1; k >= 8; --k) {
+            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
+            chunk(k, j < nd ? s_fin[base + j] : NONE32);
         }
+#pragma unroll
+        for (int k = 7; k >= 0; --k)
+            if (k < nchunks) chunk(k, fpre[k]);
         newmin = __reduce_min_sync(FULL, newmin);
         if (lane == owner) {
             ndec[g] = (uint16_t)n;

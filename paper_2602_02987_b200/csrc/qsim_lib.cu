@@ -95,7 +95,7 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
     if (cfg->C < 1 || cfg->C > 65535) return fail(QSIM_EINVAL, "C must be in 1..65535");
     if (cfg->nblk < 1) return fail(QSIM_EINVAL, "nblk must be >= 1");
     if (cfg->qcap < 1 || cfg->qcap > (1u << 24)) return fail(QSIM_EINVAL, "qcap must be in 1..2^24");
-    if (cfg->gate > 1 || cfg->router > 1 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
+    if (cfg->gate > 2 || cfg->router > 1 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
         return fail(QSIM_EINVAL, "enum out of range");
     if (cfg->nblk > 1 && !(cfg->block_len > 0.0 && std::isfinite(cfg->block_len)))
         return fail(QSIM_EINVAL, "block_len must be positive when nblk > 1");
@@ -168,6 +168,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
     if (c.nblk > 1) f |= F_BLOCKS;
     if (c.placement == QSIM_PLACE_RANDOM) f |= F_RANDOM;
     if (c.gate == QSIM_GATE_OCCUPANCY) f |= F_OCC;
+    if (c.gate == QSIM_GATE_FCFS) f |= F_FCFS;
     return f;
 }
 
@@ -208,7 +209,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
         if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
         // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits
         // (abandonment, KV slope, blocks) may be present without being used
-        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_HIST | F_SLOTS;
+        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_FCFS | F_HIST | F_SLOTS;
         if (feat == ~0u || (feat & MODES) != (v.feat & MODES) || (feat & ~v.feat) != 0) continue;
         const int extra = __builtin_popcount(v.feat & ~feat);
         if (extra < best_bits) { best = &v; best_bits = extra; }

@@ -23,6 +23,7 @@ NBIN = 1024       # bins of the log-linear latency histograms (32 octaves x 32 s
 # prefill gate
 GATE_OCCUPANCY = 0   # occupancy-deviation gate (Section 4.1, "Upstream (prefill) gate")
 GATE_PRIORITY = 1    # largest D_i/P_i first (Section 5.1.1, Prioritize-and-Route)
+GATE_FCFS = 2        # oldest waiting request first, no class rule (ablation FG-SP of the EC ablation study)
 # decode router
 ROUTER_SOLO_FIRST = 0      # single FCFS buffer, solo GPUs first (Section 4.1, "Downstream routing")
 ROUTER_SLI = 1             # randomized split with p_s,i, two buffers (Section 5.2)

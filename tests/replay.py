@@ -173,6 +173,9 @@ class Replay:
             cand = [i for i in waiting if xs[i] > 0]
             key = {i: ((self.X[i] - nx[i]) / xs[i], -(len(self.pq[i]) - nq[i]), i) for i in cand}
             assert cls == min(cand, key=lambda i: key[i]), ("occupancy gate argmin violated", key, cls)
+        elif inp.gate == 2:
+            oldest = min(waiting, key=lambda i: (self.jobs[(i, self.pq[i][0])]["t_arr"], i))
+            assert cls == oldest, "FCFS gate violated"
         else:
             assert cls == min(waiting, key=lambda i: (int(inp.prio_rank[i]), i)), "priority gate violated"
         cands = [h for h in range(M) if self.pf[h] is None and len(self.dec[h]) <= self.B - 1]

@@ -66,6 +66,12 @@ def test_paper_instance_all_policy_modes(gate, placement, router):
     check(inp, 6000)
 
 
+def test_fcfs_gate_ablation():
+    from qsim_inputs.spec import GATE_FCFS
+    check(presets.paper_instance(n=20, R=4, gate=GATE_FCFS), 6000)
+    check(presets.cfg1(R=4).with_(gate=GATE_FCFS), 1000)
+
+
 def test_cfg1_subset_lognormal_tables_priority_gate():
     inp = presets.cfg1(R=8)
     check(inp, 1500)

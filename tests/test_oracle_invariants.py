@@ -5,7 +5,7 @@ import pytest
 
 from oracle import OracleSim, run_oracle
 from qsim_inputs import presets
-from qsim_inputs.spec import (GATE_OCCUPANCY, GATE_PRIORITY, PLACE_LEAST_LOADED, PLACE_RANDOM, ROUTER_SLI)
+from qsim_inputs.spec import (GATE_FCFS, GATE_OCCUPANCY, GATE_PRIORITY, PLACE_LEAST_LOADED, PLACE_RANDOM, ROUTER_SLI)
 
 from replay import Replay, expected_counts, isclose
 
@@ -27,6 +27,8 @@ def small_cases():
     yield presets.cfg0(R=2, horizon_iters=400)
     yield presets.cfg0(R=2, horizon_iters=400, placement=PLACE_RANDOM)
     yield presets.cfg0(R=1, horizon_iters=400).with_(gate=GATE_PRIORITY)
+    yield presets.cfg0(R=1, horizon_iters=400).with_(gate=GATE_FCFS)
+    yield presets.paper_instance(n=6, R=1, horizon_iters=1500, gate=GATE_FCFS)
     yield presets.paper_instance(n=5, R=2, horizon_iters=1500)
     yield presets.paper_instance(n=8, R=1, horizon_iters=1500, placement=PLACE_LEAST_LOADED, gate=GATE_PRIORITY)
     c1 = presets.cfg1(R=1, horizon_iters=150)
