@@ -926,16 +926,9 @@ struct Sim {
         const int owner = (int)(g & 31u);
         uint32_t n = nd, newmin = NONE32, Kdrop = 0;
         const size_t base = (size_t)g * p.B;
-        const int nchunks = (int)((nd + 31u) >> 5);
-        // the first 8 chunks of finish stamps are fetched up front so their latencies overlap
-        uint32_t fpre[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            const uint32_t j = ((uint32_t)c << 5) + (uint32_t)lane;
-            fpre[c] = (c < nchunks && j < nd) ? s_fin[base + j] : NONE32;
-        }
-        // one chunk: account the requests that finish now and move tail entries into their places
-        auto chunk = [&](int k, uint32_t f) {
+        for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
+            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
+            const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
             const bool hit = f == itg;
             if (!hit) newmin = min(newmin, f);
             uint32_t hits = __ballot_sync(FULL, hit);
@@ -954,14 +947,7 @@ struct Sim {
                 }
                 n = last;
             }
-        };
-        for (int k = nchunks - 1; k >= 8; --k) {
-            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
-            chunk(k, j < nd ? s_fin[base + j] : NONE32);
         }
-#pragma unroll
-        for (int k = 7; k >= 0; --k)
-            if (k < nchunks) chunk(k, fpre[k]);
         newmin = __reduce_min_sync(FULL, newmin);
         if (lane == owner) {
             ndec[g] = (uint16_t)n;
