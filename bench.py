@@ -32,9 +32,9 @@ METRIC = "simulated GPU-server-iterations/sec"
 UNIT = "server-iterations/s"
 JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
                            # decode-buffer pass, each written and read once at 32-byte sector granularity
-# DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from the ncu capture summarised in
-# profiles/qsim_run_kernel_cfg1_lookahead.md (740.6 MB for 1.414e8 iterations; traffic grows with the iterations
-# of a launch, so a full launch is that figure times its iterations)
+# DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from an ncu capture of a 2000-iteration
+# launch (dram__bytes_read.sum + dram__bytes_write.sum = 740.6 MB for 1.414e8 iterations); traffic grows with the
+# iterations of a launch, so a full launch is that figure times its iterations
 NCU_DRAM_BYTES_PER_ITER = 740.6e6 / 1.414e8
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
 R_PER_GPU = 1024
