@@ -15,7 +15,8 @@
  * waiting class with the smallest occupancy deviation (X_i - n x*_i)/x*_i, ties to the largest
  * Q_p,i - n q*_p,i [Section 4.1], or the class with the largest D_i/P_i [Section 5.1.1].  The decode
  * router serves one FCFS buffer, solo GPUs first [Section 4.1], or splits jobs between a solo and a
- * mixed buffer with probability p_s,i [Section 5.2].  Rates and targets are piecewise constant over
+ * mixed buffer with probability p_s,i [Section 5.2], optionally picking the class inside each pool by
+ * the weights varpi [EC, General SLI-aware Extension].  Rates and targets are piecewise constant over
  * blocks of block_len seconds and switch without pre-emption [Section 6.2].  Revenue is reported
  * under bundled and separate charging [Eq. (21)-(23)] from integer token counters.
  *
@@ -55,7 +56,10 @@ enum {
 
 enum { QSIM_GATE_OCCUPANCY = 0, QSIM_GATE_PRIORITY = 1,
        QSIM_GATE_FCFS = 2 /* oldest waiting request first: the FCFS-and-Route ablation of the paper's EC */ };
-enum { QSIM_ROUTER_SOLO_FIRST = 0, QSIM_ROUTER_SLI = 1 };
+enum { QSIM_ROUTER_SOLO_FIRST = 0, QSIM_ROUTER_SLI = 1,
+       QSIM_ROUTER_SLI_GENERAL = 2 /* two pools as QSIM_ROUTER_SLI; a freed slot goes to a class drawn with the pool's
+                                      weights varpi among the classes that wait there, oldest request of the class
+                                      first [EC, General SLI-aware Extension] */ };
 enum { QSIM_PLACE_RANDOM = 0, QSIM_PLACE_LEAST_LOADED = 1 };
 enum { QSIM_PRICING_BUNDLED = 0, QSIM_PRICING_SEPARATE = 1 };
 enum { QSIM_LENGTH_FIXED = 0, QSIM_LENGTH_TABLE = 1 };
@@ -89,6 +93,8 @@ typedef struct {           /* policy parameters of one block, from the steady-st
     double n_xstar[QSIM_MAXI];   /* n x*_i */
     double n_qpstar[QSIM_MAXI];  /* n q*_p,i */
     double p_solo[QSIM_MAXI];    /* p_s,i of the SLI-aware router */
+    double w_solo[QSIM_MAXI];    /* varpi_s,i >= 0: class-selection weights of the solo pool (QSIM_ROUTER_SLI_GENERAL only) */
+    double w_mix[QSIM_MAXI];     /* varpi_m,i >= 0: the same for the mixed pool */
 } qsim_targets;
 
 typedef struct {

@@ -109,7 +109,7 @@ uint32_t orc_hist_bin(double x)
 /* ------------------------------------------------------------------------------------------ */
 
 enum { STREAM_ARRIVAL = 0, STREAM_ABANDON_P = 1, STREAM_ABANDON_D0 = 2, STREAM_ABANDON_D1 = 3,
-       STREAM_PLACEMENT = 4, STREAM_SLI = 5 };
+       STREAM_PLACEMENT = 4, STREAM_SLI = 5, STREAM_SELECT0 = 6, STREAM_SELECT1 = 7 };
 
 typedef struct { double t_arr; uint32_t P, D; uint64_t ord; } job_t;
 typedef struct { double t_pf; uint32_t P, D, cls; uint64_t ord; } djob_t;
@@ -146,7 +146,7 @@ typedef struct {
     uint32_t Qd_pool[2][ORC_MAXI];
     abclock_t abp[ORC_MAXI], abd[2][ORC_MAXI];
     server_t *srv;
-    uint64_t place_ord, sli_ord[ORC_MAXI];
+    uint64_t place_ord, sli_ord[ORC_MAXI], sel_ord[2];
     /* state counts and their time integrals */
     uint32_t X[ORC_MAXI], Ym[ORC_MAXI], Ys[ORC_MAXI];
     area_t aQp[ORC_MAXI], aX[ORC_MAXI], aQd[ORC_MAXI], aYm[ORC_MAXI], aYs[ORC_MAXI];
@@ -311,12 +311,13 @@ static int choose_server(orc_sim *s, uint32_t r, int want)
     return best;
 }
 
-static void place_decode(orc_sim *s, uint32_t r, uint32_t pool, uint32_t g, double t)
+/* entry `pos` of the pool's buffer (0 = head) starts decoding on GPU g */
+static void place_decode(orc_sim *s, uint32_t r, uint32_t pool, uint32_t g, uint32_t pos, double t)
 {
     rep_t *R = &s->reps[r];
     server_t *v = &R->srv[g];
-    djob_t j = R->dq[pool][0];
-    memmove(R->dq[pool], R->dq[pool] + 1, (size_t)(R->dq_n[pool] - 1) * sizeof(djob_t));
+    djob_t j = R->dq[pool][pos];
+    memmove(R->dq[pool] + pos, R->dq[pool] + pos + 1, (size_t)(R->dq_n[pool] - 1 - pos) * sizeof(djob_t));
     uint32_t i = j.cls;
     ab_change(&R->abd[pool][i], s->cls[i].theta, R->Qd_pool[pool][i], R->Qd_pool[pool][i] - 1, t);
     area_touch(&R->aQd[i], R->Qd_pool[0][i] + R->Qd_pool[1][i], t);
@@ -379,6 +380,38 @@ static void start_iteration(orc_sim *s, rep_t *R, uint32_t g, double t)
     v->running = 1;
 }
 
+/* General SLI-aware router: when a slot of the pool frees up, the class is drawn with probabilities
+ * proportional to varpi restricted to the classes that wait in the pool's buffer; its oldest request goes.
+ * One waiting class needs no draw; if every waiting class has weight 0 the oldest request of the buffer goes. */
+static uint32_t select_in_pool(orc_sim *s, uint32_t r, uint32_t pool)
+{
+    rep_t *R = &s->reps[r];
+    const orc_targets *tg = &s->tg[R->blk];
+    const double *w = pool == 0 ? tg->w_solo : tg->w_mix;
+    uint32_t I = s->cfg.I, nonempty = 0, only = 0;
+    double Wsum = 0.0;
+    for (uint32_t i = 0; i < I; ++i)
+        if (R->Qd_pool[pool][i] > 0) { ++nonempty; only = i; Wsum = Wsum + w[i]; }
+    uint32_t cls = only;
+    if (nonempty > 1) {
+        if (!(Wsum > 0.0)) return 0;
+        uint32_t wd[4];
+        draw(s, r, (pool == 0 ? STREAM_SELECT0 : STREAM_SELECT1) << 8, R->sel_ord[pool]++, wd);
+        double x = orc_u53(wd[0], wd[1]) * Wsum, cum = 0.0;
+        int chosen = -1, last = -1;
+        for (uint32_t i = 0; i < I && chosen < 0; ++i) {
+            if (R->Qd_pool[pool][i] == 0) continue;
+            cum = cum + w[i];
+            if (w[i] > 0.0) last = (int)i;
+            if (w[i] > 0.0 && cum >= x) chosen = (int)i;
+        }
+        cls = (uint32_t)(chosen >= 0 ? chosen : last);
+    }
+    uint32_t pos = 0;
+    while (R->dq[pool][pos].cls != cls) ++pos;
+    return pos;
+}
+
 static void dispatch(orc_sim *s, uint32_t r, double t)
 {
     rep_t *R = &s->reps[r];
@@ -389,14 +422,14 @@ static void dispatch(orc_sim *s, uint32_t r, double t)
             int g = choose_server(s, r, WANT_SOLO_DECODE);
             if (g < 0) g = choose_server(s, r, WANT_MIX_DECODE);
             if (g < 0) break;
-            place_decode(s, r, 0, (uint32_t)g, t);
+            place_decode(s, r, 0, (uint32_t)g, 0, t);
         }
     } else {
         for (uint32_t pool = 0; pool < 2; ++pool)
             while (R->dq_n[pool] > 0) {
                 int g = choose_server(s, r, pool == 0 ? WANT_SOLO_DECODE : WANT_MIX_DECODE);
                 if (g < 0) break;
-                place_decode(s, r, pool, (uint32_t)g, t);
+                place_decode(s, r, pool, (uint32_t)g, c->router == 2 ? select_in_pool(s, r, pool) : 0u, t);
             }
     }
     /* prefill gate on the mixed GPUs whose prefill slot is idle */
@@ -534,14 +567,14 @@ static void on_server(orc_sim *s, uint32_t r, uint32_t g, double t)
             double ttft = t - v->pf_job.t_arr;
             cs->sum_ttft = cs->sum_ttft + ttft;
             if (R->h_ttft) R->h_ttft[(size_t)i * ORC_NBIN + orc_hist_bin(ttft)]++;
-            trace(s, r, ORC_EV_PREFILL_DONE, t, (int)i, (int)g, v->pf_job.ord, 0.0);
             /* hand over to the decode stage: pool drawn once per job under the SLI-aware router */
             uint32_t pool = 0;
-            if (c->router == 1) {
+            if (c->router >= 1) {
                 uint32_t w[4];
                 draw(s, r, (STREAM_SLI << 8) | i, R->sli_ord[i]++, w);
                 pool = (orc_u53(w[0], w[1]) <= s->tg[R->blk].p_solo[i]) ? 0u : 1u;
             }
+            trace(s, r, ORC_EV_PREFILL_DONE, t, (int)i, (int)g, v->pf_job.ord, (double)pool);   /* aux = pool */
             if (R->dq_n[pool] >= c->qcap) {
                 cs->overflow_d++;
                 trace(s, r, ORC_EV_OVERFLOW, t, (int)i, (int)g, v->pf_job.ord, 0.0);

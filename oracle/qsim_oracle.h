@@ -18,7 +18,8 @@
  *   - static planning: GPUs 0..M-1 mixed, M..N-1 solo                   [Section 4.1]
  *   - prefill gate: occupancy deviation xi_i, or static D_i/P_i priority [Sections 4.1, 5.1.1]
  *   - decode router: solo-first with one FCFS buffer, or the SLI-aware
- *     randomized split with two buffers                                  [Sections 4.1, 5.2]
+ *     randomized split with two buffers, optionally with class selection
+ *     inside each pool by the weights varpi                              [Sections 4.1, 5.2, EC general SLI extension]
  *   - revenue under bundled and separate charging                        [Eq. (21)-(23)]
  *   - piecewise-constant rate / target tables switched at block ends without pre-emption
  *                                                                        [Section 6.2, online controller]
@@ -58,6 +59,7 @@ typedef struct {
 typedef struct {
     uint32_t M, pad;
     double xstar[ORC_MAXI], n_xstar[ORC_MAXI], n_qpstar[ORC_MAXI], p_solo[ORC_MAXI];
+    double w_solo[ORC_MAXI], w_mix[ORC_MAXI];   /* varpi_s,i, varpi_m,i of the general SLI-aware router */
 } orc_targets;
 
 typedef struct {

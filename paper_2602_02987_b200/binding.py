@@ -39,7 +39,8 @@ class qsim_class(C.Structure):
 
 class qsim_targets(C.Structure):
     _fields_ = [("M", C.c_uint32), ("reserved", C.c_uint32), ("xstar", C.c_double * MAXI),
-                ("n_xstar", C.c_double * MAXI), ("n_qpstar", C.c_double * MAXI), ("p_solo", C.c_double * MAXI)]
+                ("n_xstar", C.c_double * MAXI), ("n_qpstar", C.c_double * MAXI), ("p_solo", C.c_double * MAXI),
+                ("w_solo", C.c_double * MAXI), ("w_mix", C.c_double * MAXI)]
 
 
 class qsim_class_stats(C.Structure):
@@ -123,6 +124,8 @@ def marshal(inp):
             tg[b].n_xstar[i] = float(inp.n_xstar[b, i])
             tg[b].n_qpstar[i] = float(inp.n_qpstar[b, i])
             tg[b].p_solo[i] = float(inp.p_solo[b, i])
+            tg[b].w_solo[i] = float(inp.w_solo[b, i])
+            tg[b].w_mix[i] = float(inp.w_mix[b, i])
     rates = np.ascontiguousarray(inp.rates, np.float64)
     lengths = None if inp.lengths is None else np.ascontiguousarray(inp.lengths, np.uint32)
     prices = np.ascontiguousarray(inp.prices, np.float64)
@@ -182,12 +185,14 @@ class QSim:
     def run_until(self, T: float) -> None:
         _check(self.L.qsim_run_until(self.h, float(T)))
 
-    def set_targets(self, M, xstar, n_xstar, n_qpstar, p_solo) -> None:
+    def set_targets(self, M, xstar, n_xstar, n_qpstar, p_solo, w_solo=None, w_mix=None) -> None:
         tg = qsim_targets()
         tg.M = int(M)
         for i in range(self.inp.I):
             tg.xstar[i] = float(xstar[i]); tg.n_xstar[i] = float(n_xstar[i])
             tg.n_qpstar[i] = float(n_qpstar[i]); tg.p_solo[i] = float(p_solo[i])
+            if w_solo is not None:
+                tg.w_solo[i] = float(w_solo[i]); tg.w_mix[i] = float(w_mix[i])
         _check(self.L.qsim_set_targets(self.h, C.byref(tg)))
 
     def sync(self) -> None:

@@ -45,7 +45,7 @@ constexpr int TOUCH_CAP = 48;
 // run time; otherwise the set bits say which features the instance contains and everything else is
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
-                   F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024;
+                   F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024, F_SLIG = 2048;
 // F_MW: several warps per replication.  Warp 0 (the master) runs the round loop and every event handler; the
 // other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
 // round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
@@ -58,7 +58,7 @@ constexpr int MW_MAX = 16;
 constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
 
 enum { STREAM_ARRIVAL = 0, STREAM_ABANDON_P = 1, STREAM_ABANDON_D0 = 2, STREAM_ABANDON_D1 = 3,
-       STREAM_PLACEMENT = 4, STREAM_SLI = 5 };
+       STREAM_PLACEMENT = 4, STREAM_SLI = 5, STREAM_SELECT0 = 6, STREAM_SELECT1 = 7 };
 enum { WANT_SOLO = 0, WANT_MIX = 1, WANT_PREFILL = 2 };
 enum { ERR_NONE = 0, ERR_INTERNAL = 1 };
 
@@ -82,6 +82,7 @@ struct RepHeader {
     unsigned long long place_ord, events, H_total, rounds;
     uint32_t blk, done, err, force;    // force: the next event must be followed by a dispatch (targets were replaced)
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
+    unsigned long long sel_ord0, sel_ord1;   // class selections drawn so far in the solo / mixed pool (general SLI router)
     unsigned long long iters_mixed[32], iters_solo[32];
     double busy_mixed[32], busy_solo[32];
     ClassState cs[MAXI];
@@ -98,7 +99,7 @@ struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: 
 struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
 
 struct ClassPar { double theta; uint32_t P, D, prio, pad; };
-struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI]; };
+struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI], ws[MAXI], wm[MAXI]; };
 
 struct Params {
     uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance, any_theta, slots_smem;
@@ -282,7 +283,8 @@ __device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long l
 template <int SPL, uint32_t F>
 struct Sim {
     __device__ __forceinline__ bool f_abandon() const { return (F & F_GENERIC) ? p.any_theta != 0 : (F & F_ABANDON) != 0; }
-    __device__ __forceinline__ bool f_sli() const { return (F & F_GENERIC) ? p.router == 1 : (F & F_SLI) != 0; }
+    __device__ __forceinline__ bool f_sli() const { return (F & F_GENERIC) ? p.router >= 1 : (F & F_SLI) != 0; }
+    __device__ __forceinline__ bool f_slig() const { return (F & F_GENERIC) ? p.router == 2 : false; }
     __device__ __forceinline__ bool f_kappa() const { return (F & F_GENERIC) ? p.coef[5] != 0.0 : (F & F_KAPPA) != 0; }
     __device__ __forceinline__ bool f_hist() const { return (F & F_GENERIC) ? hist != nullptr : (F & F_HIST) != 0; }
     __device__ __forceinline__ bool f_blocks() const { return (F & F_GENERIC) ? p.nblk > 1 : (F & F_BLOCKS) != 0; }
@@ -325,7 +327,7 @@ struct Sim {
     uint32_t n_idle_pf;          // mixed GPUs whose prefill slot is idle (and that may take a prefill)
     uint32_t idle_hint;          // when n_idle_pf == 1: that GPU if known, else NONE32
     uint32_t need_start;         // per lane: rows of own GPUs touched by the current event
-    unsigned long long place_ord, events, rounds;
+    unsigned long long place_ord, events, rounds, sel_ord0, sel_ord1;
     bool drain_dirty, gate_dirty, touch_all;
     bool force_nonlocal;         // treat the next event, whatever it is, as non-local (it must end with a dispatch)
     // per-lane partial sums
@@ -612,13 +614,64 @@ struct Sim {
     }
 
     // --- decode placement ------------------------------------------------------------------------
-    // head of the pool's buffer goes to GPU g
-    __device__ void place_decode(uint32_t pool, uint32_t g)
+    // General SLI-aware router: position (in buffer order) of the request that gets the freed slot of the pool.
+    // The class is drawn with probabilities proportional to varpi over the classes that wait in the pool; one
+    // waiting class needs no draw, and with no positive weight among them the head of the buffer goes.
+    __device__ uint32_t select_in_pool(uint32_t pool)
+    {
+        const BlockPar &bp = p.blocks[blk];
+        uint32_t nonempty = 0, cls = 0;
+        double Wsum = 0.0;
+        for (uint32_t i = 0; i < p.I; ++i)
+            if ((pool ? cs[i].Qd1 : cs[i].Qd0) > 0) { ++nonempty; cls = i; Wsum = __dadd_rn(Wsum, pool ? bp.wm[i] : bp.ws[i]); }
+        if (nonempty > 1) {
+            if (!(Wsum > 0.0)) return 0;
+            uint32_t w0, w1, w2, w3;
+            if (pool) draw(p, rep, STREAM_SELECT1 << 8, sel_ord1++, w0, w1, w2, w3);
+            else      draw(p, rep, STREAM_SELECT0 << 8, sel_ord0++, w0, w1, w2, w3);
+            const double x = __dmul_rn(u53(w0, w1), Wsum);
+            double cum = 0.0;
+            uint32_t chosen = NONE32, last = NONE32;
+            for (uint32_t i = 0; i < p.I && chosen == NONE32; ++i) {
+                if ((pool ? cs[i].Qd1 : cs[i].Qd0) == 0) continue;
+                const double w = pool ? bp.wm[i] : bp.ws[i];
+                cum = __dadd_rn(cum, w);
+                if (w > 0.0) { last = i; if (cum >= x) chosen = i; }
+            }
+            cls = chosen != NONE32 ? chosen : last;
+        }
+        // oldest request of the class
+        const QEntry *ring = dq + (size_t)pool * p.qcap;
+        const uint32_t head = pool ? dq_head1 : dq_head0, n = pool ? dq_n1 : dq_n0;
+        for (uint32_t k = 0; k < n; k += 32) {
+            const uint32_t j = k + (uint32_t)lane;
+            bool mine = false;
+            if (j < n) {
+                uint32_t src = head + j; if (src >= p.qcap) src -= p.qcap;
+                mine = ring[src].cls == cls;
+            }
+            const uint32_t b = __ballot_sync(FULL, mine);
+            if (b) return k + (uint32_t)__ffs((int)b) - 1u;
+        }
+        err = ERR_INTERNAL;
+        return 0;
+    }
+
+    // entry pos (0 = head) of the pool's buffer goes to GPU g
+    __device__ void place_decode(uint32_t pool, uint32_t g, uint32_t pos = 0)
     {
         const uint32_t head = pool ? dq_head1 : dq_head0;
-        const QEntry e = dq[(size_t)pool * p.qcap + head];
-        if (pool) { dq_head1 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n1--; }
-        else      { dq_head0 = (head + 1 == p.qcap) ? 0 : head + 1; dq_n0--; }
+        QEntry *ring = dq + (size_t)pool * p.qcap;
+        uint32_t src = head + pos; if (src >= p.qcap) src -= p.qcap;
+        const QEntry e = ring[src];
+        if (pos == 0) {
+            if (pool) dq_head1 = (head + 1 == p.qcap) ? 0 : head + 1;
+            else      dq_head0 = (head + 1 == p.qcap) ? 0 : head + 1;
+        } else {
+            __syncwarp();
+            ring_remove(ring, head, pool ? dq_n1 : dq_n0, pos);
+        }
+        if (pool) dq_n1--; else dq_n0--;
         place_job(pool, g, e.cls, job_P(e.pk), job_D(e.pk), e.t, true);
     }
 
@@ -790,13 +843,13 @@ struct Sim {
                 while (dq_n0 > 0) {
                     const uint32_t g = choose_server(WANT_SOLO);
                     if (g == NONE32) break;
-                    place_decode(0, g);
+                    place_decode(0, g, f_slig() ? select_in_pool(0) : 0u);
                     __syncwarp();
                 }
                 while (dq_n1 > 0) {
                     const uint32_t g = choose_server(WANT_MIX);
                     if (g == NONE32) break;
-                    place_decode(1, g);
+                    place_decode(1, g, f_slig() ? select_in_pool(1) : 0u);
                     __syncwarp();
                 }
             }
@@ -1563,7 +1616,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_ke
         s.t = 0.0;
         s.load_block(h.blk);
         s.dq_head0 = h.dq_head0; s.dq_head1 = h.dq_head1; s.dq_n0 = h.dq_n0; s.dq_n1 = h.dq_n1;
-        s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds;
+        s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds; s.sel_ord0 = h.sel_ord0; s.sel_ord1 = h.sel_ord1;
         s.n_touch = 0; s.touch_all = false; s.need_start = 0; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
         s.force_nonlocal = p.force_dispatch != 0 || h.force != 0;
@@ -1617,6 +1670,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_ke
             h.T_end = T_end; h.H_total = H_total; h.blk = s.blk;
             h.dq_head0 = s.dq_head0; h.dq_head1 = s.dq_head1; h.dq_n0 = s.dq_n0; h.dq_n1 = s.dq_n1;
             h.place_ord = s.place_ord; h.events = s.events; h.rounds = s.rounds; h.err = s.err;
+            h.sel_ord0 = s.sel_ord0; h.sel_ord1 = s.sel_ord1;
             h.done = finished ? 1u : 0u;
             h.force = s.force_nonlocal ? 1u : 0u;
             if (!finished) atomicAdd(p.not_done, 1u);

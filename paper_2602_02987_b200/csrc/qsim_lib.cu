@@ -95,7 +95,7 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
     if (cfg->C < 1 || cfg->C > 65535) return fail(QSIM_EINVAL, "C must be in 1..65535");
     if (cfg->nblk < 1) return fail(QSIM_EINVAL, "nblk must be >= 1");
     if (cfg->qcap < 1 || cfg->qcap > (1u << 24)) return fail(QSIM_EINVAL, "qcap must be in 1..2^24");
-    if (cfg->gate > 2 || cfg->router > 1 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
+    if (cfg->gate > 2 || cfg->router > 2 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
         return fail(QSIM_EINVAL, "enum out of range");
     if (cfg->nblk > 1 && !(cfg->block_len > 0.0 && std::isfinite(cfg->block_len)))
         return fail(QSIM_EINVAL, "block_len must be positive when nblk > 1");
@@ -115,7 +115,8 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
         if (tg[b].M > cfg->N) return fail(QSIM_EINVAL, "M must be <= N");
         for (uint32_t i = 0; i < cfg->I; ++i) {
             if (!std::isfinite(tg[b].xstar[i]) || tg[b].xstar[i] < 0.0 || !std::isfinite(tg[b].n_xstar[i]) ||
-                !std::isfinite(tg[b].n_qpstar[i]) || !(tg[b].p_solo[i] >= 0.0 && tg[b].p_solo[i] <= 1.0))
+                !std::isfinite(tg[b].n_qpstar[i]) || !(tg[b].p_solo[i] >= 0.0 && tg[b].p_solo[i] <= 1.0) ||
+                !(tg[b].w_solo[i] >= 0.0) || !std::isfinite(tg[b].w_solo[i]) || !(tg[b].w_mix[i] >= 0.0) || !std::isfinite(tg[b].w_mix[i]))
                 return fail(QSIM_EINVAL, "LP targets out of range");
         }
     }
@@ -163,6 +164,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
     for (uint32_t i = 0; i < c.I; ++i)
         if (cls[i].theta > 0.0) f |= F_ABANDON;
     if (c.router == QSIM_ROUTER_SLI) f |= F_SLI;
+    if (c.router == QSIM_ROUTER_SLI_GENERAL) f |= F_SLI | F_SLIG;
     if (coef[5] != 0.0) f |= F_KAPPA;
     if (c.hist) f |= F_HIST;
     if (c.nblk > 1) f |= F_BLOCKS;
@@ -209,7 +211,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
         if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
         // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits
         // (abandonment, KV slope, blocks) may be present without being used
-        constexpr uint32_t MODES = F_SLI | F_RANDOM | F_OCC | F_FCFS | F_HIST | F_SLOTS;
+        constexpr uint32_t MODES = F_SLI | F_SLIG | F_RANDOM | F_OCC | F_FCFS | F_HIST | F_SLOTS;
         if (feat == ~0u || (feat & MODES) != (v.feat & MODES) || (feat & ~v.feat) != 0) continue;
         const int extra = __builtin_popcount(v.feat & ~feat);
         if (extra < best_bits) { best = &v; best_bits = extra; }
@@ -265,7 +267,7 @@ void fill_blocks(BlockPar *blocks, const qsim_config &cfg, const double *rates, 
         bp.M = tg[b].M;
         for (uint32_t i = 0; i < cfg.I; ++i) {
             bp.xstar[i] = tg[b].xstar[i]; bp.nx[i] = tg[b].n_xstar[i]; bp.nq[i] = tg[b].n_qpstar[i];
-            bp.ps[i] = tg[b].p_solo[i]; bp.rate[i] = rates[(size_t)b * cfg.I + i];
+            bp.ps[i] = tg[b].p_solo[i]; bp.ws[i] = tg[b].w_solo[i]; bp.wm[i] = tg[b].w_mix[i]; bp.rate[i] = rates[(size_t)b * cfg.I + i];
         }
     }
 }
@@ -445,9 +447,11 @@ int qsim_set_targets(qsim_t *h, const qsim_targets *tg)
     bp.M = tg->M;
     for (uint32_t i = 0; i < h->cfg.I; ++i) {
         if (!std::isfinite(tg->xstar[i]) || tg->xstar[i] < 0.0 || !std::isfinite(tg->n_xstar[i]) || !std::isfinite(tg->n_qpstar[i]) ||
-            !(tg->p_solo[i] >= 0.0 && tg->p_solo[i] <= 1.0))
+            !(tg->p_solo[i] >= 0.0 && tg->p_solo[i] <= 1.0) || !(tg->w_solo[i] >= 0.0) || !std::isfinite(tg->w_solo[i]) ||
+            !(tg->w_mix[i] >= 0.0) || !std::isfinite(tg->w_mix[i]))
             return fail(QSIM_EINVAL, "LP targets out of range");
         bp.xstar[i] = tg->xstar[i]; bp.nx[i] = tg->n_xstar[i]; bp.nq[i] = tg->n_qpstar[i]; bp.ps[i] = tg->p_solo[i];
+        bp.ws[i] = tg->w_solo[i]; bp.wm[i] = tg->w_mix[i];
     }
     CUDA_TRY(cudaMemcpyAsync(h->d_blocks, &bp, sizeof bp, cudaMemcpyHostToDevice, h->stream));
     CUDA_TRY(cudaStreamSynchronize(h->stream));

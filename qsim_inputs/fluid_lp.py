@@ -122,6 +122,16 @@ class Plan:
         return np.clip(out, 0.0, 1.0)
 
 
+def pool_weights(plan: "Plan", mu_m, mu_s):
+    """Class-selection weights of the general SLI-aware router: varpi_m,i = mu_m y*_m,i / sum_j mu_m,j y*_m,j and
+    the same for the solo pool (0/0 := 0)."""
+    wm = mu_m * plan.ym
+    ws = mu_s * plan.ys
+    wm = wm / wm.sum() if wm.sum() > 0 else np.zeros_like(wm)
+    ws = ws / ws.sum() if ws.sum() > 0 else np.zeros_like(ws)
+    return ws, wm
+
+
 def solve_plan(lam, P, D, theta, B: int, C: int, tau_mix: float, tau_solo: float,
                c_p: float, c_d: float, separate: bool = False,
                qd_zero: bool = False,

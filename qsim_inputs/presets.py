@@ -53,7 +53,7 @@ def _plan_block(lam, Pm, Dm, theta, N, B, C, coeffs, prices, separate, nchunks=N
         start = (tm0, ts0)
     tau_mix, tau_solo, plan = lp.consistent_taus(coeffs, B, C, solve, start=start)
     _, mu_m, mu_s = lp.service_rates(Pm, Dm, C, tau_mix, tau_solo, **ck)
-    return plan, plan.M(N), plan.p_solo(mu_m, mu_s)
+    return plan, plan.M(N), plan.p_solo(mu_m, mu_s), lp.pool_weights(plan, mu_m, mu_s)
 
 
 def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, router, placement,
@@ -67,12 +67,14 @@ def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, 
     sli = sli or {}
     M = np.zeros(nblk, np.uint32)
     xs = np.zeros((nblk, I)); nx = np.zeros((nblk, I)); nq = np.zeros((nblk, I)); ps = np.zeros((nblk, I))
+    wso = np.zeros((nblk, I)); wmi = np.zeros((nblk, I))
     values, plans = [], []
     for b in range(nblk):
-        plan, Mb, p_solo = _plan_block(lam_blocks[b], Pm, Dm, theta, N, B, C, coeffs, prices,
+        plan, Mb, p_solo, (w_s, w_m) = _plan_block(lam_blocks[b], Pm, Dm, theta, N, B, C, coeffs, prices,
                                        pricing == PRICING_SEPARATE, nchunks=nchunks, **sli)
         M[b] = Mb
         xs[b] = plan.x; nx[b] = N * plan.x; nq[b] = N * plan.qp; ps[b] = p_solo
+        wso[b] = w_s; wmi[b] = w_m
         values.append(plan.value)
         plans.append(dict(x=plan.x.tolist(), ym=plan.ym.tolist(), ys=plan.ys.tolist(), qp=plan.qp.tolist(),
                           qd=plan.qd.tolist()))
@@ -88,7 +90,7 @@ def build(name, *, N, R, B, C, Pm, Dm, lam_blocks, theta, prices, coeffs, gate, 
         theta=theta.copy(), prio_rank=lp.priority_ranks(Pm, Dm),
         rates=np.ascontiguousarray(lam_blocks), lengths=lengths,
         prices=np.asarray(prices, float), coeffs=np.asarray(coeffs, float).copy(),
-        M=M, xstar=xs, n_xstar=nx, n_qpstar=nq, p_solo=ps,
+        M=M, xstar=xs, n_xstar=nx, n_qpstar=nq, p_solo=ps, w_solo=wso, w_mix=wmi,
         meta=dict(lp_value=values, plan=plans, Pm=list(map(float, Pm)), Dm=list(map(float, Dm)),
                   horizon_iters=int(horizon_iters), tau_ref=tau_ref(coeffs, B)),
     )

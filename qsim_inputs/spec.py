@@ -27,6 +27,7 @@ GATE_FCFS = 2        # oldest waiting request first, no class rule (ablation FG-
 # decode router
 ROUTER_SOLO_FIRST = 0      # single FCFS buffer, solo GPUs first (Section 4.1, "Downstream routing")
 ROUTER_SLI = 1             # randomized split with p_s,i, two buffers (Section 5.2)
+ROUTER_SLI_GENERAL = 2     # as ROUTER_SLI, plus class selection inside each pool by the weights varpi (EC, General SLI-aware Extension)
 # choice of GPU inside the eligible set
 PLACE_RANDOM = 0           # uniformly at random (paper)
 PLACE_LEAST_LOADED = 1     # fewest decodes, lowest index on ties
@@ -73,6 +74,8 @@ class SimInputs:
     n_xstar: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))       # [nblk, I]   n x*_i
     n_qpstar: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))      # [nblk, I]   n q*_p,i
     p_solo: np.ndarray = field(default_factory=lambda: np.zeros((0, 0)))        # [nblk, I]   p_s,i
+    w_solo: Optional[np.ndarray] = None    # [nblk, I] varpi_s,i  (class-selection weights of the general SLI router)
+    w_mix: Optional[np.ndarray] = None     # [nblk, I] varpi_m,i
     # optional injected arrivals replacing the Poisson source (same list for every replication):
     # times [K] ascending, and (class, P, D) [K, 3]
     inject_t: Optional[np.ndarray] = None
@@ -93,6 +96,11 @@ class SimInputs:
         assert self.M.shape == (nblk,)
         for a in (self.xstar, self.n_xstar, self.n_qpstar, self.p_solo):
             assert a.shape == (nblk, I)
+        if self.w_solo is None:
+            self.w_solo = np.zeros((nblk, I))
+        if self.w_mix is None:
+            self.w_mix = np.zeros((nblk, I))
+        assert self.w_solo.shape == (nblk, I) and self.w_mix.shape == (nblk, I)
         if self.length_mode == LENGTH_TABLE:
             assert self.lengths is not None and self.lengths.shape == (I, 2, LMAX)
             assert self.lengths.dtype == np.uint32

@@ -72,6 +72,20 @@ def test_fcfs_gate_ablation():
     check(presets.cfg1(R=4).with_(gate=GATE_FCFS), 1000)
 
 
+@pytest.mark.parametrize("placement", [PLACE_RANDOM, PLACE_LEAST_LOADED])
+def test_general_sli_router_class_selection(placement):
+    # both pools backlogged with two classes: selections are drawn, requests leave from inside the buffers;
+    # run in three pieces so that the selection ordinals cross launches
+    from qsim_inputs.spec import ROUTER_SLI_GENERAL
+    inp = presets.paper_instance(n=20, R=5, router=ROUTER_SLI_GENERAL, placement=placement)
+    inp = inp.with_(p_solo=np.array([[0.8, 0.8]]), w_solo=np.array([[0.25, 0.75]]), w_mix=np.array([[0.6, 0.4]]))
+    st = check(inp, 8000, chunks=[3000, 1, 4999])
+    assert st["abandoned_d"].sum() > 0 and st["Qd"].sum() > 0
+    # a cluster wide enough for the multi-warp instance, LP weights, one zero weight
+    inp = presets.paper_instance(n=700, R=2, router=ROUTER_SLI_GENERAL, placement=placement)
+    check(inp, 300)
+
+
 def test_cfg1_subset_lognormal_tables_priority_gate():
     inp = presets.cfg1(R=8)
     check(inp, 1500)

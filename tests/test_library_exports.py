@@ -33,7 +33,7 @@ def test_binding_struct_layouts_match_the_header_sizes():
     # sizes implied by the header's field lists (natural alignment)
     assert ctypes.sizeof(b.qsim_config) == 14 * 4 + 2 * 8 + 8
     assert ctypes.sizeof(b.qsim_class) == 24
-    assert ctypes.sizeof(b.qsim_targets) == 8 + 4 * 8 * 8
+    assert ctypes.sizeof(b.qsim_targets) == 8 + 6 * 8 * 8
     assert ctypes.sizeof(b.qsim_class_stats) == 14 * 8 + 6 * 4 + 7 * 8
     assert ctypes.sizeof(b.qsim_rep_stats) == 8 * ctypes.sizeof(b.qsim_class_stats) + 6 * 8
 
