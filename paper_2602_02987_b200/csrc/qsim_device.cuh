@@ -245,6 +245,11 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+// Copies are committed one group per copy, so a thread can wait for an older copy of its own and leave the
+// N groups it committed after it in flight.
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N_>
+__device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N_) : "memory"); }
 
 // 1 + #{j < LMAX-1 : thr[j] <= w} by binary search
 __device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, uint32_t w)
@@ -319,6 +324,7 @@ struct Sim {
     double *st_te;
     QEntry *pqh;
     uint32_t n_pend;
+    uint32_t rec_after;          // per lane: record copies committed since this lane's last queue-head copy
     QEntry *pq, *dq;
     uint32_t *hist;
     // replicated scalars
@@ -769,8 +775,13 @@ struct Sim {
 
     __device__ void admit(uint32_t i, uint32_t g)
     {
-        // the head of the class queue is kept in shared memory (copied there asynchronously after each pop)
-        cp_async_wait_all();
+        // the head of the class queue is kept in shared memory (copied there asynchronously after each pop);
+        // record copies of finished requests that this lane committed later stay in flight
+        if (lane == (int)i) {
+            if (rec_after == 1) cp_async_wait_group<1>();
+            else if (rec_after == 2) cp_async_wait_group<2>();
+            else cp_async_wait_group<0>();
+        }
         __syncwarp();
         const QEntry e = pqh[i];
         __syncwarp();
@@ -781,7 +792,7 @@ struct Sim {
             area_touch(c.aQp, c.pq_n, t);
             c.pq_n--;
             c.pq_head = (head + 1 == p.qcap) ? 0 : head + 1;
-            if (c.pq_n > 0) cp_async16(&pqh[i], &pq[(size_t)i * p.qcap + c.pq_head]);
+            if (c.pq_n > 0) { cp_async16(&pqh[i], &pq[(size_t)i * p.qcap + c.pq_head]); cp_async_commit(); rec_after = 0; }
             area_touch(c.aX, c.X, t);
             c.X++;
             c.admitted++;
@@ -799,24 +810,25 @@ struct Sim {
     // Called by the owner: a GPU with work that is between iterations starts one at time ts.  The batch
     // (prefill chunk, decodes) is frozen here for the whole iteration, and with it what its end will bring:
     // bit 14 of nact = some decode emits its last token, bit 15 = the prefill finishes.
-    __device__ __forceinline__ void start_at(uint32_t g, double ts)
+    // Straight-line: every field is read first and the stores are predicated on `act`, so that the calls for
+    // the rows of one lane overlap.  g is always inside the padded arrays.
+    __device__ __forceinline__ void start_at(uint32_t g, double ts, bool act = true)
     {
-        if (!(tnext[g] < dinf())) {
-            const uint32_t nd = ndec[g];
-            const uint32_t pj = pfjob[g];
-            if (nd > 0 || (pj >> 31)) {
-                uint32_t Kg = 0;
-                if (f_kappa()) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
-                const uint32_t rem = pfrem[g];
-                const uint32_t pc = (pj >> 31) ? min(p.C, rem) : 0u;
-                pfcur[g] = (uint16_t)pc;
-                uint32_t fl = (nfin[g] == it[g] + 1u) ? 0x4000u : 0u;
-                if (pc > 0 && pc == rem) fl |= 0x8000u;
-                nact[g] = (uint16_t)(nd | fl);
-                const double tau = iter_time(p, pc, nd, Kg, f_kappa());
-                taucur[g] = tau;
-                tnext[g] = __dadd_rn(ts, tau);
-            }
+        const unsigned long long tn = (unsigned long long)__double_as_longlong(tnext[g]);
+        const uint32_t nd = ndec[g], pj = pfjob[g], rem = pfrem[g], nf = nfin[g], it0 = it[g];
+        uint32_t Kg = 0;
+        if (f_kappa()) Kg = K[g] + Kpend[g];
+        const bool has_pf = (pj >> 31) != 0;
+        const uint32_t pc = has_pf ? min(p.C, rem) : 0u;
+        uint32_t fl = (nf == it0 + 1u) ? 0x4000u : 0u;
+        if (pc > 0 && pc == rem) fl |= 0x8000u;
+        const double tau = iter_time(p, pc, nd, Kg, f_kappa());
+        if (act && tn >= 0x7ff0000000000000ull && (nd > 0 || has_pf)) {
+            if (f_kappa()) { K[g] = Kg; Kpend[g] = 0; }
+            pfcur[g] = (uint16_t)pc;
+            nact[g] = (uint16_t)(nd | fl);
+            taucur[g] = tau;
+            tnext[g] = __dadd_rn(ts, tau);
         }
     }
     __device__ __forceinline__ void start_if_needed(uint32_t g) { start_at(g, t); }
@@ -874,7 +886,7 @@ struct Sim {
             // every owner starts its touched GPUs; different lanes work in parallel
 #pragma unroll
             for (uint32_t k = 0; k < (uint32_t)(SPL > 0 ? SPL : 1); ++k)
-                if (need_start & (1u << k)) start_if_needed((k << 5) + (uint32_t)lane);
+                start_at((k << 5) + (uint32_t)lane, t, ((need_start >> k) & 1u) != 0);
             need_start = 0;
         } else if (touch_all) {
             for (uint32_t k = 0; k < n_rows(); ++k) {
@@ -947,6 +959,8 @@ struct Sim {
                     if (hit) {
                         const uint32_t pos = n_pend + (uint32_t)__popc(hits & ((1u << lane) - 1u));
                         cp_async16(&st_rec[pos], &s_rec[(size_t)g * p.B + j]);
+                        cp_async_commit();
+                        rec_after++;
                         st_te[pos] = te;
                     }
                     n_pend += (uint32_t)__popc(hits);
@@ -1016,29 +1030,38 @@ struct Sim {
         const int owner = (int)(g & 31u);
         uint32_t flags = 0, itg = 0, nd = 0;
         bool recount_idle = false;
-        if (lane == owner) {
-            itg = it[g] + 1;
-            it[g] = itg;
-            const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
-            const double tau = taucur[g];
-            if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
-            else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
-            if (f_kappa()) K[g] = Kg + na;
-            tnext[g] = dinf();
-            nd = ndec[g];
-            if (nfin[g] == itg) flags |= 1u;
-            if (pc > 0) {
-                const uint32_t rem = pfrem[g] - pc;
-                pfrem[g] = rem;
-                if (rem == 0) flags |= 2u;
+        if (SPL > 0) {
+            // the round's passes have ended the iteration and retired its finished decodes; the frozen batch
+            // flags say what the end brought
+            const uint32_t na = nact[g];
+            flags = ((na >> 14) & 1u) | (((na >> 15) & 1u) << 1);
+        } else {
+            if (lane == owner) {
+                itg = it[g] + 1;
+                it[g] = itg;
+                const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
+                const double tau = taucur[g];
+                if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
+                else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
+                if (f_kappa()) K[g] = Kg + na;
+                tnext[g] = dinf();
+                nd = ndec[g];
+                if (nfin[g] == itg) flags |= 1u;
+                if (pc > 0) {
+                    const uint32_t rem = pfrem[g] - pc;
+                    pfrem[g] = rem;
+                    if (rem == 0) flags |= 2u;
+                }
+                pfcur[g] = 0;
             }
-            pfcur[g] = 0;
+            flags = __shfl_sync(FULL, flags, owner);
+            if (flags & 1u) {
+                itg = __shfl_sync(FULL, itg, owner);
+                nd = __shfl_sync(FULL, nd, owner);
+                retire_decodes(g, itg, nd, t);
+            }
         }
-        flags = __shfl_sync(FULL, flags, owner);
         if (flags & 1u) {
-            itg = __shfl_sync(FULL, itg, owner);
-            nd = __shfl_sync(FULL, nd, owner);
-            retire_decodes(g, itg, nd, t);
             drain_dirty = true;
             gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
             recount_idle = true;
@@ -1124,34 +1147,37 @@ struct Sim {
     // --- local end of an iteration (owner lane only) ----------------------------------------------------
     // The iteration of GPU g ends at te and nothing outside g depends on it.  Returns true when a decode
     // finished: the GPU then waits for retire_decodes before it starts its next iteration.
-    __device__ __forceinline__ bool local_end(uint32_t g, double te)
+    // evt: the end is the round's non-local event; the GPU is then not restarted here (the event's handler and
+    // the dispatch that follows may change its batch first).
+    __device__ __forceinline__ bool local_end(uint32_t g, double te, bool act = true, bool evt = false)
     {
-        const uint32_t itg = it[g] + 1u;
-        it[g] = itg;
-        const uint32_t na_raw = nact[g], pc = pfcur[g];
+        // straight-line: all fields are read first and the stores are predicated on `act` (see start_at)
+        const uint32_t it0 = it[g], na_raw = nact[g], pc = pfcur[g], nd = ndec[g], pj = pfjob[g], pr = pfrem[g], nf = nfin[g];
         const double tau = taucur[g];
-        if (f_kappa()) K[g] += na_raw & 0x3fffu;
-        uint32_t rem = 0;
-        if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); rem = pfrem[g] - pc; pfrem[g] = rem; }
-        else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
-        if (na_raw & 0x4000u) { pfcur[g] = 0; tnext[g] = dinf(); return true; }
-        // restart at te with what the GPU holds now (requests placed meanwhile join here)
-        const uint32_t nd = ndec[g];
-        const uint32_t pj = pfjob[g];
+        uint32_t K0 = 0, Kp = 0;
+        if (f_kappa()) { K0 = K[g]; Kp = Kpend[g]; }
+        const uint32_t itg = it0 + 1u;
+        const uint32_t rem = pr - pc;                       // prompt tokens left after this iteration's chunk
+        const bool retire = (na_raw & 0x4000u) != 0;        // a decode finished: the GPU waits for retire_decodes
         const bool has_pf = (pj >> 31) != 0;
-        if (nd == 0 && !has_pf) { pfcur[g] = 0; tnext[g] = dinf(); return false; }
-        if (has_pf && pc == 0) rem = pfrem[g];
-        uint32_t Kg = 0;
-        if (f_kappa()) { Kg = K[g] + Kpend[g]; K[g] = Kg; Kpend[g] = 0; }
+        const bool restart = !retire && !evt && (nd != 0 || has_pf);
+        // restart at te with what the GPU holds now (requests placed meanwhile join here)
+        const uint32_t Kend = K0 + (na_raw & 0x3fffu);
+        const uint32_t Kg = Kend + Kp;
         const uint32_t pc2 = has_pf ? min(p.C, rem) : 0u;
-        uint32_t fl = (nfin[g] == itg + 1u) ? 0x4000u : 0u;
+        uint32_t fl = (nf == itg + 1u) ? 0x4000u : 0u;
         if (pc2 > 0 && pc2 == rem) fl |= 0x8000u;
         const double tau2 = iter_time(p, pc2, nd, Kg, f_kappa());
-        pfcur[g] = (uint16_t)pc2;
-        nact[g] = (uint16_t)(nd | fl);
-        taucur[g] = tau2;
-        tnext[g] = __dadd_rn(te, tau2);
-        return false;
+        if (act) {
+            it[g] = itg;
+            if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] = rem; }
+            else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
+            if (f_kappa()) { K[g] = restart ? Kg : Kend; if (restart) Kpend[g] = 0; }
+            pfcur[g] = restart ? (uint16_t)pc2 : (uint16_t)0;
+            if (restart) { nact[g] = (uint16_t)(nd | fl); taucur[g] = tau2; }
+            tnext[g] = restart ? __dadd_rn(te, tau2) : dinf();
+        }
+        return act && retire;
     }
 
     // Class lanes of the master: add every warp's accounting of finished requests to the class records.
@@ -1305,14 +1331,16 @@ struct Sim {
             } else {
 #pragma unroll
                 for (uint32_t k = 0; k < rows; ++k) {
+                    // straight-line (INF is the identity of the minimum; padded GPUs never run)
                     const uint32_t g = (k << 5) + (uint32_t)lane;
                     const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-                    const bool loc = v < INF && is_local(g, buffered);
+                    const uint32_t na = nact[g], nd = ndec[g];
+                    const bool nl = force_nonlocal || (na & 0x8000u) != 0 ||
+                                    ((na & 0x4000u) != 0 && (buffered || (g < M && nd > p.B - 1)));
+                    const bool loc = v < INF && !nl;
                     if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
-                    if (v < INF) {
-                        tmin = min(tmin, v);
-                        if (!loc && v < bt) { bt = v; bs = SRC_SERVER + g; }
-                    }
+                    tmin = min(tmin, v);
+                    if (v < INF && nl && v < bt) { bt = v; bs = SRC_SERVER + g; }
                 }
                 // warp argmin of (time bits, source id) over non-local events; warp min over all pending times
                 warp_keys(bt, bs, tmin, tint, src, tmin_all);
@@ -1347,6 +1375,18 @@ struct Sim {
                     progressed = true;
                 }
             }
+            // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
+            // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
+            bool redo = sched_pending;
+            if (f_abandon() && lane < (int)p.I) {
+                const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
+                redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
+            }
+            // the non-local event happens in this round if it comes before anything a new iteration could bring
+            const bool any_redo = __any_sync(FULL, redo);
+            const bool do_event = !any_redo && tint < wt && tint <= tend_bits;
+            // with unrolled rows the event GPU's iteration ends in pass 1 and its decodes retire in pass 2
+            const uint32_t ev_g = (SPL > 0 && do_event && src >= SRC_SERVER) ? src - SRC_SERVER : NONE32;
             // pass 1: every lane ends the local iterations of its own GPUs (straight-line over the rows)
             uint32_t retire_rows = 0;
             if (SPL == 0) {
@@ -1364,10 +1404,10 @@ struct Sim {
                 for (uint32_t k = 0; k < rows; ++k) {
                     const uint32_t g = (k << 5) + (uint32_t)lane;
                     const unsigned long long v = vrow[k];
-                    if (lrow[k] && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
-                        if (local_end(g, __longlong_as_double((long long)v))) retire_rows |= 1u << k;
-                        progressed = true;
-                    }
+                    const bool evt = g == ev_g;
+                    const bool act = evt || (lrow[k] && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s)));
+                    if (local_end(g, __longlong_as_double((long long)v), act, evt)) retire_rows |= 1u << k;
+                    progressed = progressed || act;
                 }
             }
             if (SPL > 0) {
@@ -1383,21 +1423,16 @@ struct Sim {
                             const uint32_t gg = (k << 5) + (uint32_t)l;
                             const double te = __longlong_as_double((long long)__shfl_sync(FULL, vrow[k], l));
                             retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
-                            if (lane == l) start_at(gg, te);
                         }
                     }
+                    // the retired GPUs restart where their iteration ended (straight-line over the rows)
+#pragma unroll
+                    for (uint32_t k = 0; k < rows; ++k)
+                        start_at((k << 5) + (uint32_t)lane, __longlong_as_double((long long)vrow[k]),
+                                 ((retire_rows >> k) & 1u) != 0 && (k << 5) + (uint32_t)lane != ev_g);
                 }
             }
-            // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
-            // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
-            bool redo = sched_pending;
-            if (f_abandon() && lane < (int)p.I) {
-                const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
-                redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
-            }
-            if (__any_sync(FULL, redo)) continue;
-            // the non-local event, if it comes before anything a new iteration could bring
-            if (tint < wt && tint <= tend_bits) {
+            if (do_event) {
                 t = __longlong_as_double((long long)tint);
                 if (src >= SRC_SERVER) {
                     on_server(src - SRC_SERVER);
@@ -1411,7 +1446,7 @@ struct Sim {
                 if (err) return true;
                 dispatch();
                 force_nonlocal = false;
-            } else if (!__any_sync(FULL, progressed)) {
+            } else if (!any_redo && !__any_sync(FULL, progressed)) {
                 err = ERR_INTERNAL;     // a round that neither ended an iteration nor handled an event: never spin
                 return true;
             }
@@ -1509,6 +1544,7 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.cmd = reinterpret_cast<MwCmd *>(sm + L.off_cmd);
     s.res = reinterpret_cast<MwRes *>(sm + L.off_res);
     s.n_pend = 0;
+    s.rec_after = 0;
     s.ring_n = 0; s.ring_pos = 0; s.sched_pending = false; s.t0_pending = 0.0;
     const Params &p = s.p;
     const size_t r = s.rep;
