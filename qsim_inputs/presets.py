@@ -16,7 +16,7 @@ from . import fluid_lp as lp
 from .lengths import lognormal_tables, table_mean, table_mean_chunks
 from .spec import (GATE_OCCUPANCY, GATE_PRIORITY, LENGTH_FIXED, LENGTH_TABLE, PLACE_LEAST_LOADED,
                    PLACE_RANDOM, PRICING_BUNDLED, PRICING_SEPARATE, ROUTER_SLI, ROUTER_SOLO_FIRST,
-                   SimInputs)
+                   CtmcInputs, SimInputs)
 
 # alpha_m, beta, delta_m, alpha_s, delta_s, kappa
 # benchmark family: tau = 5 ms + 0.02 ms * prefill_tokens + 0.05 ms * decode_count
@@ -299,3 +299,40 @@ def trace_replay(n=10, R=2, T=90.0, seed=42, placement=PLACE_RANDOM, coeffs=COEF
                 seed=seed, qcap=4096)
     inp = inp.with_(inject_t=np.ascontiguousarray(ts, np.float64), inject_job=np.ascontiguousarray(jobs, np.uint32))
     return inp, Pm, Dm
+
+
+def ctmc_instance(n=50, R=8, router=ROUTER_SOLO_FIRST, gate=GATE_OCCUPANCY, B=16, C=256, seed=11,
+                  P=(300, 3000), D=(1000, 400), lam=(0.5, 0.5), theta=(0.1, 0.1), prices=(0.1, 0.2),
+                  separate=True, coeffs=COEFFS_PAPER) -> CtmcInputs:
+    """The exponential-service model of Section 2.3 on the paper's two-class synthetic instance (EC,
+    "Convergence Analysis"): rates from Eq. (4) with tau = tau_mix(C) and gamma = 1/tau_solo, targets
+    from the steady-state LP, M = ceil(n sum x*).  B and tau_solo as in `paper_instance`."""
+    P = np.asarray(P, float); D = np.asarray(D, float); lam = np.asarray(lam, float); theta = np.asarray(theta, float)
+    tau_mix, tau_solo = lp.nominal_taus(coeffs, B, C)
+    mu_p, mu_m, mu_s = lp.service_rates(P, D, C, tau_mix, tau_solo)
+    sli = dict(qd_zero=True) if router == ROUTER_SLI else {}
+    plan = lp.solve_plan(lam, P, D, theta, B, C, tau_mix, tau_solo, prices[0], prices[1], separate=separate, **sli)
+    I = len(P)
+    inp = CtmcInputs(
+        name=f"ctmc_n{n}", I=I, N=n, M=int(plan.M(n)), B=B, R=R, gate=gate, router=router,
+        qcap=max(256, _next_pow2(64.0 * math.sqrt(n))), seed=seed,
+        lam=lam.copy(), theta=theta.copy(), mu_p=np.asarray(mu_p, float), mu_m=np.asarray(mu_m, float),
+        mu_s=np.asarray(mu_s, float), P=P.copy(), D=D.copy(), prices=np.asarray(prices, float),
+        prio_rank=lp.priority_ranks(P, D), xstar=np.asarray(plan.x, float), n_xstar=n * np.asarray(plan.x, float),
+        n_qpstar=n * np.asarray(plan.qp, float), p_solo=np.asarray(plan.p_solo(mu_m, mu_s), float),
+        meta=dict(lp_value=float(plan.value), separate=bool(separate), tau_mix=tau_mix, tau_solo=tau_solo,
+                  plan=dict(x=plan.x.tolist(), ym=plan.ym.tolist(), ys=plan.ys.tolist(), qp=plan.qp.tolist(),
+                            qd=plan.qd.tolist())))
+    inp.validate()
+    return inp
+
+
+def ctmc_revenue_rate(inp: CtmcInputs, st: dict, separate=None) -> np.ndarray:
+    """Per-GPU revenue rate of every replication from the integer counters: bundled charging credits
+    c_p P_i + c_d D_i at decode completion (Eq. (21)-(22)); separate charging credits c_p P_i at prefill
+    completion and c_d D_i at decode completion (Eq. (23))."""
+    sep = inp.meta.get("separate", False) if separate is None else separate
+    done = (st["done_mixed"] + st["done_solo"]).astype(float)
+    pf = st["prefill_done"].astype(float) if sep else done
+    rev = (inp.prices[0] * inp.P * pf + inp.prices[1] * inp.D * done).sum(axis=1)
+    return rev / (inp.N * st["T_elapsed"])

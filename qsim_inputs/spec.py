@@ -134,3 +134,53 @@ CLASS_SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", 
 # Per-replication scalars.
 REP_COUNTERS = ("iters_mixed", "iters_solo", "events")      # uint64 [R]
 REP_SUMS = ("busy_mixed", "busy_solo", "T_elapsed")          # float64 [R]
+
+
+# ---------------------------------------------------------------------------------------------
+# Exponential-service (Markov chain) model of Section 2.3: plain data, no arithmetic.
+# ---------------------------------------------------------------------------------------------
+CTMC_COUNTERS = ("arrivals", "admitted", "prefill_done", "placed_mixed", "placed_solo", "done_mixed", "done_solo",
+                 "abandoned_p", "abandoned_d", "overflow_d")      # uint64 [R, I]
+CTMC_STATE = ("Qp", "X", "Qd", "Ym", "Ys")                       # uint32 [R, I] at the end time
+CTMC_AREAS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys")   # float64 [R, I] time integrals
+
+
+@dataclass
+class CtmcInputs:
+    """One instance of the exponential-service model: classes are described by rates, not lengths."""
+    name: str
+    I: int
+    N: int
+    M: int                      # mixed GPUs of the static partition
+    B: int
+    R: int
+    gate: int = GATE_OCCUPANCY  # GATE_OCCUPANCY or GATE_PRIORITY
+    router: int = ROUTER_SOLO_FIRST   # ROUTER_SOLO_FIRST or ROUTER_SLI
+    qcap: int = 4096            # capacity of each decode buffer (entries)
+    seed: int = 0
+    rep_offset: int = 0
+    lam: np.ndarray = field(default_factory=lambda: np.zeros(0))     # [I] per-GPU arrival rates lambda_i
+    theta: np.ndarray = field(default_factory=lambda: np.zeros(0))   # [I] patience rates
+    mu_p: np.ndarray = field(default_factory=lambda: np.zeros(0))    # [I] Eq. (4)
+    mu_m: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    mu_s: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    P: np.ndarray = field(default_factory=lambda: np.zeros(0))       # [I] token lengths, for revenue only
+    D: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    prices: np.ndarray = field(default_factory=lambda: np.zeros(2))  # (c_p, c_d)
+    prio_rank: np.ndarray = field(default_factory=lambda: np.zeros(0, np.uint32))
+    xstar: np.ndarray = field(default_factory=lambda: np.zeros(0))   # [I] x*_i
+    n_xstar: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    n_qpstar: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    p_solo: np.ndarray = field(default_factory=lambda: np.zeros(0))
+    meta: dict = field(default_factory=dict)
+
+    def with_(self, **kw) -> "CtmcInputs":
+        return replace(self, **kw)
+
+    def validate(self) -> None:
+        I = self.I
+        assert 1 <= I <= MAXI and self.N >= 1 and 0 <= self.M <= self.N and self.B >= 1 and self.R >= 1
+        assert self.gate in (GATE_OCCUPANCY, GATE_PRIORITY) and self.router in (ROUTER_SOLO_FIRST, ROUTER_SLI)
+        for a in (self.lam, self.theta, self.mu_p, self.mu_m, self.mu_s, self.P, self.D, self.xstar, self.n_xstar,
+                  self.n_qpstar, self.p_solo, self.prio_rank):
+            assert a.shape == (I,)
