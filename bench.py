@@ -153,6 +153,73 @@ def run_reference(args, workload):
     }))
 
 
+def run_ctmc(args):
+    """Second workload: the exponential-service model of Section 2.3 on the paper's two-class synthetic instance,
+    n = 1000 GPUs, SLI-aware router, 8192 replications per GPU; one step advances every replication by 10 s."""
+    import torch
+    import torch.distributed as dist
+    from paper_2602_02987_b200 import QSimCTMC
+    from paper_2602_02987_b200.sharding import shard
+    from qsim_inputs import presets
+    from qsim_inputs.spec import ROUTER_SLI
+    world = int(os.environ.get("WORLD_SIZE", "1")); rank = int(os.environ.get("RANK", "0")); local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the simulator has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    n, R, dT = 1000, 8192, 10.0
+    count, offset = shard(R * world, world, rank)
+    inp = presets.ctmc_instance(n=n, R=count, router=ROUTER_SLI).with_(rep_offset=offset)
+    sim = QSimCTMC(inp, device=f"cuda:{local}")
+    T = 0.0
+    for _ in range(max(args.warmup, 3)):
+        T += dT; sim.run_until(T)
+    ev0 = int(sim.stats()["events"].sum()); l0 = sim.launches
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        T += dT; sim.run_until(T)
+    b.record()
+    torch.cuda.synchronize()
+    my = torch.tensor([a.elapsed_time(b), float(int(sim.stats()["events"].sum()) - ev0), float(sim.launches - l0)], dtype=torch.float64, device="cuda")
+    tmax = my[:1].clone()
+    if world > 1:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX); dist.all_reduce(my[1:], op=dist.ReduceOp.SUM)
+    if rank == 0:
+        out = {"metric": "simulated jumps of the exponential-service model/sec", "value": float(my[1]) / (float(tmax[0]) * 1e-3),
+               "unit": "jumps/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+               "ms_per_step": float(tmax[0]) / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+               "dtype": "f64", "data": "synthetic", "gpu_launches": int(my[2]),
+               "config": {"workload": f"exponential-service model, paper synthetic instance, n={n}, SLI-aware router, "
+                                      f"{R} replications per GPU, {dT} s of simulated time per step"}}
+        if not args.no_cpu_baseline and world == 1:
+            from oracle import run_ctmc_oracle
+            cores = os.cpu_count() or 1
+            done = [0] * cores
+            T_cpu = 10_000.0      # about 10 s of work for the host cores
+
+            def work(k):
+                st = run_ctmc_oracle(inp.with_(R=1, rep_offset=k), T_cpu)
+                done[k] = int(st["events"].sum())
+            t0 = time.perf_counter()
+            th = [threading.Thread(target=work, args=(k,)) for k in range(cores)]
+            for t in th:
+                t.start()
+            for t in th:
+                t.join()
+            dt = time.perf_counter() - t0
+            out["cpu_baseline"] = {"value": sum(done) / dt, "unit": "jumps/s", "cores": cores, "kind": "oracle",
+                                   "sample": f"{cores} replications x {T_cpu:.0f} s of simulated time, one per thread, {dt:.1f} s"}
+        print(json.dumps(out))
+    sim.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -163,7 +230,12 @@ def main():
     ap.add_argument("--reps", type=int, default=R_PER_GPU, help="replications per GPU")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "ctmc"],
+                    help="cfg1: the iteration-level benchmark (default); ctmc: the exponential-service model, reported in jumps/s")
     args = ap.parse_args()
+    if args.workload == "ctmc":
+        run_ctmc(args)
+        return
     workload = (f"cfg1: 2 lognormal classes, N=64 GPUs, B=128, C=256, separate pricing, priority gate, solo-first "
                 f"router, least-loaded placement, R={args.reps} replications per GPU, {args.horizon} iterations "
                 f"of horizon per step")
@@ -280,7 +352,7 @@ def main():
             out["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:
             cores = os.cpu_count() or 1
-            h_s = 3000
+            h_s = 50_000       # about 10 s of work for the host cores
             v, it_s, dt = oracle_throughput(inp, h_s, 2 * cores, cores)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                    "sample": f"{2 * cores} replications x {h_s} iterations of horizon of cfg1, one per thread, {dt:.1f} s"}

@@ -248,6 +248,63 @@ int qsim_layout_info(const qsim_t *h, uint64_t out[4]);
 /* Kernel launches issued by this handle so far (for accounting in benchmarks). */
 int qsim_launch_count(const qsim_t *h, uint64_t *launches);
 
+/*
+ * Exponential-service model [Section 2.3].  The paper's analysis models prefill, mixed decode and solo decode
+ * service times as independent exponentials with the rates of Eq. (4), mu_p,i = C/(P_i tau), mu_m,i = 1/(D_i tau),
+ * mu_s,i = gamma/D_i; arrivals are Poisson of rate n lambda_i and waiting requests have exponential patience
+ * theta_i in the prefill queue and in the decode buffer, all driven by unit-rate Poisson processes on the
+ * integrated intensities of Eq. (7)-(9).  The policy is the static partition with M mixed GPUs, the occupancy or
+ * priority gate and the solo-first or SLI-aware router [Sections 4.1, 5.1.1, 5.2].  Requests of a class are
+ * exchangeable, so a replication's state is (Q_p,i, X_i, Q_d,i, Y_m,i, Y_s,i) and the class order of the decode
+ * buffers, with the capacities the optimality proof uses: sum_i X_i <= M, sum_i Y_m,i <= M (B-1),
+ * sum_i Y_s,i <= (N-M) B.  These entry points keep no handle: the caller's device workspace holds all state.
+ */
+typedef struct {
+    uint32_t size;             /* sizeof(qsim_ctmc_config) */
+    uint32_t I, N, M, B, R;    /* classes, GPUs, mixed GPUs, decode cap per GPU, replications */
+    uint32_t qcap;             /* capacity (requests) of each decode buffer; a finished prefill that finds it full is dropped and counted */
+    uint32_t gate;             /* QSIM_GATE_OCCUPANCY or QSIM_GATE_PRIORITY */
+    uint32_t router;           /* QSIM_ROUTER_SOLO_FIRST or QSIM_ROUTER_SLI */
+    uint32_t reserved;
+    uint64_t seed, rep_offset; /* Philox key; global index of replication 0 */
+} qsim_ctmc_config;
+
+typedef struct {
+    double lambda, theta;                       /* per-GPU arrival rate, patience rate */
+    double mu_p, mu_m, mu_s;                    /* Eq. (4) */
+    double xstar, n_xstar, n_qpstar, p_solo;    /* x*_i, n x*_i, n q*_p,i, p_s,i as in qsim_targets */
+    uint32_t prio_rank, reserved;               /* 0 = admitted first by QSIM_GATE_PRIORITY */
+} qsim_ctmc_class;
+
+typedef struct {
+    /* per class: A, U_p, S_p, U_dm, U_ds, S_dm, S_ds, B_p, B_d, finished prefills dropped at a full buffer */
+    uint64_t cnt[QSIM_MAXI][10];
+    uint32_t state[QSIM_MAXI][5];   /* Q_p, X, Q_d, Y_m, Y_s at the end time */
+    uint32_t reserved[QSIM_MAXI];
+    double area[QSIM_MAXI][5];      /* time integrals of the same five counts over [0, T_elapsed] */
+    uint64_t events;                /* jumps processed */
+    double T_elapsed;               /* end time reached */
+} qsim_ctmc_rep_stats;
+
+/* Bytes of device memory the three calls below need for this configuration. */
+int qsim_ctmc_workspace_bytes(const qsim_ctmc_config *cfg, size_t *bytes);
+
+/* Empty system at t = 0 in [device] dev_workspace (256-byte aligned, at least qsim_ctmc_workspace_bytes; owned by
+ * the caller); [host] cfg, classes[I].  One asynchronous launch on cuda_stream (a cudaStream_t, NULL = default). */
+int qsim_ctmc_init(const qsim_ctmc_config *cfg, const qsim_ctmc_class *classes, void *dev_workspace, size_t bytes,
+                   void *cuda_stream);
+
+/* Process every jump with t <= T_end (seconds; T_end must not decrease between calls) in all R replications,
+ * with the same cfg and classes as qsim_ctmc_init.  Returns after the stream has finished; launches (may be NULL)
+ * receives the number of kernel launches it took. */
+int qsim_ctmc_run_until(const qsim_ctmc_config *cfg, const qsim_ctmc_class *classes, void *dev_workspace, size_t bytes,
+                        void *cuda_stream, double T_end, uint64_t *launches);
+
+/* Copy the statistics of all replications to [host] per_rep[R]; time integrals are closed at the end time.
+ * Synchronises the stream.  QSIM_EOVERFLOW if a replication stopped on an internal error. */
+int qsim_ctmc_stats(const qsim_ctmc_config *cfg, const void *dev_workspace, size_t bytes, void *cuda_stream,
+                    qsim_ctmc_rep_stats *per_rep);
+
 int qsim_destroy(qsim_t *h);
 
 const char *qsim_last_error(void);

@@ -19,7 +19,8 @@ _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_
 EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_run_until", "qsim_set_injected",
            "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
-           "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error")
+           "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error",
+           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats")
 
 
 class QSimError(RuntimeError):
@@ -54,6 +55,26 @@ class qsim_rep_stats(C.Structure):
                 ("T_elapsed", C.c_double)]
 
 
+class qsim_ctmc_config(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in ("size", "I", "N", "M", "B", "R", "qcap", "gate", "router", "reserved")] + \
+               [("seed", C.c_uint64), ("rep_offset", C.c_uint64)]
+
+
+class qsim_ctmc_class(C.Structure):
+    _fields_ = [(n, C.c_double) for n in ("lam", "theta", "mu_p", "mu_m", "mu_s", "xstar", "n_xstar", "n_qpstar",
+                                          "p_solo")] + [("prio_rank", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+_CTMC_COUNTERS = ("arrivals", "admitted", "prefill_done", "placed_mixed", "placed_solo", "done_mixed", "done_solo",
+                  "abandoned_p", "abandoned_d", "overflow_d")
+_CTMC_AREAS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys")
+
+
+class qsim_ctmc_rep_stats(C.Structure):
+    _fields_ = [("cnt", (C.c_uint64 * 10) * MAXI), ("state", (C.c_uint32 * 5) * MAXI), ("reserved", C.c_uint32 * MAXI),
+                ("area", (C.c_double * 5) * MAXI), ("events", C.c_uint64), ("T_elapsed", C.c_double)]
+
+
 _lib = None
 
 
@@ -78,6 +99,11 @@ def load_library():
         L.qsim_sync.argtypes = [vp]
         L.qsim_stats.argtypes = [vp, vp, vp, vp, vp]
         L.qsim_reset_stats.argtypes = [vp]
+        L.qsim_ctmc_workspace_bytes.argtypes = [C.POINTER(qsim_ctmc_config), C.POINTER(C.c_size_t)]
+        L.qsim_ctmc_init.argtypes = [C.POINTER(qsim_ctmc_config), C.POINTER(qsim_ctmc_class), vp, C.c_size_t, vp]
+        L.qsim_ctmc_run_until.argtypes = [C.POINTER(qsim_ctmc_config), C.POINTER(qsim_ctmc_class), vp, C.c_size_t, vp,
+                                          C.c_double, C.POINTER(C.c_uint64)]
+        L.qsim_ctmc_stats.argtypes = [C.POINTER(qsim_ctmc_config), vp, C.c_size_t, vp, vp]
         L.qsim_revenue.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.qsim_server_state.argtypes = [vp, C.c_uint32, vp, vp, vp, vp]
         L.qsim_simulate.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
@@ -290,3 +316,70 @@ def simulate_static(inp, horizon_iters: int, stream=None) -> dict:
     out = _unpack(per, inp.R, inp.I)
     out["_totals"] = _unpack((tot,), 1, inp.I)
     return out
+
+
+class QSimCTMC:
+    """The exponential-service model (qsim_ctmc_* of include/qsim.h) on a CtmcInputs; the workspace is a torch tensor."""
+
+    def __init__(self, inp, device="cuda:0", stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise QSimError("no CUDA device: the simulator has no CPU path")
+        self.L = load_library()
+        self.inp = inp
+        self.device = torch.device(device)
+        self.cfg = qsim_ctmc_config(size=C.sizeof(qsim_ctmc_config), I=inp.I, N=inp.N, M=inp.M, B=inp.B, R=inp.R,
+                                    qcap=inp.qcap, gate=inp.gate, router=inp.router, reserved=0, seed=inp.seed,
+                                    rep_offset=inp.rep_offset)
+        self.classes = (qsim_ctmc_class * inp.I)()
+        for i in range(inp.I):
+            self.classes[i] = qsim_ctmc_class(
+                lam=float(inp.lam[i]), theta=float(inp.theta[i]), mu_p=float(inp.mu_p[i]), mu_m=float(inp.mu_m[i]),
+                mu_s=float(inp.mu_s[i]), xstar=float(inp.xstar[i]), n_xstar=float(inp.n_xstar[i]),
+                n_qpstar=float(inp.n_qpstar[i]), p_solo=float(inp.p_solo[i]), prio_rank=int(inp.prio_rank[i]), reserved=0)
+        nbytes = C.c_size_t()
+        _check(self.L.qsim_ctmc_workspace_bytes(C.byref(self.cfg), C.byref(nbytes)))
+        self.nbytes = nbytes.value
+        with torch.cuda.device(self.device):
+            self.ws = torch.empty(self.nbytes + 256, dtype=torch.uint8, device=self.device)
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            self.ptr = (self.ws.data_ptr() + 255) & ~255
+            _check(self.L.qsim_ctmc_init(C.byref(self.cfg), self.classes, C.c_void_p(self.ptr), self.nbytes,
+                                         C.c_void_p(self.stream.cuda_stream)))
+        self.launches = 1
+
+    def run_until(self, T_end: float) -> None:
+        import torch
+        n = C.c_uint64()
+        with torch.cuda.device(self.device):
+            _check(self.L.qsim_ctmc_run_until(C.byref(self.cfg), self.classes, C.c_void_p(self.ptr), self.nbytes,
+                                              C.c_void_p(self.stream.cuda_stream), float(T_end), C.byref(n)))
+        self.launches += n.value
+
+    def stats(self) -> dict:
+        import torch
+        R, I = self.inp.R, self.inp.I
+        per = (qsim_ctmc_rep_stats * R)()
+        with torch.cuda.device(self.device):
+            _check(self.L.qsim_ctmc_stats(C.byref(self.cfg), C.c_void_p(self.ptr), self.nbytes,
+                                          C.c_void_p(self.stream.cuda_stream), per))
+        raw = np.frombuffer(per, dtype=np.uint8).reshape(R, C.sizeof(qsim_ctmc_rep_stats))
+        o_state = 10 * 8 * MAXI
+        o_area = o_state + 5 * 4 * MAXI + 4 * MAXI
+        cnt = raw[:, :o_state].copy().view(np.uint64).reshape(R, MAXI, 10)
+        state = raw[:, o_state:o_state + 5 * 4 * MAXI].copy().view(np.uint32).reshape(R, MAXI, 5)
+        area = raw[:, o_area:o_area + 5 * 8 * MAXI].copy().view(np.float64).reshape(R, MAXI, 5)
+        tail = raw[:, o_area + 5 * 8 * MAXI:].copy()
+        out = {}
+        for k, n in enumerate(_CTMC_COUNTERS):
+            out[n] = np.ascontiguousarray(cnt[:, :I, k])
+        for k, n in enumerate(_STATE):
+            out[n] = np.ascontiguousarray(state[:, :I, k])
+        for k, n in enumerate(_CTMC_AREAS):
+            out[n] = np.ascontiguousarray(area[:, :I, k])
+        out["events"] = tail[:, :8].copy().view(np.uint64).reshape(R)
+        out["T_elapsed"] = tail[:, 8:16].copy().view(np.float64).reshape(R)
+        return out
+
+    def close(self) -> None:
+        self.ws = None

@@ -458,11 +458,12 @@ struct Sim {
 
     __device__ uint32_t count_idle_pf()
     {
+        // per-lane count over the lane's rows (branch-free), one warp-wide sum
         uint32_t cnt = 0;
-#pragma unroll
+#pragma unroll 4
         for (uint32_t k = 0; k < n_rows(); ++k)
-            cnt += (uint32_t)__popc(__ballot_sync(FULL, eligible((k << 5) + (uint32_t)lane, WANT_PREFILL)));
-        return cnt;
+            cnt += eligible((k << 5) + (uint32_t)lane, WANT_PREFILL) ? 1u : 0u;
+        return __reduce_add_sync(FULL, cnt);
     }
 
     // --- abandonment ---------------------------------------------------------------------------
@@ -550,13 +551,14 @@ struct Sim {
     // --- GPU choice ----------------------------------------------------------------------------
     __device__ __forceinline__ bool eligible(uint32_t g, int want) const
     {
-        if (g >= p.N) return false;
+        // g is always inside the padded arrays; every field is read first so that calls over rows overlap
         const uint32_t nd = ndec[g];
         const bool pf = (pfjob[g] >> 31) != 0;
-        const uint32_t cap = (g < M || pf) ? p.B - 1 : p.B;   // a mixed GPU keeps one slot for prefill
-        if (want == WANT_SOLO) return g >= M && nd < cap;
-        if (want == WANT_MIX) return g < M && nd < cap;
-        return g < M && !pf && nd <= p.B - 1;
+        const bool mix = g < M;
+        const uint32_t cap = (mix || pf) ? p.B - 1 : p.B;   // a mixed GPU keeps one slot for prefill
+        const bool ok = want == WANT_PREFILL ? (mix && !pf && nd <= p.B - 1)
+                                             : ((want == WANT_MIX) == mix && nd < cap);
+        return ok && g < p.N;
     }
 
     // uniformly at random among the eligible GPUs (k-th in index order) or least loaded, lowest index
@@ -564,15 +566,14 @@ struct Sim {
     __device__ __forceinline__ uint32_t choose_solo_first()
     {
         uint32_t best = NONE32;
-#pragma unroll
+#pragma unroll 4
         for (uint32_t k = 0; k < n_rows(); ++k) {
             const uint32_t g = (k << 5) + (uint32_t)lane;
-            if (g < p.N) {
-                const uint32_t nd = ndec[g];
-                const bool mix = g < M;
-                const uint32_t cap = (mix || (pfjob[g] >> 31)) ? p.B - 1 : p.B;
-                if (nd < cap) best = min(best, (mix ? 0x40000000u : 0u) | (nd << 16) | g);
-            }
+            const uint32_t nd = ndec[g];
+            const bool mix = g < M;
+            const uint32_t cap = (mix || (pfjob[g] >> 31)) ? p.B - 1 : p.B;
+            const uint32_t key = (mix ? 0x40000000u : 0u) | (nd << 16) | g;
+            best = min(best, (nd < cap && g < p.N) ? key : NONE32);
         }
         best = __reduce_min_sync(FULL, best);
         return best == NONE32 ? NONE32 : (best & 0xffffu);
@@ -583,10 +584,10 @@ struct Sim {
         const uint32_t rows = n_rows();
         if (!f_random()) {
             uint32_t best = NONE32;
-#pragma unroll
+#pragma unroll 4
             for (uint32_t k = 0; k < rows; ++k) {
                 const uint32_t g = (k << 5) + (uint32_t)lane;
-                if (eligible(g, want)) best = min(best, ((uint32_t)ndec[g] << 16) | g);
+                best = min(best, eligible(g, want) ? (((uint32_t)ndec[g] << 16) | g) : NONE32);
             }
             best = __reduce_min_sync(FULL, best);
             return best == NONE32 ? NONE32 : (best & 0xffffu);
@@ -1201,13 +1202,16 @@ struct Sim {
     __device__ void scan_share(bool buffered, unsigned long long &bt, uint32_t &bs, unsigned long long &tmin)
     {
         const unsigned long long INF = 0x7ff0000000000000ull;
+#pragma unroll 4
         for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
+            // straight-line (INF is the identity of the minimum; padded GPUs never run)
             const uint32_t g = (k << 5) + (uint32_t)lane;
             const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-            if (v < INF) {
-                tmin = min(tmin, v);
-                if (!is_local(g, buffered) && v < bt) { bt = v; bs = SRC_SERVER + g; }
-            }
+            const uint32_t na = nact[g], nd = ndec[g];
+            const bool nl = force_nonlocal || (na & 0x8000u) != 0 ||
+                            ((na & 0x4000u) != 0 && (buffered || (g < M && nd > p.B - 1)));
+            tmin = min(tmin, v);
+            if (v < INF && nl && v < bt) { bt = v; bs = SRC_SERVER + g; }
         }
     }
 

@@ -763,3 +763,5 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     h.bound = false;
     return rc;
 }
+
+#include "qsim_ctmc.cuh"

@@ -1,0 +1,74 @@
+"""GPU parity of the exponential-service model (qsim_ctmc_* through the C ABI) against its CPU oracle: integer
+counters and end state bit-exact, time integrals within 1e-9 relative (clocks are bit-identical by construction)."""
+import numpy as np
+import pytest
+
+from qsim_inputs import presets
+from qsim_inputs.spec import CTMC_AREAS, CTMC_COUNTERS, CTMC_STATE, GATE_PRIORITY, ROUTER_SLI, ROUTER_SOLO_FIRST
+
+pytestmark = pytest.mark.gpu
+RTOL = 1e-9
+
+
+def compare(gpu, ref, what):
+    for k in CTMC_COUNTERS + CTMC_STATE + ("events",):
+        assert np.array_equal(gpu[k], ref[k]), f"{what}: {k} differs at {np.argwhere(gpu[k] != ref[k])[:4].tolist()}"
+    for k in CTMC_AREAS + ("T_elapsed",):
+        assert np.allclose(gpu[k], ref[k], rtol=RTOL, atol=1e-300), f"{what}: {k}"
+
+
+def gpu_run(inp, times):
+    from paper_2602_02987_b200 import QSimCTMC
+    sim = QSimCTMC(inp, device="cuda:0")
+    for T in times:
+        sim.run_until(T)
+    st = sim.stats()
+    sim.close()
+    return st
+
+
+@pytest.mark.parametrize("router,gate,theta,lam", [
+    (ROUTER_SOLO_FIRST, 0, (0.1, 0.1), (0.5, 0.5)),        # the paper's synthetic instance
+    (ROUTER_SLI, 0, (0.1, 0.1), (0.5, 0.5)),               # randomized router, two decode buffers
+    (ROUTER_SOLO_FIRST, GATE_PRIORITY, (0.0, 0.3), (0.8, 0.8)),   # overload: buffers fill, one patient class, drops at a full buffer
+    (ROUTER_SLI, GATE_PRIORITY, (0.3, 0.3), (0.9, 0.7)),
+])
+def test_ctmc_parity_element_by_element(router, gate, theta, lam):
+    from oracle import run_ctmc_oracle
+    inp = presets.ctmc_instance(n=24, R=70, router=router, gate=gate, theta=theta, lam=lam)     # 70: two blocks, ragged tail
+    ref = run_ctmc_oracle(inp, 120.0)
+    compare(gpu_run(inp, [120.0]), ref, "one call")
+    compare(gpu_run(inp, [7.5, 7.5, 60.0, 120.0]), ref, "resumed")
+    assert ref["abandoned_d"].sum() > 0 or min(theta) == 0.0
+
+
+def test_ctmc_replication_keyed_and_large_cluster():
+    from oracle import run_ctmc_oracle
+    inp = presets.ctmc_instance(n=400, R=1024, router=ROUTER_SLI)
+    gpu = gpu_run(inp, [30.0])
+    # sampled replications against the oracle (the Philox counter holds the global replication index)
+    for r in (0, 517, 1023):
+        ref = run_ctmc_oracle(inp.with_(rep_offset=r, R=1), 30.0)
+        for k in CTMC_COUNTERS + CTMC_STATE + ("events",):
+            assert np.array_equal(gpu[k][r:r + 1], ref[k]), (r, k)
+        for k in CTMC_AREAS:
+            assert np.allclose(gpu[k][r:r + 1], ref[k], rtol=RTOL, atol=1e-300), (r, k)
+    # flow balance Eq. (15)-(20) on every replication
+    g = lambda k: gpu[k].astype(np.int64)
+    assert np.array_equal(g("Qp"), g("arrivals") - g("admitted") - g("abandoned_p"))
+    assert np.array_equal(g("X"), g("admitted") - g("prefill_done"))
+    assert np.array_equal(g("Qd"), g("prefill_done") - g("placed_mixed") - g("placed_solo") - g("abandoned_d") - g("overflow_d"))
+    assert np.array_equal(g("Ym") + g("Ys"), g("placed_mixed") + g("placed_solo") - g("done_mixed") - g("done_solo"))
+
+
+def test_ctmc_eight_classes_and_argument_errors():
+    from oracle import run_ctmc_oracle
+    from paper_2602_02987_b200 import QSimCTMC, QSimError
+    rng = np.random.default_rng(5)
+    P = tuple(int(v) for v in rng.integers(200, 3000, 8)); D = tuple(int(v) for v in rng.integers(200, 3000, 8))
+    inp = presets.ctmc_instance(n=16, R=33, P=P, D=D, lam=(0.12,) * 8, theta=(0.1,) * 8, router=ROUTER_SLI)
+    compare(gpu_run(inp, [60.0]), run_ctmc_oracle(inp, 60.0), "eight classes")
+    with pytest.raises(QSimError):
+        QSimCTMC(inp.with_(M=inp.N + 1))
+    with pytest.raises(QSimError):
+        QSimCTMC(inp.with_(gate=2))
