@@ -152,7 +152,12 @@ const std::vector<RunVariant> &run_variants()
         add_variants<2>(v);
         add_variants<4>(v);
         v.push_back({0, F_GENERIC, qsim_run_kernel<0, F_GENERIC>});
-        v.push_back({-1, F_GENERIC | F_MW, qsim_run_kernel<0, F_GENERIC | F_MW>});     // several warps per replication
+        // several warps per replication (large clusters): instances for the occupancy gate with abandonment under
+        // the solo-first and (with histograms) the SLI-aware router, the priority gate with blocks and histograms, and the generic one
+        v.push_back({-1, F_MW | F_OCC | F_ABANDON, qsim_run_kernel<0, F_MW | F_OCC | F_ABANDON>});
+        v.push_back({-1, F_MW | F_OCC | F_ABANDON | F_SLI | F_HIST, qsim_run_kernel<0, F_MW | F_OCC | F_ABANDON | F_SLI | F_HIST>});
+        v.push_back({-1, F_MW | F_ABANDON | F_BLOCKS | F_HIST, qsim_run_kernel<0, F_MW | F_ABANDON | F_BLOCKS | F_HIST>});
+        v.push_back({-1, F_GENERIC | F_MW, qsim_run_kernel<0, F_GENERIC | F_MW>});
         return v;
     }();
     return table;
@@ -176,7 +181,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
 
 // Large clusters: per-replication shared memory allows only a few blocks per SM, so each replication gets
 // several warps (master + helpers) that share the per-GPU scans.  QSIM_WARPS overrides the choice (1 = off).
-void choose_multiwarp(uint32_t N, Params &p, RunKernel &fn, uint32_t &nwarps)
+void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
     uint32_t W = rows >= 64 ? 16u : (rows >= 16 ? 4u : 1u);
@@ -185,8 +190,20 @@ void choose_multiwarp(uint32_t N, Params &p, RunKernel &fn, uint32_t &nwarps)
         if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
     }
     if (W <= 1 || rows < 2) return;
-    for (const RunVariant &v : run_variants())
-        if (v.spl < 0) { fn = v.fn; break; }
+    const char *force = std::getenv("QSIM_KERNEL");
+    const bool generic_only = force && std::strcmp(force, "generic") == 0;
+    // mode bits must match exactly, capability bits may be present unused (as in pick_run_kernel)
+    constexpr uint32_t MODES = F_SLI | F_SLIG | F_RANDOM | F_OCC | F_FCFS | F_HIST;
+    const RunVariant *best = nullptr;
+    int best_bits = 99;
+    for (const RunVariant &v : run_variants()) {
+        if (v.spl >= 0) continue;
+        if (v.feat & F_GENERIC) { if (!best) best = &v; continue; }
+        if (generic_only || (feat & MODES) != (v.feat & MODES) || (feat & ~(v.feat | F_SLOTS)) != 0) continue;
+        const int extra = __builtin_popcount(v.feat & ~feat & ~F_MW);
+        if (extra < best_bits) { best = &v; best_bits = extra; }
+    }
+    fn = best->fn;
     nwarps = W;
     p.Npad = rows * 32u;
     p.slots_smem = 0;       // helpers retire through the global slot lists
@@ -250,7 +267,7 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     if (p.slots_smem) v = pick_run_kernel(cfg.N, feat | F_SLOTS);
     h.run_fn = v.fn;
     h.nwarps = 1;
-    choose_multiwarp(cfg.N, p, h.run_fn, h.nwarps);
+    choose_multiwarp(cfg.N, feat, p, h.run_fn, h.nwarps);
     h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa);
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u)
@@ -428,11 +445,12 @@ int qsim_set_injected(qsim_t *h, const double *t, const uint32_t *job, uint64_t 
     h->par.n_inject = (uint32_t)n;
     // the trace source lives in the run-time-configured instance
     RunVariant v = pick_run_kernel(h->cfg.N, ~0u);
-    if (h->nwarps == 1) {
-        h->run_fn = v.fn;
-        if (h->lay.total > 48u * 1024u)
-            CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void *>(h->run_fn), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total));
-    }
+    if (h->nwarps > 1)
+        for (const RunVariant &mw : run_variants())
+            if (mw.spl < 0 && (mw.feat & F_GENERIC)) v = mw;
+    h->run_fn = v.fn;
+    if (h->lay.total > 48u * 1024u)
+        CUDA_TRY(cudaFuncSetAttribute(reinterpret_cast<const void *>(h->run_fn), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h->lay.total));
     return QSIM_OK;
 }
 

@@ -111,6 +111,23 @@ def test_cfg4_subset_sli_router_constrained_targets():
         check(inp, 1200 if N == 16 else 500)
 
 
+def test_multi_warp_instances_large_clusters():
+    # N >= 512 runs several warps per replication; each specialised instance and the generic one against the oracle
+    import os
+    inp = presets.cfg3(N=512, R=2, block_len=0.25)          # priority gate, blocks, histograms
+    H = inp.meta["horizon_iters"]
+    st = check(inp, H)
+    assert st["hist_tpot"].sum() == (st["done_mixed"] + st["done_solo"]).sum()
+    inp4 = presets.cfg4(N=512, R=2)                          # occupancy gate, SLI router, histograms
+    g = check(inp4, 300)
+    os.environ["QSIM_KERNEL"] = "generic"
+    try:
+        g2, _ = gpu_run(inp4, 300)
+    finally:
+        del os.environ["QSIM_KERNEL"]
+    assert_parity(g2, g, what="generic multi-warp instance")
+
+
 def test_large_n_one_replication():
     inp = presets.cfg4(N=4096, R=1)
     check(inp, 60)
