@@ -33,9 +33,9 @@ UNIT = "server-iterations/s"
 JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
                            # decode-buffer pass, each written and read once at 32-byte sector granularity
 # DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from an ncu capture of a 2000-iteration
-# launch (dram__bytes_read.sum + dram__bytes_write.sum = 740.6 MB for 1.414e8 iterations); traffic grows with the
+# launch (dram__bytes_read.sum + dram__bytes_write.sum = 735.8 MB for 1.415e8 iterations); traffic grows with the
 # iterations of a launch, so a full launch is that figure times its iterations
-NCU_DRAM_BYTES_PER_ITER = 740.6e6 / 1.414e8
+NCU_DRAM_BYTES_PER_ITER = 735.8e6 / 1.415e8
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
 R_PER_GPU = 1024
 
@@ -168,7 +168,7 @@ def run_ctmc(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    n, R, dT = 1000, 8192, 10.0
+    n, R, dT = 1000, 8192, args.ctmc_seconds
     count, offset = shard(R * world, world, rank)
     inp = presets.ctmc_instance(n=n, R=count, router=ROUTER_SLI).with_(rep_offset=offset)
     sim = QSimCTMC(inp, device=f"cuda:{local}")
@@ -200,7 +200,7 @@ def run_ctmc(args):
             from oracle import run_ctmc_oracle
             cores = os.cpu_count() or 1
             done = [0] * cores
-            T_cpu = 10_000.0      # about 10 s of work for the host cores
+            T_cpu = 30_000.0      # about 10 s of work for the host cores
 
             def work(k):
                 st = run_ctmc_oracle(inp.with_(R=1, rep_offset=k), T_cpu)
@@ -232,6 +232,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="cfg1", choices=["cfg1", "ctmc"],
                     help="cfg1: the iteration-level benchmark (default); ctmc: the exponential-service model, reported in jumps/s")
+    ap.add_argument("--ctmc-seconds", type=float, default=10.0, help="simulated seconds per step of the ctmc workload")
     args = ap.parse_args()
     if args.workload == "ctmc":
         run_ctmc(args)

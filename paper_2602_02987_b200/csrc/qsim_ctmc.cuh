@@ -11,6 +11,9 @@
 // time is recomputed whenever n changes.  Per event a thread scans its 7 I jump times, applies the jump,
 // lets the policy act (decode buffers into free slots, solo group first; then the prefill gate) and updates
 // the clocks whose counts changed.  All clock arithmetic is single IEEE operations in a fixed order.
+// While a launch runs, a replication's clocks, counts and statistics sit in shared memory (word w of thread t
+// at w * blockDim + t); the four processes that take one request out of one count share one code path, so
+// the threads of a warp diverge only between arrivals, buffer abandonments and that path.
 #pragma once
 
 namespace qsimdev {
@@ -22,7 +25,7 @@ enum { CA_QP = 0, CA_X, CA_QD, CA_YM, CA_YS, CA_N };
 
 struct CtmcClk { double acc, lvl, t_last, t_fire; unsigned long long m; };
 
-// state of one replication (global memory between launches, thread-local while a launch runs)
+// state of one replication in global memory between launches
 struct CtmcRep {
     double T_end;
     unsigned long long events;
@@ -47,15 +50,35 @@ struct CtmcParams {
     uint32_t *not_done;
 };
 
+// Working copy of one replication in shared memory: 8-byte words, word w of thread t at [w * blockDim + t]
+// (consecutive threads hit consecutive banks).  Only the I classes in use take space: 5 + 62 I words.
+struct CtmcWords {
+    unsigned long long *base;   // this thread's word 0
+    uint32_t stride, I;
+    enum { W_EVENTS = 0, W_HEAD0 = 1, W_HEAD1 = 2, W_N0 = 3, W_N1 = 4, W_BASE = 5 };
+    __device__ __forceinline__ uint32_t clk(uint32_t k, uint32_t i, uint32_t f) const { return W_BASE + (k * I + i) * 5u + f; }   // f: acc, lvl, t_last, t_fire, m
+    __device__ __forceinline__ uint32_t count(uint32_t c, uint32_t i) const { return W_BASE + 35u * I + c * I + i; }             // c: Qp, X, Qd0, Qd1, Ym, Ys
+    __device__ __forceinline__ uint32_t sli(uint32_t i) const { return W_BASE + 41u * I + i; }
+    __device__ __forceinline__ uint32_t area(uint32_t a, uint32_t i) const { return W_BASE + 42u * I + a * I + i; }
+    __device__ __forceinline__ uint32_t area_t(uint32_t a, uint32_t i) const { return W_BASE + 47u * I + a * I + i; }
+    __device__ __forceinline__ uint32_t cnt(uint32_t i, uint32_t c) const { return W_BASE + 52u * I + i * 10u + c; }
+    __host__ __device__ static uint32_t words(uint32_t I) { return 5u + 62u * I; }
+    __device__ __forceinline__ unsigned long long u(uint32_t w) const { return base[(size_t)w * stride]; }
+    __device__ __forceinline__ void su(uint32_t w, unsigned long long v) const { base[(size_t)w * stride] = v; }
+    __device__ __forceinline__ double d(uint32_t w) const { return __longlong_as_double((long long)u(w)); }
+    __device__ __forceinline__ void sd(uint32_t w, double v) const { su(w, (unsigned long long)__double_as_longlong(v)); }
+};
+enum { CQ_QP = 0, CQ_X = 1, CQ_QD0 = 2, CQ_QD1 = 3, CQ_YM = 4, CQ_YS = 5 };
+
 struct CtmcSim {
     const CtmcParams &p;
-    CtmcRep &S;
+    const CtmcWords W;
     uint8_t *ring0, *ring1;
     const uint32_t rep;
-    uint32_t totX, totYm, totYs;
+    uint32_t totX, totYm, totYs, err;
 
-    __device__ CtmcSim(const CtmcParams &p_, CtmcRep &S_, uint32_t rep_)
-        : p(p_), S(S_), ring0(p_.rings + (size_t)rep_ * 2 * p_.qcap), ring1(ring0 + p_.qcap), rep(rep_), totX(0), totYm(0), totYs(0) {}
+    __device__ CtmcSim(const CtmcParams &p_, const CtmcWords &W_, uint32_t rep_)
+        : p(p_), W(W_), ring0(p_.rings + (size_t)rep_ * 2 * p_.qcap), ring1(ring0 + p_.qcap), rep(rep_), totX(0), totYm(0), totYs(0), err(0) {}
 
     __device__ __forceinline__ uint32_t stream_of(uint32_t k, uint32_t i) const
     {
@@ -72,49 +95,63 @@ struct CtmcSim {
         const CtmcClassPar &c = p.cls[i];
         return k <= CK_ABD1 ? (k == CK_ARR ? 0.0 : c.theta) : (k == CK_SP ? c.mu_p : (k == CK_SDM ? c.mu_m : c.mu_s));
     }
+    __device__ __forceinline__ uint32_t cq(uint32_t c, uint32_t i) const { return (uint32_t)W.u(W.count(c, i)); }
     __device__ __forceinline__ void touch(uint32_t a, uint32_t i, uint32_t count, double t)
     {
-        S.area[a][i] = __dadd_rn(S.area[a][i], __dmul_rn((double)count, __dsub_rn(t, S.area_t[a][i])));
-        S.area_t[a][i] = t;
+        W.sd(W.area(a, i), __dadd_rn(W.d(W.area(a, i)), __dmul_rn((double)count, __dsub_rn(t, W.d(W.area_t(a, i))))));
+        W.sd(W.area_t(a, i), t);
     }
     // the count that process k of class i runs on changes from n_old to n_new at time t
     __device__ void clk_change(uint32_t k, uint32_t i, uint32_t n_old, uint32_t n_new, double t)
     {
         const double c = coef(k, i);
         if (!(c > 0.0)) return;
-        CtmcClk &q = S.clk[k][i];
-        q.acc = __dadd_rn(q.acc, __dmul_rn(__dmul_rn(c, (double)n_old), __dsub_rn(t, q.t_last)));
-        q.t_last = t;
+        const double acc = __dadd_rn(W.d(W.clk(k, i, 0)), __dmul_rn(__dmul_rn(c, (double)n_old), __dsub_rn(t, W.d(W.clk(k, i, 2)))));
+        W.sd(W.clk(k, i, 0), acc);
+        W.sd(W.clk(k, i, 2), t);
+        double tf = dinf();
         if (n_new > 0) {
-            double rem = __dsub_rn(q.lvl, q.acc);
+            double rem = __dsub_rn(W.d(W.clk(k, i, 1)), acc);
             if (rem < 0.0) rem = 0.0;
-            q.t_fire = __dadd_rn(t, __ddiv_rn(rem, __dmul_rn(c, (double)n_new)));
-        } else {
-            q.t_fire = dinf();
+            tf = __dadd_rn(t, __ddiv_rn(rem, __dmul_rn(c, (double)n_new)));
         }
+        W.sd(W.clk(k, i, 3), tf);
     }
     // process k of class i has just jumped at t and its count is now n_new: next level from draw m
     __device__ void clk_fired(uint32_t k, uint32_t i, uint32_t n_new, double t, uint32_t &w2)
     {
-        CtmcClk &q = S.clk[k][i];
+        const unsigned long long m = W.u(W.clk(k, i, 4));
         uint32_t w0, w1, w3;
-        rnd(stream_of(k, i), q.m, w0, w1, w2, w3);
-        q.lvl = -qlog(u53(w0, w1));
-        q.m += 1;
-        q.acc = 0.0;
-        q.t_last = t;
-        q.t_fire = n_new > 0 ? __dadd_rn(t, __ddiv_rn(q.lvl, __dmul_rn(coef(k, i), (double)n_new))) : dinf();
+        rnd(stream_of(k, i), m, w0, w1, w2, w3);
+        const double lvl = -qlog(u53(w0, w1));
+        W.sd(W.clk(k, i, 1), lvl);
+        W.su(W.clk(k, i, 4), m + 1);
+        W.sd(W.clk(k, i, 0), 0.0);
+        W.sd(W.clk(k, i, 2), t);
+        W.sd(W.clk(k, i, 3), n_new > 0 ? __dadd_rn(t, __ddiv_rn(lvl, __dmul_rn(coef(k, i), (double)n_new))) : dinf());
     }
-    __device__ void set_Qp(uint32_t i, uint32_t v, double t) { clk_change(CK_ABP, i, S.Qp[i], v, t); touch(CA_QP, i, S.Qp[i], t); S.Qp[i] = v; }
-    __device__ void set_X(uint32_t i, uint32_t v, double t) { clk_change(CK_SP, i, S.X[i], v, t); touch(CA_X, i, S.X[i], t); totX += v - S.X[i]; S.X[i] = v; }
+    // setters that keep the time integral and the process that runs on the count in step
+    __device__ void set_count(uint32_t c, uint32_t i, uint32_t v, double t)
+    {
+        // c -> (process, integral): Qp -> (ABP, Q_p), X -> (SP, X), Ym -> (SDM, Y_m), Ys -> (SDS, Y_s)
+        const uint32_t k = c == CQ_QP ? CK_ABP : (c == CQ_X ? CK_SP : (c == CQ_YM ? CK_SDM : CK_SDS));
+        const uint32_t a = c == CQ_QP ? CA_QP : (c == CQ_X ? CA_X : (c == CQ_YM ? CA_YM : CA_YS));
+        const uint32_t old = cq(c, i);
+        clk_change(k, i, old, v, t);
+        touch(a, i, old, t);
+        W.su(W.count(c, i), v);
+        if (c == CQ_X) totX += v - old;
+        if (c == CQ_YM) totYm += v - old;
+        if (c == CQ_YS) totYs += v - old;
+    }
     __device__ void set_Qd(uint32_t pool, uint32_t i, uint32_t v, double t)
     {
-        clk_change(pool ? CK_ABD1 : CK_ABD0, i, S.Qd[pool][i], v, t);
-        touch(CA_QD, i, S.Qd[0][i] + S.Qd[1][i], t);
-        S.Qd[pool][i] = v;
+        const uint32_t q0 = cq(CQ_QD0, i), q1 = cq(CQ_QD1, i);
+        clk_change(pool ? CK_ABD1 : CK_ABD0, i, pool ? q1 : q0, v, t);
+        touch(CA_QD, i, q0 + q1, t);
+        W.su(W.count(pool ? CQ_QD1 : CQ_QD0, i), v);
     }
-    __device__ void set_Ym(uint32_t i, uint32_t v, double t) { clk_change(CK_SDM, i, S.Ym[i], v, t); touch(CA_YM, i, S.Ym[i], t); totYm += v - S.Ym[i]; S.Ym[i] = v; }
-    __device__ void set_Ys(uint32_t i, uint32_t v, double t) { clk_change(CK_SDS, i, S.Ys[i], v, t); touch(CA_YS, i, S.Ys[i], t); totYs += v - S.Ys[i]; S.Ys[i] = v; }
+    __device__ __forceinline__ void bump(uint32_t i, uint32_t c) { W.su(W.cnt(i, c), W.u(W.cnt(i, c)) + 1ull); }
 
     // Section 4.1 occupancy gate (xi_i = (X_i - n x*_i)/x*_i, ties to the largest Q_p,i - n q*_p,i) or the
     // Section 5.1.1 priority gate (smallest static rank); ties to the lowest class index
@@ -123,14 +160,15 @@ struct CtmcSim {
         uint32_t best = NONE32;
         if (p.gate == 1) {
             for (uint32_t i = 0; i < p.I; ++i)
-                if (S.Qp[i] > 0 && (best == NONE32 || p.cls[i].prio < p.cls[best].prio)) best = i;
+                if (cq(CQ_QP, i) > 0 && (best == NONE32 || p.cls[i].prio < p.cls[best].prio)) best = i;
             return best;
         }
         double bxi = 0.0, bdq = 0.0;
         for (uint32_t i = 0; i < p.I; ++i) {
-            if (S.Qp[i] == 0 || !(p.cls[i].xstar > 0.0)) continue;
-            const double xi = __ddiv_rn(__dsub_rn((double)S.X[i], p.cls[i].nx), p.cls[i].xstar);
-            const double dq = __dsub_rn((double)S.Qp[i], p.cls[i].nq);
+            const uint32_t Qp = cq(CQ_QP, i);
+            if (Qp == 0 || !(p.cls[i].xstar > 0.0)) continue;
+            const double xi = __ddiv_rn(__dsub_rn((double)cq(CQ_X, i), p.cls[i].nx), p.cls[i].xstar);
+            const double dq = __dsub_rn((double)Qp, p.cls[i].nq);
             if (best == NONE32 || xi < bxi || (xi == bxi && dq > bdq)) { best = i; bxi = xi; bdq = dq; }
         }
         return best;
@@ -142,7 +180,9 @@ struct CtmcSim {
         const uint32_t npools = p.router == 1 ? 2u : 1u;
         for (uint32_t pool = 0; pool < npools; ++pool) {
             uint8_t *ring = pool ? ring1 : ring0;
-            while (S.n[pool] > 0) {
+            const uint32_t wn = pool ? CtmcWords::W_N1 : CtmcWords::W_N0, wh = pool ? CtmcWords::W_HEAD1 : CtmcWords::W_HEAD0;
+            uint32_t n = (uint32_t)W.u(wn);
+            while (n > 0) {
                 bool to_solo;
                 if (p.router == 1) {
                     to_solo = pool == 0;
@@ -152,151 +192,205 @@ struct CtmcSim {
                     else if (totYm < cap_m) to_solo = false;
                     else break;
                 }
-                const uint32_t i = ring[S.head[pool]];
-                S.head[pool] = S.head[pool] + 1 == p.qcap ? 0 : S.head[pool] + 1;
-                S.n[pool] -= 1;
-                set_Qd(pool, i, S.Qd[pool][i] - 1, t);
-                if (to_solo) { set_Ys(i, S.Ys[i] + 1, t); S.cnt[i][CC_PLACED_SOLO]++; }
-                else         { set_Ym(i, S.Ym[i] + 1, t); S.cnt[i][CC_PLACED_MIXED]++; }
+                uint32_t head = (uint32_t)W.u(wh);
+                const uint32_t i = ring[head];
+                head = head + 1 == p.qcap ? 0 : head + 1;
+                W.su(wh, head);
+                n -= 1;
+                W.su(wn, n);
+                set_Qd(pool, i, cq(pool ? CQ_QD1 : CQ_QD0, i) - 1, t);
+                set_count(to_solo ? CQ_YS : CQ_YM, i, cq(to_solo ? CQ_YS : CQ_YM, i) + 1, t);
+                bump(i, to_solo ? CC_PLACED_SOLO : CC_PLACED_MIXED);
             }
         }
         while (totX < p.M) {
             const uint32_t i = gate_class();
             if (i == NONE32) break;
-            set_Qp(i, S.Qp[i] - 1, t);
-            set_X(i, S.X[i] + 1, t);
-            S.cnt[i][CC_ADMITTED]++;
+            set_count(CQ_QP, i, cq(CQ_QP, i) - 1, t);
+            set_count(CQ_X, i, cq(CQ_X, i) + 1, t);
+            bump(i, CC_ADMITTED);
         }
     }
 
+    // empty system at t = 0: every process gets its first level, the arrival processes their first jump time
     __device__ void init()
     {
+        for (uint32_t w = 0; w < CtmcWords::words(p.I); ++w) W.su(w, 0ull);
         for (uint32_t i = 0; i < p.I; ++i) {
             for (uint32_t k = 0; k < CK_N; ++k) {
-                CtmcClk &q = S.clk[k][i];
                 uint32_t w0, w1, w2, w3;
                 rnd(stream_of(k, i), 0, w0, w1, w2, w3);
-                q.acc = 0.0; q.t_last = 0.0; q.t_fire = dinf(); q.lvl = -qlog(u53(w0, w1)); q.m = 1;
+                W.sd(W.clk(k, i, 1), -qlog(u53(w0, w1)));
+                W.sd(W.clk(k, i, 3), dinf());
+                W.su(W.clk(k, i, 4), 1ull);
             }
             const double Lam = __dmul_rn((double)p.N, p.cls[i].lambda);
-            if (Lam > 0.0) S.clk[CK_ARR][i].t_fire = __dadd_rn(0.0, __ddiv_rn(S.clk[CK_ARR][i].lvl, Lam));
+            if (Lam > 0.0) W.sd(W.clk(CK_ARR, i, 3), __dadd_rn(0.0, __ddiv_rn(W.d(W.clk(CK_ARR, i, 1)), Lam)));
         }
     }
 
     // events with t <= T_end, at most `budget` of them; returns true when none is left up to T_end
     __device__ bool run(double T_end, unsigned long long budget)
     {
-        for (uint32_t i = 0; i < p.I; ++i) { totX += S.X[i]; totYm += S.Ym[i]; totYs += S.Ys[i]; }
-        S.T_end = T_end;
+        for (uint32_t i = 0; i < p.I; ++i) { totX += cq(CQ_X, i); totYm += cq(CQ_YM, i); totYs += cq(CQ_YS, i); }
+        unsigned long long events = W.u(CtmcWords::W_EVENTS);
+        bool finished;
         for (;;) {
             // earliest process; ties by process kind, then class (strict '<' in that scan order)
             double te = dinf();
             uint32_t bk = 0, bi = 0;
+#pragma unroll
             for (uint32_t k = 0; k < CK_N; ++k)
                 for (uint32_t i = 0; i < p.I; ++i) {
-                    const double tf = S.clk[k][i].t_fire;
+                    const double tf = W.d(W.clk(k, i, 3));
                     if (tf < te) { te = tf; bk = k; bi = i; }
                 }
-            if (!(te <= T_end)) return true;
-            if (budget == 0) return false;
+            if (!(te <= T_end)) { finished = true; break; }
+            if (budget == 0) { finished = false; break; }
             --budget;
             const double t = te;
             const uint32_t i = bi;
-            S.events++;
+            ++events;
             uint32_t w2 = 0;
             if (bk == CK_ARR) {
-                S.cnt[i][CC_ARRIVALS]++;
-                set_Qp(i, S.Qp[i] + 1, t);
-                CtmcClk &q = S.clk[CK_ARR][i];
+                bump(i, CC_ARRIVALS);
+                set_count(CQ_QP, i, cq(CQ_QP, i) + 1, t);
+                const unsigned long long m = W.u(W.clk(CK_ARR, i, 4));
                 uint32_t w0, w1, w3;
-                rnd(stream_of(CK_ARR, i), q.m, w0, w1, w2, w3);
-                q.lvl = -qlog(u53(w0, w1));
-                q.m += 1;
-                q.t_fire = __dadd_rn(t, __ddiv_rn(q.lvl, __dmul_rn((double)p.N, p.cls[i].lambda)));
-            } else if (bk == CK_ABP) {
-                touch(CA_QP, i, S.Qp[i], t);
-                S.Qp[i] -= 1;
-                S.cnt[i][CC_ABANDONED_P]++;
-                clk_fired(CK_ABP, i, S.Qp[i], t, w2);
+                rnd(stream_of(CK_ARR, i), m, w0, w1, w2, w3);
+                const double lvl = -qlog(u53(w0, w1));
+                W.sd(W.clk(CK_ARR, i, 1), lvl);
+                W.su(W.clk(CK_ARR, i, 4), m + 1);
+                W.sd(W.clk(CK_ARR, i, 3), __dadd_rn(t, __ddiv_rn(lvl, __dmul_rn((double)p.N, p.cls[i].lambda))));
             } else if (bk == CK_ABD0 || bk == CK_ABD1) {
                 const uint32_t pool = bk == CK_ABD1 ? 1u : 0u;
-                const uint32_t Q = S.Qd[pool][i];
+                const uint32_t Q = cq(pool ? CQ_QD1 : CQ_QD0, i);
                 clk_fired(bk, i, Q - 1, t, w2);
                 // a uniformly chosen waiting class-i request leaves the pool's buffer; the rest keep their order
                 uint8_t *ring = pool ? ring1 : ring0;
+                const uint32_t wn = pool ? CtmcWords::W_N1 : CtmcWords::W_N0;
                 uint32_t rank = __umulhi(w2, Q), pos = 0;
-                const uint32_t n = S.n[pool], head = S.head[pool];
+                const uint32_t n = (uint32_t)W.u(wn), head = (uint32_t)W.u(pool ? CtmcWords::W_HEAD1 : CtmcWords::W_HEAD0);
                 for (pos = 0; pos < n; ++pos) {
                     uint32_t a = head + pos; if (a >= p.qcap) a -= p.qcap;
                     if (ring[a] != i) continue;
                     if (rank == 0) break;
                     --rank;
                 }
-                if (pos >= n) { S.err = ERR_INTERNAL; return true; }
+                if (pos >= n) { err = ERR_INTERNAL; finished = true; break; }
                 for (uint32_t k = pos; k + 1 < n; ++k) {
                     uint32_t a = head + k, b = head + k + 1;
                     if (a >= p.qcap) a -= p.qcap;
                     if (b >= p.qcap) b -= p.qcap;
                     ring[a] = ring[b];
                 }
-                S.n[pool] = n - 1;
-                touch(CA_QD, i, S.Qd[0][i] + S.Qd[1][i], t);
-                S.Qd[pool][i] = Q - 1;
-                S.cnt[i][CC_ABANDONED_D]++;
-            } else if (bk == CK_SP) {
-                touch(CA_X, i, S.X[i], t);
-                S.X[i] -= 1; totX -= 1;
-                S.cnt[i][CC_PREFILL_DONE]++;
-                clk_fired(CK_SP, i, S.X[i], t, w2);
-                uint32_t pool = 0;
-                if (p.router == 1) {
-                    // SLI-aware router: one uniform per finished prefill decides the pool (Section 5.2)
-                    uint32_t w0, w1, w3;
-                    rnd((STREAM_SLI << 8) | i, S.sli_ord[i]++, w0, w1, w2, w3);
-                    pool = u53(w0, w1) <= p.cls[i].ps ? 0u : 1u;
-                }
-                if (S.n[pool] >= p.qcap) {
-                    S.cnt[i][CC_OVERFLOW_D]++;
-                } else {
-                    uint32_t a = S.head[pool] + S.n[pool]; if (a >= p.qcap) a -= p.qcap;
-                    (pool ? ring1 : ring0)[a] = (uint8_t)i;
-                    S.n[pool] += 1;
-                    set_Qd(pool, i, S.Qd[pool][i] + 1, t);
-                }
-            } else if (bk == CK_SDM) {
-                touch(CA_YM, i, S.Ym[i], t);
-                S.Ym[i] -= 1; totYm -= 1;
-                S.cnt[i][CC_DONE_MIXED]++;
-                clk_fired(CK_SDM, i, S.Ym[i], t, w2);
+                W.su(wn, n - 1);
+                touch(CA_QD, i, cq(CQ_QD0, i) + cq(CQ_QD1, i), t);
+                W.su(W.count(pool ? CQ_QD1 : CQ_QD0, i), Q - 1);
+                bump(i, CC_ABANDONED_D);
             } else {
-                touch(CA_YS, i, S.Ys[i], t);
-                S.Ys[i] -= 1; totYs -= 1;
-                S.cnt[i][CC_DONE_SOLO]++;
-                clk_fired(CK_SDS, i, S.Ys[i], t, w2);
+                // a process that runs on one count and takes one request out of it: abandonment from the prefill queue,
+                // prefill completion, mixed or solo decode completion (one code path for the four)
+                const uint32_t c = bk == CK_ABP ? CQ_QP : (bk == CK_SP ? CQ_X : (bk == CK_SDM ? CQ_YM : CQ_YS));
+                const uint32_t a = bk == CK_ABP ? CA_QP : (bk == CK_SP ? CA_X : (bk == CK_SDM ? CA_YM : CA_YS));
+                const uint32_t cc = bk == CK_ABP ? CC_ABANDONED_P : (bk == CK_SP ? CC_PREFILL_DONE : (bk == CK_SDM ? CC_DONE_MIXED : CC_DONE_SOLO));
+                const uint32_t old = cq(c, i);
+                touch(a, i, old, t);
+                W.su(W.count(c, i), old - 1);
+                totX -= bk == CK_SP ? 1u : 0u; totYm -= bk == CK_SDM ? 1u : 0u; totYs -= bk == CK_SDS ? 1u : 0u;
+                bump(i, cc);
+                clk_fired(bk, i, old - 1, t, w2);
+                if (bk == CK_SP) {
+                    uint32_t pool = 0;
+                    if (p.router == 1) {
+                        // SLI-aware router: one uniform per finished prefill decides the pool (Section 5.2)
+                        const unsigned long long ord = W.u(W.sli(i));
+                        W.su(W.sli(i), ord + 1);
+                        uint32_t w0, w1, w3;
+                        rnd((STREAM_SLI << 8) | i, ord, w0, w1, w2, w3);
+                        pool = u53(w0, w1) <= p.cls[i].ps ? 0u : 1u;
+                    }
+                    const uint32_t wn = pool ? CtmcWords::W_N1 : CtmcWords::W_N0;
+                    const uint32_t n = (uint32_t)W.u(wn);
+                    if (n >= p.qcap) {
+                        bump(i, CC_OVERFLOW_D);
+                    } else {
+                        uint32_t pos = (uint32_t)W.u(pool ? CtmcWords::W_HEAD1 : CtmcWords::W_HEAD0) + n; if (pos >= p.qcap) pos -= p.qcap;
+                        (pool ? ring1 : ring0)[pos] = (uint8_t)i;
+                        W.su(wn, n + 1);
+                        set_Qd(pool, i, cq(pool ? CQ_QD1 : CQ_QD0, i) + 1, t);
+                    }
+                }
             }
             dispatch(t);
+        }
+        W.su(CtmcWords::W_EVENTS, events);
+        return finished;
+    }
+
+    // the record in global memory <-> the working copy
+    __device__ void load(const CtmcRep &S)
+    {
+        W.su(CtmcWords::W_EVENTS, S.events);
+        W.su(CtmcWords::W_HEAD0, S.head[0]); W.su(CtmcWords::W_HEAD1, S.head[1]); W.su(CtmcWords::W_N0, S.n[0]); W.su(CtmcWords::W_N1, S.n[1]);
+        for (uint32_t i = 0; i < p.I; ++i) {
+            for (uint32_t k = 0; k < CK_N; ++k) {
+                const CtmcClk &q = S.clk[k][i];
+                W.sd(W.clk(k, i, 0), q.acc); W.sd(W.clk(k, i, 1), q.lvl); W.sd(W.clk(k, i, 2), q.t_last); W.sd(W.clk(k, i, 3), q.t_fire);
+                W.su(W.clk(k, i, 4), q.m);
+            }
+            W.su(W.count(CQ_QP, i), S.Qp[i]); W.su(W.count(CQ_X, i), S.X[i]); W.su(W.count(CQ_QD0, i), S.Qd[0][i]);
+            W.su(W.count(CQ_QD1, i), S.Qd[1][i]); W.su(W.count(CQ_YM, i), S.Ym[i]); W.su(W.count(CQ_YS, i), S.Ys[i]);
+            W.su(W.sli(i), S.sli_ord[i]);
+            for (uint32_t a = 0; a < CA_N; ++a) { W.sd(W.area(a, i), S.area[a][i]); W.sd(W.area_t(a, i), S.area_t[a][i]); }
+            for (uint32_t c = 0; c < CC_N; ++c) W.su(W.cnt(i, c), S.cnt[i][c]);
+        }
+    }
+    __device__ void store(CtmcRep &S) const
+    {
+        S.events = W.u(CtmcWords::W_EVENTS);
+        S.head[0] = (uint32_t)W.u(CtmcWords::W_HEAD0); S.head[1] = (uint32_t)W.u(CtmcWords::W_HEAD1);
+        S.n[0] = (uint32_t)W.u(CtmcWords::W_N0); S.n[1] = (uint32_t)W.u(CtmcWords::W_N1);
+        for (uint32_t i = 0; i < p.I; ++i) {
+            for (uint32_t k = 0; k < CK_N; ++k) {
+                CtmcClk &q = S.clk[k][i];
+                q.acc = W.d(W.clk(k, i, 0)); q.lvl = W.d(W.clk(k, i, 1)); q.t_last = W.d(W.clk(k, i, 2)); q.t_fire = W.d(W.clk(k, i, 3));
+                q.m = W.u(W.clk(k, i, 4));
+            }
+            S.Qp[i] = cq(CQ_QP, i); S.X[i] = cq(CQ_X, i); S.Qd[0][i] = cq(CQ_QD0, i); S.Qd[1][i] = cq(CQ_QD1, i);
+            S.Ym[i] = cq(CQ_YM, i); S.Ys[i] = cq(CQ_YS, i);
+            S.sli_ord[i] = W.u(W.sli(i));
+            for (uint32_t a = 0; a < CA_N; ++a) { S.area[a][i] = W.d(W.area(a, i)); S.area_t[a][i] = W.d(W.area_t(a, i)); }
+            for (uint32_t c = 0; c < CC_N; ++c) S.cnt[i][c] = W.u(W.cnt(i, c));
         }
     }
 };
 
-// One thread per replication, working on its record in global memory (a few KB that stay in the L1/L2 caches
-// while the thread runs).  init != 0: start from the empty system at t = 0 (no events are processed).
+// One thread per replication.  The replication's record lives in global memory between launches; a launch works on a
+// copy in shared memory.  init != 0: start from the empty system at t = 0 (no events are processed).
 __global__ void __launch_bounds__(64) qsim_ctmc_kernel(CtmcParams p)
 {
+    extern __shared__ __align__(16) unsigned long long ctmc_sm[];
     const uint32_t rep = blockIdx.x * blockDim.x + threadIdx.x;
     if (rep >= p.R) return;
     CtmcRep &S = p.reps[rep];
+    CtmcWords W;
+    W.base = ctmc_sm + threadIdx.x; W.stride = blockDim.x; W.I = p.I;
+    CtmcSim sim(p, W, rep);
     if (p.init) {
         uint32_t *w = reinterpret_cast<uint32_t *>(&S);
         for (uint32_t o = 0; o < sizeof(CtmcRep) / 4; ++o) w[o] = 0;
-        CtmcSim sim(p, S, rep);
         sim.init();
+        sim.store(S);
         S.done = 1;
         return;
     }
     if (S.err || (S.done && S.T_end == p.T_end)) return;
-    CtmcSim sim(p, S, rep);
+    sim.load(S);
     const bool finished = sim.run(p.T_end, p.event_budget);
+    sim.store(S);
+    S.T_end = p.T_end;
+    S.err = sim.err;
     S.done = finished ? 1u : 0u;
     if (!finished) atomicAdd(p.not_done, 1u);
 }
@@ -341,6 +435,17 @@ CtmcSections ctmc_sections(const qsim_ctmc_config &c)
     return s;
 }
 
+// one warp per block: many small blocks spread the replications over all SMs; the working copies of a block's
+// replications take 32 (5 + 62 I) 8-byte words of shared memory
+int ctmc_launch_shape(uint32_t I, uint32_t &threads, size_t &smem)
+{
+    threads = 32;
+    smem = (size_t)threads * CtmcWords::words(I) * 8;
+    if (smem > 48u * 1024u)
+        CUDA_TRY(cudaFuncSetAttribute(qsim_ctmc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    return QSIM_OK;
+}
+
 int ctmc_params(const qsim_ctmc_config *cfg, const qsim_ctmc_class *cls, void *ws, size_t bytes, CtmcParams &p)
 {
     int rc = ctmc_validate(cfg, cls);
@@ -383,7 +488,11 @@ int qsim_ctmc_init(const qsim_ctmc_config *cfg, const qsim_ctmc_class *classes, 
     if (rc != QSIM_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     p.init = 1;
-    qsim_ctmc_kernel<<<(cfg->R + 63u) / 64u, 64, 0, st>>>(p);
+    uint32_t threads = 0;
+    size_t smem = 0;
+    rc = ctmc_launch_shape(cfg->I, threads, smem);
+    if (rc != QSIM_OK) return rc;
+    qsim_ctmc_kernel<<<(cfg->R + threads - 1u) / threads, threads, smem, st>>>(p);
     CUDA_TRY(cudaGetLastError());
     return QSIM_OK;
 }
@@ -398,11 +507,15 @@ int qsim_ctmc_run_until(const qsim_ctmc_config *cfg, const qsim_ctmc_class *clas
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     p.T_end = T_end;
     uint64_t n = 0;
+    uint32_t threads = 0;
+    size_t smem = 0;
+    rc = ctmc_launch_shape(cfg->I, threads, smem);
+    if (rc != QSIM_OK) return rc;
     // a replication that used up its per-launch event budget is continued by further launches
     for (int guard = 0; guard < 100000; ++guard) {
         uint32_t flag = 0;
         CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, st));
-        qsim_ctmc_kernel<<<(cfg->R + 63u) / 64u, 64, 0, st>>>(p);
+        qsim_ctmc_kernel<<<(cfg->R + threads - 1u) / threads, threads, smem, st>>>(p);
         CUDA_TRY(cudaGetLastError());
         ++n;
         CUDA_TRY(cudaMemcpyAsync(&flag, p.not_done, 4, cudaMemcpyDeviceToHost, st));

@@ -175,10 +175,13 @@ __device__ __forceinline__ double qlog(double x)
     }
     const double s = __ddiv_rn(__dsub_rn(m, 1.0), __dadd_rn(m, 1.0));
     const double z = __dmul_rn(s, s);
-    double acc = __ddiv_rn(1.0, 25.0);
+    // series coefficients 1/(2k+1): the correctly rounded quotients, formed once at compile time
+    constexpr double inv_odd[13] = { 1.0 / 1.0, 1.0 / 3.0, 1.0 / 5.0, 1.0 / 7.0, 1.0 / 9.0, 1.0 / 11.0, 1.0 / 13.0, 1.0 / 15.0,
+                                     1.0 / 17.0, 1.0 / 19.0, 1.0 / 21.0, 1.0 / 23.0, 1.0 / 25.0 };
+    double acc = inv_odd[12];
 #pragma unroll
     for (int k = 11; k >= 0; --k)
-        acc = __dadd_rn(__dmul_rn(acc, z), __ddiv_rn(1.0, (double)(2 * k + 1)));
+        acc = __dadd_rn(__dmul_rn(acc, z), inv_odd[k]);
     const double logm = __dmul_rn(__dmul_rn(2.0, s), acc);
     return __dadd_rn(__dmul_rn((double)e, 0.6931471805599453), logm);
 }
