@@ -42,13 +42,13 @@ def test_ctmc_parity_element_by_element(router, gate, theta, lam):
     assert ref["abandoned_d"].sum() > 0 or min(theta) == 0.0
 
 
-def test_ctmc_replication_keyed_and_large_cluster():
+def test_ctmc_full_size_in_the_bench_launch_configuration():
     from oracle import run_ctmc_oracle
-    inp = presets.ctmc_instance(n=400, R=1024, router=ROUTER_SLI)
-    gpu = gpu_run(inp, [30.0])
+    inp = presets.ctmc_instance(n=1000, R=8192, router=ROUTER_SLI)       # what `bench.py --workload ctmc` times
+    gpu = gpu_run(inp, [10.0, 20.0])
     # sampled replications against the oracle (the Philox counter holds the global replication index)
-    for r in (0, 517, 1023):
-        ref = run_ctmc_oracle(inp.with_(rep_offset=r, R=1), 30.0)
+    for r in (0, 4097, 8191):
+        ref = run_ctmc_oracle(inp.with_(rep_offset=r, R=1), 20.0)
         for k in CTMC_COUNTERS + CTMC_STATE + ("events",):
             assert np.array_equal(gpu[k][r:r + 1], ref[k]), (r, k)
         for k in CTMC_AREAS:
@@ -72,3 +72,26 @@ def test_ctmc_eight_classes_and_argument_errors():
         QSimCTMC(inp.with_(M=inp.N + 1))
     with pytest.raises(QSimError):
         QSimCTMC(inp.with_(gate=2))
+
+
+def test_ctmc_degenerate_cases():
+    from oracle import run_ctmc_oracle
+    base = presets.ctmc_instance(n=6, R=3)
+    cases = {
+        "one replication": base.with_(R=1),
+        "no mixed GPU: nothing is ever admitted": base.with_(M=0),
+        "every GPU mixed: no solo slots": base.with_(M=base.N),
+        "B = 1: mixed GPUs hold no decode": base.with_(B=1),
+        "a class without arrivals": base.with_(lam=np.array([0.5, 0.0])),
+        "no patience": base.with_(theta=np.zeros(2)),
+        "buffer of one request": base.with_(qcap=1, lam=np.array([2.0, 2.0])),
+    }
+    for what, inp in cases.items():
+        ref = run_ctmc_oracle(inp, 50.0)
+        compare(gpu_run(inp, [50.0]), ref, what)
+    st = gpu_run(cases["no mixed GPU: nothing is ever admitted"], [50.0])
+    assert st["admitted"].sum() == 0 and st["arrivals"].sum() > 0
+    assert gpu_run(cases["buffer of one request"], [50.0])["overflow_d"].sum() > 0
+    # an end time of zero processes nothing
+    z = gpu_run(base, [0.0])
+    assert z["events"].sum() == 0 and z["T_elapsed"].max() == 0.0

@@ -28,6 +28,22 @@ def _worker(rank, world, port, R, horizon, out_dir):
     dist.destroy_process_group()
 
 
+def _ctmc_worker(rank, world, port, R, T_end, out_dir):
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from oracle import run_ctmc_oracle
+    from paper_2602_02987_b200.sharding import gather_stats, shard
+    from qsim_inputs import presets
+    dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
+    count, offset = shard(R, world, rank)
+    inp = presets.ctmc_instance(n=12, R=count, router=1).with_(rep_offset=offset)
+    everything = gather_stats(run_ctmc_oracle(inp, T_end))
+    if rank == 0:
+        np.savez(os.path.join(out_dir, "ctmc.npz"), **everything)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def test_shard_covers_all_replications_once():
     from paper_2602_02987_b200.sharding import shard
     for R in (0, 1, 7, 8, 1024, 1000):
@@ -57,3 +73,14 @@ def test_two_ranks_reproduce_the_single_process_run(tmp_path):
     wt = totals(want)
     for k in wt:
         assert np.array_equal(tot[k], wt[k]), k
+
+
+def test_two_ranks_reproduce_the_exponential_service_run(tmp_path):
+    from oracle import run_ctmc_oracle
+    from qsim_inputs import presets
+    R, T_end, port = 5, 40.0, 29531
+    mp.spawn(_ctmc_worker, args=(2, port, R, T_end, str(tmp_path)), nprocs=2, join=True)
+    got = dict(np.load(tmp_path / "ctmc.npz"))
+    want = run_ctmc_oracle(presets.ctmc_instance(n=12, R=R, router=1), T_end)
+    for k in want:
+        assert np.array_equal(got[k], want[k]), k
