@@ -90,10 +90,12 @@ struct CtmcSim {
         const unsigned long long grep = p.rep_offset + rep;
         philox((uint32_t)index, (uint32_t)(index >> 32), stream, (uint32_t)grep, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w0, w1, w2, w3);
     }
+    // intensity of process k of class i per unit of the count it runs on (the arrival process runs on the constant 1)
     __device__ __forceinline__ double coef(uint32_t k, uint32_t i) const
     {
         const CtmcClassPar &c = p.cls[i];
-        return k <= CK_ABD1 ? (k == CK_ARR ? 0.0 : c.theta) : (k == CK_SP ? c.mu_p : (k == CK_SDM ? c.mu_m : c.mu_s));
+        return k <= CK_ABD1 ? (k == CK_ARR ? __dmul_rn((double)p.N, c.lambda) : c.theta)
+                            : (k == CK_SP ? c.mu_p : (k == CK_SDM ? c.mu_m : c.mu_s));
     }
     __device__ __forceinline__ uint32_t cq(uint32_t c, uint32_t i) const { return (uint32_t)W.u(W.count(c, i)); }
     __device__ __forceinline__ void touch(uint32_t a, uint32_t i, uint32_t count, double t)
@@ -252,17 +254,7 @@ struct CtmcSim {
             const uint32_t i = bi;
             ++events;
             uint32_t w2 = 0;
-            if (bk == CK_ARR) {
-                bump(i, CC_ARRIVALS);
-                set_count(CQ_QP, i, cq(CQ_QP, i) + 1, t);
-                const unsigned long long m = W.u(W.clk(CK_ARR, i, 4));
-                uint32_t w0, w1, w3;
-                rnd(stream_of(CK_ARR, i), m, w0, w1, w2, w3);
-                const double lvl = -qlog(u53(w0, w1));
-                W.sd(W.clk(CK_ARR, i, 1), lvl);
-                W.su(W.clk(CK_ARR, i, 4), m + 1);
-                W.sd(W.clk(CK_ARR, i, 3), __dadd_rn(t, __ddiv_rn(lvl, __dmul_rn((double)p.N, p.cls[i].lambda))));
-            } else if (bk == CK_ABD0 || bk == CK_ABD1) {
+            if (bk == CK_ABD0 || bk == CK_ABD1) {
                 const uint32_t pool = bk == CK_ABD1 ? 1u : 0u;
                 const uint32_t Q = cq(pool ? CQ_QD1 : CQ_QD0, i);
                 clk_fired(bk, i, Q - 1, t, w2);
@@ -289,17 +281,20 @@ struct CtmcSim {
                 W.su(W.count(pool ? CQ_QD1 : CQ_QD0, i), Q - 1);
                 bump(i, CC_ABANDONED_D);
             } else {
-                // a process that runs on one count and takes one request out of it: abandonment from the prefill queue,
-                // prefill completion, mixed or solo decode completion (one code path for the four)
-                const uint32_t c = bk == CK_ABP ? CQ_QP : (bk == CK_SP ? CQ_X : (bk == CK_SDM ? CQ_YM : CQ_YS));
-                const uint32_t a = bk == CK_ABP ? CA_QP : (bk == CK_SP ? CA_X : (bk == CK_SDM ? CA_YM : CA_YS));
-                const uint32_t cc = bk == CK_ABP ? CC_ABANDONED_P : (bk == CK_SP ? CC_PREFILL_DONE : (bk == CK_SDM ? CC_DONE_MIXED : CC_DONE_SOLO));
-                const uint32_t old = cq(c, i);
+                // One code path for the five processes that move one request across one count: an arrival adds one to the
+                // prefill queue (and redraws on the constant count 1); abandonment from the prefill queue, prefill
+                // completion and mixed / solo decode completion take one out of the count they run on.
+                const bool arr = bk == CK_ARR;
+                const uint32_t c = (arr || bk == CK_ABP) ? CQ_QP : (bk == CK_SP ? CQ_X : (bk == CK_SDM ? CQ_YM : CQ_YS));
+                const uint32_t a = (arr || bk == CK_ABP) ? CA_QP : (bk == CK_SP ? CA_X : (bk == CK_SDM ? CA_YM : CA_YS));
+                const uint32_t cc = arr ? CC_ARRIVALS : (bk == CK_ABP ? CC_ABANDONED_P : (bk == CK_SP ? CC_PREFILL_DONE : (bk == CK_SDM ? CC_DONE_MIXED : CC_DONE_SOLO)));
+                const uint32_t old = cq(c, i), now = arr ? old + 1 : old - 1;
+                if (arr) clk_change(CK_ABP, i, old, now, t);       // the queue's abandonment process sees the new length
                 touch(a, i, old, t);
-                W.su(W.count(c, i), old - 1);
+                W.su(W.count(c, i), now);
                 totX -= bk == CK_SP ? 1u : 0u; totYm -= bk == CK_SDM ? 1u : 0u; totYs -= bk == CK_SDS ? 1u : 0u;
                 bump(i, cc);
-                clk_fired(bk, i, old - 1, t, w2);
+                clk_fired(bk, i, arr ? 1u : now, t, w2);
                 if (bk == CK_SP) {
                     uint32_t pool = 0;
                     if (p.router == 1) {
