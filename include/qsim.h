@@ -59,7 +59,10 @@ enum { QSIM_GATE_OCCUPANCY = 0, QSIM_GATE_PRIORITY = 1,
 enum { QSIM_ROUTER_SOLO_FIRST = 0, QSIM_ROUTER_SLI = 1,
        QSIM_ROUTER_SLI_GENERAL = 2 /* two pools as QSIM_ROUTER_SLI; a freed slot goes to a class drawn with the pool's
                                       weights varpi among the classes that wait there, oldest request of the class
-                                      first [EC, General SLI-aware Extension] */ };
+                                      first [EC, General SLI-aware Extension] */,
+       QSIM_ROUTER_IMMEDIATE = 3   /* no router: a request decodes on the GPU that prefilled it, in the slot it holds
+                                      (the "immediate same-slot decoding" ablations of the EC ablation study; with
+                                      M = N it also drops the static partition) */ };
 enum { QSIM_PLACE_RANDOM = 0, QSIM_PLACE_LEAST_LOADED = 1 };
 enum { QSIM_PRICING_BUNDLED = 0, QSIM_PRICING_SEPARATE = 1 };
 enum { QSIM_LENGTH_FIXED = 0, QSIM_LENGTH_TABLE = 1 };

@@ -417,7 +417,7 @@ static void dispatch(orc_sim *s, uint32_t r, double t)
     rep_t *R = &s->reps[r];
     const orc_config *c = &s->cfg;
     /* decode routing: buffered jobs first (FCFS), solo GPUs before mixed ones */
-    if (c->router == 0) {
+    if (c->router == 0 || c->router == 3) {      /* router 3 never leaves a request in the buffer */
         while (R->dq_n[0] > 0) {
             int g = choose_server(s, r, WANT_SOLO_DECODE);
             if (g < 0) g = choose_server(s, r, WANT_MIX_DECODE);
@@ -569,7 +569,7 @@ static void on_server(orc_sim *s, uint32_t r, uint32_t g, double t)
             if (R->h_ttft) R->h_ttft[(size_t)i * ORC_NBIN + orc_hist_bin(ttft)]++;
             /* hand over to the decode stage: pool drawn once per job under the SLI-aware router */
             uint32_t pool = 0;
-            if (c->router >= 1) {
+            if (c->router == 1 || c->router == 2) {
                 uint32_t w[4];
                 draw(s, r, (STREAM_SLI << 8) | i, R->sli_ord[i]++, w);
                 pool = (orc_u53(w[0], w[1]) <= s->tg[R->blk].p_solo[i]) ? 0u : 1u;
@@ -584,6 +584,9 @@ static void on_server(orc_sim *s, uint32_t r, uint32_t g, double t)
                 djob_t *d = &R->dq[pool][R->dq_n[pool]++];
                 d->t_pf = t; d->P = v->pf_job.P; d->D = v->pf_job.D; d->cls = i; d->ord = v->pf_job.ord;
                 R->Qd_pool[pool][i]++;
+                /* ablation "immediate same-slot decoding" (EC, additional ablation studies): no router, the request
+                 * goes on decoding on this GPU, in the slot it already holds (it passes through the empty buffer) */
+                if (c->router == 3) place_decode(s, r, 0, g, R->dq_n[0] - 1, t);
             }
         }
     }

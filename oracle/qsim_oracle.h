@@ -19,7 +19,8 @@
  *   - prefill gate: occupancy deviation xi_i, or static D_i/P_i priority [Sections 4.1, 5.1.1]
  *   - decode router: solo-first with one FCFS buffer, or the SLI-aware
  *     randomized split with two buffers, optionally with class selection
- *     inside each pool by the weights varpi                              [Sections 4.1, 5.2, EC general SLI extension]
+ *     inside each pool by the weights varpi; or no router at all (decode on the
+ *     GPU that prefilled, EC ablation study)                              [Sections 4.1, 5.2, EC general SLI extension]
  *   - revenue under bundled and separate charging                        [Eq. (21)-(23)]
  *   - piecewise-constant rate / target tables switched at block ends without pre-emption
  *                                                                        [Section 6.2, online controller]

@@ -45,7 +45,7 @@ constexpr int TOUCH_CAP = 48;
 // run time; otherwise the set bits say which features the instance contains and everything else is
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
-                   F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024, F_SLIG = 2048;
+                   F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024, F_SLIG = 2048, F_IMM = 4096;
 // F_MW: several warps per replication.  Warp 0 (the master) runs the round loop and every event handler; the
 // other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
 // round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
@@ -291,7 +291,7 @@ __device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long l
 template <int SPL, uint32_t F>
 struct Sim {
     __device__ __forceinline__ bool f_abandon() const { return (F & F_GENERIC) ? p.any_theta != 0 : (F & F_ABANDON) != 0; }
-    __device__ __forceinline__ bool f_sli() const { return (F & F_GENERIC) ? p.router >= 1 : (F & F_SLI) != 0; }
+    __device__ __forceinline__ bool f_sli() const { return (F & F_GENERIC) ? (p.router == 1 || p.router == 2) : (F & F_SLI) != 0; }
     __device__ __forceinline__ bool f_slig() const { return (F & F_GENERIC) ? p.router == 2 : false; }
     __device__ __forceinline__ bool f_kappa() const { return (F & F_GENERIC) ? p.coef[5] != 0.0 : (F & F_KAPPA) != 0; }
     __device__ __forceinline__ bool f_hist() const { return (F & F_GENERIC) ? hist != nullptr : (F & F_HIST) != 0; }
@@ -1098,6 +1098,13 @@ struct Sim {
             __syncwarp();   // every lane has read the finished job before its owner clears it
             if (lane == owner) pfjob[g] = 0;
             __syncwarp();
+            // No router (immediate same-slot decoding, an ablation of the paper's EC): the request goes on decoding on
+            // g, in the slot it holds; it passes through the empty buffer at this instant.
+            const bool immediate = (F & F_GENERIC) && p.router == 3;
+            if (immediate) {
+                place_job(0, g, i, P, D, t, false);
+                __syncwarp();
+            }
             // the prefill slot of g is idle again
             if (!recount_idle && g < M && ndec[g] <= p.B - 1) {
                 n_idle_pf++;
@@ -1105,8 +1112,8 @@ struct Sim {
             }
             // Decode stage.  With an empty buffer the request is its head at once: place it if a slot is free.
             const uint32_t n = pool ? dq_n1 : dq_n0;
-            bool placed = false;
-            if (n == 0) {
+            bool placed = immediate;
+            if (!immediate && n == 0) {
                 uint32_t h;
                 if (f_sli()) {
                     h = choose_server(pool == 0 ? WANT_SOLO : WANT_MIX);

@@ -95,7 +95,7 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
     if (cfg->C < 1 || cfg->C > 65535) return fail(QSIM_EINVAL, "C must be in 1..65535");
     if (cfg->nblk < 1) return fail(QSIM_EINVAL, "nblk must be >= 1");
     if (cfg->qcap < 1 || cfg->qcap > (1u << 24)) return fail(QSIM_EINVAL, "qcap must be in 1..2^24");
-    if (cfg->gate > 2 || cfg->router > 2 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
+    if (cfg->gate > 2 || cfg->router > 3 || cfg->placement > 1 || cfg->pricing > 1 || cfg->length_mode > 1 || cfg->hist > 1)
         return fail(QSIM_EINVAL, "enum out of range");
     if (cfg->nblk > 1 && !(cfg->block_len > 0.0 && std::isfinite(cfg->block_len)))
         return fail(QSIM_EINVAL, "block_len must be positive when nblk > 1");
@@ -170,6 +170,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
         if (cls[i].theta > 0.0) f |= F_ABANDON;
     if (c.router == QSIM_ROUTER_SLI) f |= F_SLI;
     if (c.router == QSIM_ROUTER_SLI_GENERAL) f |= F_SLI | F_SLIG;
+    if (c.router == QSIM_ROUTER_IMMEDIATE) f |= F_IMM;
     if (coef[5] != 0.0) f |= F_KAPPA;
     if (c.hist) f |= F_HIST;
     if (c.nblk > 1) f |= F_BLOCKS;
@@ -193,7 +194,7 @@ void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint3
     const char *force = std::getenv("QSIM_KERNEL");
     const bool generic_only = force && std::strcmp(force, "generic") == 0;
     // mode bits must match exactly, capability bits may be present unused (as in pick_run_kernel)
-    constexpr uint32_t MODES = F_SLI | F_SLIG | F_RANDOM | F_OCC | F_FCFS | F_HIST;
+    constexpr uint32_t MODES = F_SLI | F_SLIG | F_IMM | F_RANDOM | F_OCC | F_FCFS | F_HIST;
     const RunVariant *best = nullptr;
     int best_bits = 99;
     for (const RunVariant &v : run_variants()) {
@@ -228,7 +229,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
         if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
         // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits
         // (abandonment, KV slope, blocks) may be present without being used
-        constexpr uint32_t MODES = F_SLI | F_SLIG | F_RANDOM | F_OCC | F_FCFS | F_HIST | F_SLOTS;
+        constexpr uint32_t MODES = F_SLI | F_SLIG | F_IMM | F_RANDOM | F_OCC | F_FCFS | F_HIST | F_SLOTS;
         if (feat == ~0u || (feat & MODES) != (v.feat & MODES) || (feat & ~v.feat) != 0) continue;
         const int extra = __builtin_popcount(v.feat & ~feat);
         if (extra < best_bits) { best = &v; best_bits = extra; }

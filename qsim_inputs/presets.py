@@ -14,8 +14,8 @@ import numpy as np
 
 from . import fluid_lp as lp
 from .lengths import lognormal_tables, table_mean, table_mean_chunks
-from .spec import (GATE_OCCUPANCY, GATE_PRIORITY, LENGTH_FIXED, LENGTH_TABLE, PLACE_LEAST_LOADED,
-                   PLACE_RANDOM, PRICING_BUNDLED, PRICING_SEPARATE, ROUTER_SLI, ROUTER_SOLO_FIRST,
+from .spec import (GATE_FCFS, GATE_OCCUPANCY, GATE_PRIORITY, LENGTH_FIXED, LENGTH_TABLE, PLACE_LEAST_LOADED,
+                   PLACE_RANDOM, PRICING_BUNDLED, PRICING_SEPARATE, ROUTER_IMMEDIATE, ROUTER_SLI, ROUTER_SOLO_FIRST,
                    CtmcInputs, SimInputs)
 
 # alpha_m, beta, delta_m, alpha_s, delta_s, kappa
@@ -240,6 +240,25 @@ def paper_instance(n=50, R=5, router=ROUTER_SOLO_FIRST, gate=GATE_OCCUPANCY, pla
                 prices=[0.1, 0.2], coeffs=coeffs, gate=gate, router=router, placement=placement,
                 pricing=PRICING_SEPARATE, P_fixed=P, D_fixed=D, seed=seed, sli=sli,
                 horizon_iters=horizon_iters)
+    return inp
+
+
+ABLATIONS = {   # label -> (gate, router, static planning)   [EC, additional ablation studies]
+    "GG-SP": (GATE_OCCUPANCY, ROUTER_SOLO_FIRST, True),     # the full policy
+    "FG-SP": (GATE_FCFS, ROUTER_SOLO_FIRST, True),          # FCFS admission, solo-first routing, static partition
+    "GI-WSP": (GATE_OCCUPANCY, ROUTER_IMMEDIATE, False),    # occupancy gate, decode where the prefill ran, no partition
+    "FI-WSP": (GATE_FCFS, ROUTER_IMMEDIATE, False),         # none of the three components
+}
+
+
+def ablation(policy="GG-SP", n=50, R=4, placement=PLACE_RANDOM, seed=100, horizon_iters=20_000, **kw) -> SimInputs:
+    """The paper's two-class synthetic instance under one of the ablation policies of the EC ablation study.
+    Without static planning every GPU may prefill (M = n); the LP targets still parameterise the occupancy gate."""
+    gate, router, planned = ABLATIONS[policy]
+    inp = paper_instance(n=n, R=R, gate=gate, router=router, placement=placement, seed=seed, horizon_iters=horizon_iters, **kw)
+    if not planned:
+        inp.M[:] = n
+    inp.name = f"{policy}_n{n}"
     return inp
 
 

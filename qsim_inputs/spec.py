@@ -28,6 +28,7 @@ GATE_FCFS = 2        # oldest waiting request first, no class rule (ablation FG-
 ROUTER_SOLO_FIRST = 0      # single FCFS buffer, solo GPUs first (Section 4.1, "Downstream routing")
 ROUTER_SLI = 1             # randomized split with p_s,i, two buffers (Section 5.2)
 ROUTER_SLI_GENERAL = 2     # as ROUTER_SLI, plus class selection inside each pool by the weights varpi (EC, General SLI-aware Extension)
+ROUTER_IMMEDIATE = 3       # no router: a request decodes on the GPU that prefilled it, in the slot it holds (ablations FI-WSP / GI-WSP of the EC ablation study)
 # choice of GPU inside the eligible set
 PLACE_RANDOM = 0           # uniformly at random (paper)
 PLACE_LEAST_LOADED = 1     # fewest decodes, lowest index on ties

@@ -59,7 +59,7 @@ class Replay:
     def run(self, known_lengths=None):
         """known_lengths: callable (cls, job) -> (P, D); defaults to the fixed class lengths."""
         inp = self.inp
-        assert inp.router == 0, "the replay models the single-buffer solo-first router"
+        assert inp.router in (0, 3), "the replay models the single-buffer solo-first router and the no-router ablation"
         tr = self.tr
         k = 0
         while k < len(tr):
@@ -144,6 +144,16 @@ class Replay:
         self.batch[g] = None
 
     def _check_place(self, cls, job, g, t):
+        if self.inp.router == 3:
+            # immediate same-slot decoding (EC ablation study): the request goes on where it prefilled, at once
+            assert self.dq == [(cls, job)], "a request waited although there is no router"
+            self.dq.pop()
+            j = self.jobs[(cls, job)]
+            assert g == j["g_pf"] and t == j["t_pf"], "decode must continue on the prefill GPU at prefill completion"
+            assert self.pf[g] is None and len(self.dec[g]) < self.B, "more requests than slots on a GPU"
+            self.dec[g][(cls, job)] = [self.lengths(cls, job)[1], t]
+            j["t_place"] = t
+            return
         # FCFS across classes in the single decode buffer
         assert self.dq and self.dq[0] == (cls, job), "decode buffer not FCFS"
         self.dq.pop(0)

@@ -72,6 +72,16 @@ def test_fcfs_gate_ablation():
     check(presets.cfg1(R=4).with_(gate=GATE_FCFS), 1000)
 
 
+@pytest.mark.parametrize("policy", ["GI-WSP", "FI-WSP"])
+def test_immediate_decode_ablations(policy):
+    # no router and no static partition (EC ablation study): a request decodes on the GPU that prefilled it
+    for n, R, H, placement in ((12, 4, 3000, PLACE_RANDOM), (40, 3, 2500, PLACE_LEAST_LOADED), (600, 1, 150, PLACE_LEAST_LOADED)):
+        inp = presets.ablation(policy, n=n, R=R, horizon_iters=H, placement=placement)
+        st = check(inp, H)
+        assert st["placed_solo"].sum() == 0 and st["Qd"].sum() == 0       # every GPU is mixed, nothing waits for a slot
+        assert np.array_equal(st["placed_mixed"], st["prefill_done"])
+
+
 @pytest.mark.parametrize("placement", [PLACE_RANDOM, PLACE_LEAST_LOADED])
 def test_general_sli_router_class_selection(placement):
     # both pools backlogged with two classes: selections are drawn, requests leave from inside the buffers;

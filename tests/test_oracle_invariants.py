@@ -31,11 +31,13 @@ def small_cases():
     yield presets.paper_instance(n=6, R=1, horizon_iters=1500, gate=GATE_FCFS)
     yield presets.paper_instance(n=5, R=2, horizon_iters=1500)
     yield presets.paper_instance(n=8, R=1, horizon_iters=1500, placement=PLACE_LEAST_LOADED, gate=GATE_PRIORITY)
+    yield presets.ablation("GI-WSP", n=5, R=2, horizon_iters=1500)
+    yield presets.ablation("FI-WSP", n=6, R=1, horizon_iters=1500, placement=PLACE_LEAST_LOADED)
     c1 = presets.cfg1(R=1, horizon_iters=150)
     yield c1.with_(N=6, M=np.array([4], np.uint32), n_xstar=c1.xstar * 6, rates=c1.rates * 1.2)
 
 
-@pytest.mark.parametrize("inp", list(small_cases()), ids=lambda c: f"{c.name}-g{c.gate}-p{c.placement}")
+@pytest.mark.parametrize("inp", list(small_cases()), ids=lambda c: f"{c.name}-g{c.gate}-p{c.placement}-r{c.router}")
 def test_replay_of_every_event(inp):
     sim = OracleSim(inp, trace_cap=2_000_000)
     H = inp.meta["horizon_iters"]
