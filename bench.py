@@ -155,7 +155,8 @@ def run_reference(args, workload):
 
 def run_ctmc(args):
     """Second workload: the exponential-service model of Section 2.3 on the paper's two-class synthetic instance,
-    n = 1000 GPUs, SLI-aware router, 8192 replications per GPU; one step advances every replication by 10 s."""
+    n = 1000 GPUs, SLI-aware router, 28416 replications per GPU (one resident wave: 148 SMs x 6 blocks x 32 threads);
+    one step advances every replication by 10 s."""
     import torch
     import torch.distributed as dist
     from paper_2602_02987_b200 import QSimCTMC
@@ -168,7 +169,7 @@ def run_ctmc(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    n, R, dT = 1000, 8192, args.ctmc_seconds
+    n, R, dT = 1000, 28416, args.ctmc_seconds
     count, offset = shard(R * world, world, rank)
     inp = presets.ctmc_instance(n=n, R=count, router=ROUTER_SLI).with_(rep_offset=offset)
     sim = QSimCTMC(inp, device=f"cuda:{local}")
