@@ -231,8 +231,11 @@ def main():
     ap.add_argument("--reps", type=int, default=R_PER_GPU, help="replications per GPU")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "ctmc"],
-                    help="cfg1: the iteration-level benchmark (default); ctmc: the exponential-service model, reported in jumps/s")
+    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "ctmc", "cfg0", "cfg2", "cfg3", "cfg4"],
+                    help="cfg1: the iteration-level benchmark (default); ctmc: the exponential-service model, reported in "
+                         "jumps/s; cfg0 / cfg2 / cfg3 / cfg4: the other configurations (give --reps and --horizon, and "
+                         "--cluster for the GPUs of cfg2-4), without the end-to-end leg")
+    ap.add_argument("--cluster", type=int, default=0, help="simulated GPUs per replication for cfg2 / cfg3 / cfg4 (0 = the preset's)")
     ap.add_argument("--ctmc-seconds", type=float, default=10.0, help="simulated seconds per step of the ctmc workload")
     args = ap.parse_args()
     if args.workload == "ctmc":
@@ -241,6 +244,11 @@ def main():
     workload = (f"cfg1: 2 lognormal classes, N=64 GPUs, B=128, C=256, separate pricing, priority gate, solo-first "
                 f"router, least-loaded placement, R={args.reps} replications per GPU, {args.horizon} iterations "
                 f"of horizon per step")
+    other = args.workload != "cfg1"
+    if other:
+        args.no_e2e = True
+        workload = (f"{args.workload}" + (f" with N={args.cluster} GPUs" if args.cluster else "") +
+                    f", R={args.reps} replications per GPU, {args.horizon} iterations of horizon per step")
     if args.impl == "reference":
         run_reference(args, workload)
         return
@@ -269,7 +277,15 @@ def main():
     # replications are independent: rank k simulates global replications [k R, (k+1) R)  (weak scaling)
     from paper_2602_02987_b200.sharding import shard
     count, offset = shard(args.reps * world, world, rank)
-    inp = presets.cfg1(R=count).with_(rep_offset=offset)
+    if args.workload == "cfg1":
+        inp = presets.cfg1(R=count)
+    elif args.workload == "cfg0":
+        inp = presets.cfg0(R=count, horizon_iters=args.horizon)
+    elif args.workload == "cfg3":
+        inp = presets.cfg3(R=count, block_len=1.0, **({"N": args.cluster} if args.cluster else {}))
+    else:
+        inp = getattr(presets, args.workload)(R=count, horizon_iters=args.horizon, **({"N": args.cluster} if args.cluster else {}))
+    inp = inp.with_(rep_offset=offset)
     sim = QSim(inp, device=f"cuda:{local}")
     info = sim.layout_info()
     for _ in range(args.warmup):
@@ -343,8 +359,8 @@ def main():
                        "events_per_iteration": events / iters, "requests_per_iteration": jobs / iters,
                        "queue_overflow": ovf},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_DRAM_BYTES_PER_ITER * iters / world / max(n_launch / world, 1.0),
-                         "traffic_source": "ncu capture of a 2000-iteration launch, scaled by iterations",
+                         "traffic": None if other else NCU_DRAM_BYTES_PER_ITER * iters / world / max(n_launch / world, 1.0),
+                         "traffic_source": "no capture for this workload" if other else "ncu capture of a 2000-iteration launch, scaled by iterations",
                          "peak_kind": peak_kind,
                          "bytes_per_iteration": JOB_BYTES * jobs / iters,
                          "note": "latency/issue-bound event chain; HBM fraction is the contract figure"},
@@ -354,10 +370,11 @@ def main():
             out["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:
             cores = os.cpu_count() or 1
-            h_s = 50_000       # about 10 s of work for the host cores
+            # about 10 s of work for the host cores: the oracle scans every GPU at every event
+            h_s = 50_000 if not other else max(100, int(1.0e6 / inp.N))
             v, it_s, dt = oracle_throughput(inp, h_s, 2 * cores, cores)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                   "sample": f"{2 * cores} replications x {h_s} iterations of horizon of cfg1, one per thread, {dt:.1f} s"}
+                                   "sample": f"{2 * cores} replications x {h_s} iterations of horizon of {args.workload}, one per thread, {dt:.1f} s"}
         print(json.dumps(out))
     sim.close()
     if world > 1:
