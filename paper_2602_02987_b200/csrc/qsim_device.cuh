@@ -874,6 +874,7 @@ struct Sim {
         // prefill gate on mixed GPUs whose prefill slot is idle
         if (gate_dirty) {
             while (n_idle_pf > 0) {
+                if (!__any_sync(FULL, lane < (int)p.I && cs[lane & 7].pq_n > 0)) break;      // nobody waits
                 const uint32_t i = gate_class();
                 if (i == NONE32) break;
                 // a single idle slot whose GPU is known needs no search (and draws nothing: one candidate)
