@@ -246,6 +246,7 @@ def paper_instance(n=50, R=5, router=ROUTER_SOLO_FIRST, gate=GATE_OCCUPANCY, pla
 ABLATIONS = {   # label -> (gate, router, static planning)   [EC, additional ablation studies]
     "GG-SP": (GATE_OCCUPANCY, ROUTER_SOLO_FIRST, True),     # the full policy
     "FG-SP": (GATE_FCFS, ROUTER_SOLO_FIRST, True),          # FCFS admission, solo-first routing, static partition
+    "GF-WSP": (GATE_OCCUPANCY, ROUTER_SOLO_FIRST, False),   # occupancy gate, one FCFS buffer served by whichever GPU has a slot: no solo group to prefer
     "GI-WSP": (GATE_OCCUPANCY, ROUTER_IMMEDIATE, False),    # occupancy gate, decode where the prefill ran, no partition
     "FI-WSP": (GATE_FCFS, ROUTER_IMMEDIATE, False),         # none of the three components
 }

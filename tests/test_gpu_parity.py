@@ -82,6 +82,13 @@ def test_immediate_decode_ablations(policy):
         assert np.array_equal(st["placed_mixed"], st["prefill_done"])
 
 
+def test_gate_and_fcfs_ablation_without_partition():
+    # GF-WSP: every GPU is mixed, so the single FCFS buffer is served by whichever GPU has a slot
+    for n, R, H in ((12, 4, 3000), (40, 3, 2500)):
+        st = check(presets.ablation("GF-WSP", n=n, R=R, horizon_iters=H), H)
+        assert st["placed_solo"].sum() == 0 and st["placed_mixed"].sum() > 0
+
+
 @pytest.mark.parametrize("placement", [PLACE_RANDOM, PLACE_LEAST_LOADED])
 def test_general_sli_router_class_selection(placement):
     # both pools backlogged with two classes: selections are drawn, requests leave from inside the buffers;

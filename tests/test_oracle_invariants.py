@@ -31,6 +31,7 @@ def small_cases():
     yield presets.paper_instance(n=6, R=1, horizon_iters=1500, gate=GATE_FCFS)
     yield presets.paper_instance(n=5, R=2, horizon_iters=1500)
     yield presets.paper_instance(n=8, R=1, horizon_iters=1500, placement=PLACE_LEAST_LOADED, gate=GATE_PRIORITY)
+    yield presets.ablation("GF-WSP", n=5, R=1, horizon_iters=1500)
     yield presets.ablation("GI-WSP", n=5, R=2, horizon_iters=1500)
     yield presets.ablation("FI-WSP", n=6, R=1, horizon_iters=1500, placement=PLACE_LEAST_LOADED)
     c1 = presets.cfg1(R=1, horizon_iters=150)
