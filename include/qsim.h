@@ -145,6 +145,17 @@ int qsim_workspace_bytes(const qsim_t *h, size_t *bytes);
 int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
 
 /*
+ * Checkpoint / resume.  All state of the replications lives in the caller's workspace, so a checkpoint is a copy of
+ * its first qsim_workspace_bytes bytes taken between calls (after qsim_run / qsim_run_until has returned), and a
+ * resume is: qsim_create with the same arguments, copy the bytes into a [device] workspace, then this call in place of
+ * qsim_bind.  Nothing is initialised; the next qsim_run continues where the checkpointed run stopped, with bit-identical
+ * results [the time horizon of Eq. (21)-(23) composes: run(a); run(b) is run(a+b)].  Targets installed with
+ * qsim_set_targets are part of the handle, not of the workspace: install them again.  QSIM_ESTATE if the bytes hold
+ * no resumable state (a replication stopped on an internal error).
+ */
+int qsim_bind_restore(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
+
+/*
  * Advance every replication by horizon_iters more iterations of horizon [event-driven dynamics of
  * Section 2.3 under the policies of Sections 4-5]: the new end time is H * tau_ref, H the total horizon
  * requested so far and tau_ref = tau(0, B, 0) (one full solo iteration).  Events with time <= the new end

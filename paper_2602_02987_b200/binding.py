@@ -20,7 +20,7 @@ EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim
            "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
            "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error",
-           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats")
+           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats", "qsim_bind_restore")
 
 
 class QSimError(RuntimeError):
@@ -91,6 +91,7 @@ def load_library():
                                   C.POINTER(qsim_targets)]
         L.qsim_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.qsim_bind.argtypes = [vp, vp, C.c_size_t, vp]
+        L.qsim_bind_restore.argtypes = [vp, vp, C.c_size_t, vp]
         L.qsim_run.argtypes = [vp, C.c_uint64]
         L.qsim_run_until.argtypes = [vp, C.c_double]
         L.qsim_set_injected.argtypes = [vp, vp, vp, C.c_uint64]
@@ -177,7 +178,8 @@ def _unpack(per, R, I, T_hist=None):
 class QSim:
     """One handle of the CUDA library; the workspace is a torch tensor on the chosen device."""
 
-    def __init__(self, inp, device="cuda:0", stream=None):
+    def __init__(self, inp, device="cuda:0", stream=None, checkpoint=None):
+        """checkpoint: bytes of a workspace saved by `checkpoint()` of a handle with the same inputs; the run resumes there."""
         import torch
         if not torch.cuda.is_available():
             raise QSimError("no CUDA device: the simulator has no CPU path")
@@ -200,7 +202,22 @@ class QSim:
             self.ws = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.device)
             base = (self.ws.data_ptr() + 255) & ~255
             self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
-            _check(self.L.qsim_bind(self.h, C.c_void_p(base), self.workspace_bytes, C.c_void_p(self.stream.cuda_stream)))
+            self._base = base
+            if checkpoint is None:
+                _check(self.L.qsim_bind(self.h, C.c_void_p(base), self.workspace_bytes, C.c_void_p(self.stream.cuda_stream)))
+            else:
+                off = base - self.ws.data_ptr()
+                if checkpoint.numel() != self.workspace_bytes:
+                    raise QSimError("checkpoint size does not match this configuration")
+                self.ws[off:off + self.workspace_bytes].copy_(checkpoint)
+                _check(self.L.qsim_bind_restore(self.h, C.c_void_p(base), self.workspace_bytes,
+                                                C.c_void_p(self.stream.cuda_stream)))
+
+    def checkpoint(self):
+        """The workspace bytes (a CPU uint8 tensor) after the work queued so far: pass them to QSim(..., checkpoint=)."""
+        self.sync()
+        off = self._base - self.ws.data_ptr()
+        return self.ws[off:off + self.workspace_bytes].cpu()
 
     def set_event_budget(self, n: int) -> None:
         _check(self.L.qsim_set_event_budget(self.h, int(n)))

@@ -363,7 +363,8 @@ int qsim_workspace_bytes(const qsim_t *h, size_t *bytes)
     return QSIM_OK;
 }
 
-int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
+// common part of qsim_bind and qsim_bind_restore: checks the workspace and points the kernel parameters at its sections
+static int attach_workspace(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
 {
     if (!h) return fail(QSIM_EINVAL, "null handle");
     if (!ws) return fail(QSIM_EWORKSPACE, "workspace pointer is null");
@@ -386,9 +387,32 @@ int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
     p.dq = reinterpret_cast<QEntry *>(base + h->sec.dq);
     p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h->sec.flag);
-    qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(p);
+    return QSIM_OK;
+}
+
+int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
+{
+    int rc = attach_workspace(h, ws, bytes, cuda_stream);
+    if (rc != QSIM_OK) return rc;
+    qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
+    h->bound = true;
+    return QSIM_OK;
+}
+
+int qsim_bind_restore(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
+{
+    int rc = attach_workspace(h, ws, bytes, cuda_stream);
+    if (rc != QSIM_OK) return rc;
+    // the end time reached so far is in every replication's record; a state that stopped on an internal error
+    // cannot be resumed
+    RepHeader first;
+    CUDA_TRY(cudaMemcpyAsync(&first, h->par.hdr, sizeof first, cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    if (first.err != 0 || !(first.T_end >= 0.0) || !std::isfinite(first.T_end))
+        return fail(QSIM_ESTATE, "the workspace does not hold a resumable state");
+    h->T_end_abs = first.T_end;
     h->bound = true;
     return QSIM_OK;
 }

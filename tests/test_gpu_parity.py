@@ -171,6 +171,23 @@ def test_resumable_and_event_budget_do_not_change_results():
             assert np.array_equal(a[k], c[k]), ("budget", k)
 
 
+def test_checkpoint_and_resume_in_a_new_handle():
+    from paper_2602_02987_b200 import QSim, QSimError
+    for inp, h1, h2 in ((presets.cfg1(R=4), 700, 500), (presets.cfg4(N=512, R=2), 150, 150)):
+        sim = QSim(inp)
+        sim.run(h1)
+        saved = sim.checkpoint()
+        sim.close()
+        sim = QSim(inp, checkpoint=saved)           # a new handle adopts the saved state and carries on
+        sim.run(h2)
+        got = sim.stats()
+        sim.close()
+        ref, _ = oracle_run(inp, h1 + h2)
+        assert_parity(got, ref, what=f"{inp.name} resumed from a checkpoint")
+    with pytest.raises(QSimError):
+        QSim(presets.cfg1(R=5), checkpoint=saved)
+
+
 def test_replication_offset_shards_compose():
     inp = presets.cfg0(R=8, horizon_iters=2000)
     whole, _ = gpu_run(inp, 2000)
