@@ -254,10 +254,15 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N_>
 __device__ __forceinline__ void cp_async_wait_group() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N_) : "memory"); }
 
-// 1 + #{j < LMAX-1 : thr[j] <= w} by binary search
-__device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, uint32_t w)
+// Coarse index of a threshold table: entry b = #{j < LMAX-1 : thr[j] < b 2^24}, b = 0..256 (built by the host when the
+// tables are uploaded and stored behind them).  A word w with top byte b has its count between entries b and b+1.
+constexpr int LIDX = 260;       // 257 entries, padded
+
+// 1 + #{j < LMAX-1 : thr[j] <= w} by binary search inside the bucket of w's top byte
+__device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, const uint16_t *idx, uint32_t w)
 {
-    uint32_t lo = 0, hi = LMAX - 1;          // the count lies in [lo, hi]
+    const uint32_t b = w >> 24;
+    uint32_t lo = __ldg(idx + b), hi = __ldg(idx + b + 1);          // the count lies in [lo, hi]
     while (lo < hi) {
         const uint32_t mid = (lo + hi) >> 1;
         if (__ldg(thr + mid) <= w) lo = mid + 1; else hi = mid;
@@ -267,7 +272,7 @@ __device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, uint32_t w
 
 // Arrival draw `index` of class i: one Philox block gives the unit exponential and both lengths.
 // (Arguments by value: a reference to the kernel parameters would force a local copy of them.)
-__device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long long global_rep, uint32_t i,
+__device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long long global_rep, uint32_t i, uint32_t I,
                                         unsigned long long index, const uint32_t *tables, uint32_t P, uint32_t D)
 {
     uint32_t w0, w1, w2, w3;
@@ -276,8 +281,9 @@ __device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long l
     ADraw d;
     d.E = -qlog(u53(w0, w1));
     if (tables) {
-        P = table_lookup(tables + ((size_t)i * 2 + 0) * LMAX, w2);
-        D = table_lookup(tables + ((size_t)i * 2 + 1) * LMAX, w3);
+        const uint16_t *idx = reinterpret_cast<const uint16_t *>(tables + (size_t)I * 2 * LMAX);     // behind the tables
+        P = table_lookup(tables + ((size_t)i * 2 + 0) * LMAX, idx + ((size_t)i * 2 + 0) * LIDX, w2);
+        D = table_lookup(tables + ((size_t)i * 2 + 1) * LMAX, idx + ((size_t)i * 2 + 1) * LIDX, w3);
     }
     d.pk = pack_job(P, D, i, 0);
     d.pad = 0;
@@ -376,7 +382,7 @@ struct Sim {
     __device__ __forceinline__ void refill(uint32_t i)
     {
         const unsigned long long base = __shfl_sync(FULL, cs[lane & 7].adraw, i);
-        aring[i * 32 + lane] = make_draw(p.seed, p.rep_offset + rep, i, base + (unsigned long long)lane,
+        aring[i * 32 + lane] = make_draw(p.seed, p.rep_offset + rep, i, p.I, base + (unsigned long long)lane,
                                          p.length_mode == 1 ? p.lengths : nullptr, p.cls[i].P, p.cls[i].D);
         __syncwarp();
         if (lane == (int)i) {

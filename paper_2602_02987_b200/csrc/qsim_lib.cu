@@ -129,6 +129,27 @@ int validate(const qsim_config *cfg, const qsim_class *classes, const double *ra
     return QSIM_OK;
 }
 
+// Threshold tables as the kernels read them: the caller's [I][2][LMAX] words followed by a coarse index per table
+// (entry b = number of thresholds below b 2^24, b = 0..256), which narrows the binary search of a draw to one bucket.
+size_t table_bytes(uint32_t I) { return (size_t)I * 2 * QSIM_LMAX * 4 + (size_t)I * 2 * LIDX * 2; }
+
+std::vector<uint32_t> tables_with_index(const uint32_t *lengths, uint32_t I)
+{
+    std::vector<uint32_t> buf(table_bytes(I) / 4, 0u);
+    std::memcpy(buf.data(), lengths, (size_t)I * 2 * QSIM_LMAX * 4);
+    uint16_t *idx = reinterpret_cast<uint16_t *>(buf.data() + (size_t)I * 2 * QSIM_LMAX);
+    for (uint32_t t = 0; t < I * 2; ++t) {
+        const uint32_t *thr = lengths + (size_t)t * QSIM_LMAX;
+        uint32_t j = 0;
+        for (uint32_t b = 0; b <= 256; ++b) {
+            const uint64_t bound = (uint64_t)b << 24;
+            while (j < QSIM_LMAX - 1 && thr[j] < bound) ++j;
+            idx[(size_t)t * LIDX + b] = (uint16_t)j;
+        }
+    }
+    return buf;
+}
+
 // Instances of the run kernel: (GPUs per lane, feature set).  A problem runs on the smallest instance that
 // contains its features; the fully generic instance takes everything else.
 using RunKernel = void (*)(Params);
@@ -335,9 +356,9 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     cudaError_t e = cudaMalloc(&h->d_blocks, blocks.size() * sizeof(BlockPar));
     if (e == cudaSuccess) e = cudaMemcpy(h->d_blocks, blocks.data(), blocks.size() * sizeof(BlockPar), cudaMemcpyHostToDevice);
     if (e == cudaSuccess && cfg->length_mode == QSIM_LENGTH_TABLE) {
-        const size_t nb = (size_t)cfg->I * 2 * QSIM_LMAX * 4;
-        e = cudaMalloc(&h->d_lengths, nb);
-        if (e == cudaSuccess) e = cudaMemcpy(h->d_lengths, lengths, nb, cudaMemcpyHostToDevice);
+        const std::vector<uint32_t> tab = tables_with_index(lengths, cfg->I);
+        e = cudaMalloc(&h->d_lengths, tab.size() * 4);
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_lengths, tab.data(), tab.size() * 4, cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMallocHost(&h->h_flag, 256);
     if (e == cudaSuccess && h->lay.total > 48u * 1024u) {
@@ -757,7 +778,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     // scratch = [state sections | block table | length tables]
     const size_t off_blocks = h.sec.total;
     const size_t off_lengths = align256(off_blocks + (size_t)cfg->nblk * sizeof(BlockPar));
-    const size_t len_bytes = cfg->length_mode == QSIM_LENGTH_TABLE ? (size_t)cfg->I * 2 * QSIM_LMAX * 4 : 0;
+    const size_t len_bytes = cfg->length_mode == QSIM_LENGTH_TABLE ? table_bytes(cfg->I) : 0;
     const size_t need = off_lengths + len_bytes;
     if (need > QSIM_STATIC_SCRATCH_BYTES)
         return fail(QSIM_EWORKSPACE, "qsim_simulate_static: this problem needs " + std::to_string(need) +
@@ -768,7 +789,10 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     fill_blocks(blocks, *cfg, rates, tg);
     // pageable sources: these copies have returned from the host buffers when the calls return
     CUDA_TRY(cudaMemcpyAsync(base + off_blocks, blocks, (size_t)cfg->nblk * sizeof(BlockPar), cudaMemcpyHostToDevice, stream));
-    if (len_bytes) CUDA_TRY(cudaMemcpyAsync(base + off_lengths, lengths, len_bytes, cudaMemcpyHostToDevice, stream));
+    if (len_bytes) {
+        const std::vector<uint32_t> tab = tables_with_index(lengths, cfg->I);
+        CUDA_TRY(cudaMemcpyAsync(base + off_lengths, tab.data(), len_bytes, cudaMemcpyHostToDevice, stream));
+    }
     p.blocks = reinterpret_cast<const BlockPar *>(base + off_blocks);
     p.lengths = len_bytes ? reinterpret_cast<const uint32_t *>(base + off_lengths) : nullptr;
     p.hdr = reinterpret_cast<RepHeader *>(base + h.sec.hdr);
