@@ -95,7 +95,7 @@ struct SlotRec { double tpf; uint32_t pk; uint32_t pad; };  // request in a deco
 constexpr int STAGE_CAP = 64;                                 // finished-request records waiting for their accounting
 // Accounting of finished requests, one block per warp (merged into the class records at kernel exit)
 struct WarpClassStats { double sYm_out, sYs_out, sum_tpot; unsigned long long tok_in, tok_out; uint32_t done_mixed, done_solo; };
-struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential and packed lengths
+struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential (divided by the rate already when there is one block) and packed lengths
 struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill queue (t = arrival) / decode buffer (t = prefill end)
 
 struct ClassPar { double theta; uint32_t P, D, prio, pad; };
@@ -273,13 +273,14 @@ __device__ __forceinline__ uint32_t table_lookup(const uint32_t *thr, const uint
 // Arrival draw `index` of class i: one Philox block gives the unit exponential and both lengths.
 // (Arguments by value: a reference to the kernel parameters would force a local copy of them.)
 __device__ __noinline__ ADraw make_draw(unsigned long long seed, unsigned long long global_rep, uint32_t i, uint32_t I,
-                                        unsigned long long index, const uint32_t *tables, uint32_t P, uint32_t D)
+                                        unsigned long long index, const uint32_t *tables, uint32_t P, uint32_t D, double Lam)
 {
     uint32_t w0, w1, w2, w3;
     philox((uint32_t)index, (uint32_t)(index >> 32), (STREAM_ARRIVAL << 8) | i, (uint32_t)global_rep, (uint32_t)seed,
            (uint32_t)(seed >> 32), w0, w1, w2, w3);
     ADraw d;
     d.E = -qlog(u53(w0, w1));
+    if (Lam > 0.0) d.E = __ddiv_rn(d.E, Lam);      // one rate for the whole run: the interarrival time itself is stored
     if (tables) {
         const uint16_t *idx = reinterpret_cast<const uint16_t *>(tables + (size_t)I * 2 * LMAX);     // behind the tables
         P = table_lookup(tables + ((size_t)i * 2 + 0) * LMAX, idx + ((size_t)i * 2 + 0) * LIDX, w2);
@@ -382,8 +383,10 @@ struct Sim {
     __device__ __forceinline__ void refill(uint32_t i)
     {
         const unsigned long long base = __shfl_sync(FULL, cs[lane & 7].adraw, i);
+        // with a single block the class's rate never changes and the division E / Lambda is done here, 32 at a time
+        const double Lam1 = f_blocks() ? 0.0 : __dmul_rn((double)p.N, p.blocks[0].rate[i]);
         aring[i * 32 + lane] = make_draw(p.seed, p.rep_offset + rep, i, p.I, base + (unsigned long long)lane,
-                                         p.length_mode == 1 ? p.lengths : nullptr, p.cls[i].P, p.cls[i].D);
+                                         p.length_mode == 1 ? p.lengths : nullptr, p.cls[i].P, p.cls[i].D, Lam1);
         __syncwarp();
         if (lane == (int)i) {
             cs[i].adraw = base + 32ull;
@@ -426,7 +429,7 @@ struct Sim {
             }
             const ADraw d = aring[lane * 32 + ring_pos];
             ring_pos++; ring_n--;
-            const double cand = __dadd_rn(t0, __ddiv_rn(d.E, Lam));
+            const double cand = __dadd_rn(t0, f_blocks() ? __ddiv_rn(d.E, Lam) : d.E);
             if (has_next && cand >= block_start(b + 1)) {
                 ++b; t0 = block_start(b);
                 continue;
