@@ -33,9 +33,9 @@ UNIT = "server-iterations/s"
 JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
                            # decode-buffer pass, each written and read once at 32-byte sector granularity
 # DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from an ncu capture of a 2000-iteration
-# launch (dram__bytes_read.sum + dram__bytes_write.sum = 733.4 MB for 1.415e8 iterations); traffic grows with the
+# launch (dram__bytes_read.sum + dram__bytes_write.sum = 734.9 MB for 1.415e8 iterations); traffic grows with the
 # iterations of a launch, so a full launch is that figure times its iterations
-NCU_DRAM_BYTES_PER_ITER = 733.4e6 / 1.415e8
+NCU_DRAM_BYTES_PER_ITER = 734.9e6 / 1.415e8
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
 R_PER_GPU = 1024
 
