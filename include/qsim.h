@@ -202,6 +202,15 @@ int qsim_sync(qsim_t *h);
 int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint64_t *hist_ttft,
                uint64_t *hist_tpot);
 
+/*
+ * Latency percentiles over all replications from the histograms (cfg.hist must be 1): for each class i and each
+ * quantile q[k] in (0, 1], ttft[i * nq + k] and tpot[i * nq + k] receive the lower edge, in seconds, of the first
+ * histogram bin at which the cumulative count reaches ceil(q[k] * total); NaN for a class without samples.  Bins are
+ * 32 per octave, so a percentile is exact to 2.2 % [the paper reports mean / P95 / P99 TTFT and TPOT, Section 6.2,
+ * without defining an estimator].  [host] q[nq], ttft[I * nq], tpot[I * nq].  Synchronises the stream.
+ */
+int qsim_latency_percentiles(qsim_t *h, const double *q, uint32_t nq, double *ttft, double *tpot);
+
 /* Zero all counters, integrals and histograms and restart T_elapsed; the simulated state is kept. */
 int qsim_reset_stats(qsim_t *h);
 

@@ -240,6 +240,28 @@ class OracleSim:
             pass
 
 
+def bin_lower_edge(b):
+    """Smallest latency (seconds) that falls into histogram bin b: the double whose top 17 bits are b + ((1023-20) << 5)."""
+    bits = (np.asarray(b, np.uint64) + np.uint64((1023 - 20) << 5)) << np.uint64(47)
+    return bits.view(np.float64)
+
+
+def hist_percentiles(hist, q) -> np.ndarray:
+    """Percentiles of a latency histogram [R, I, NBIN] pooled over replications: for class i and quantile q the lower
+    edge of the first bin whose cumulative count reaches ceil(q * total); NaN without samples.  Returns [I, len(q)]."""
+    pooled = hist.sum(axis=0).astype(np.int64)               # [I, NBIN]
+    out = np.full((pooled.shape[0], len(q)), np.nan)
+    for i in range(pooled.shape[0]):
+        total = int(pooled[i].sum())
+        if total == 0:
+            continue
+        cum = np.cumsum(pooled[i])
+        for k, qq in enumerate(q):
+            need = min(max(int(np.ceil(qq * total)), 1), total)
+            out[i, k] = bin_lower_edge(np.array([np.searchsorted(cum, need, side="left")]))[0]
+    return out
+
+
 def run_oracle(inp, horizon_iters: int, rep_lo: int = 0, rep_hi: int | None = None) -> dict:
     sim = OracleSim(inp)
     sim.run(horizon_iters, rep_lo, rep_hi)

@@ -20,7 +20,7 @@ EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim
            "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
            "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
            "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error",
-           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats", "qsim_bind_restore")
+           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats", "qsim_bind_restore", "qsim_latency_percentiles")
 
 
 class QSimError(RuntimeError):
@@ -92,6 +92,7 @@ def load_library():
         L.qsim_workspace_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.qsim_bind.argtypes = [vp, vp, C.c_size_t, vp]
         L.qsim_bind_restore.argtypes = [vp, vp, C.c_size_t, vp]
+        L.qsim_latency_percentiles.argtypes = [vp, vp, C.c_uint32, vp, vp]
         L.qsim_run.argtypes = [vp, C.c_uint64]
         L.qsim_run_until.argtypes = [vp, C.c_double]
         L.qsim_set_injected.argtypes = [vp, vp, vp, C.c_uint64]
@@ -218,6 +219,13 @@ class QSim:
         self.sync()
         off = self._base - self.ws.data_ptr()
         return self.ws[off:off + self.workspace_bytes].cpu()
+
+    def latency_percentiles(self, q):
+        """(ttft, tpot), each [I, len(q)] seconds: lower edge of the histogram bin where the cumulative count reaches q."""
+        q = np.ascontiguousarray(q, np.float64)
+        ttft = np.zeros((self.inp.I, q.shape[0])); tpot = np.zeros((self.inp.I, q.shape[0]))
+        _check(self.L.qsim_latency_percentiles(self.h, _ptr(q), q.shape[0], _ptr(ttft), _ptr(tpot)))
+        return ttft, tpot
 
     def set_event_budget(self, n: int) -> None:
         _check(self.L.qsim_set_event_budget(self.h, int(n)))

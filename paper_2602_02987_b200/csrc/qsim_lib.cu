@@ -547,6 +547,46 @@ int qsim_layout_info(const qsim_t *h, uint64_t out[4])
     return QSIM_OK;
 }
 
+int qsim_latency_percentiles(qsim_t *h, const double *q, uint32_t nq, double *ttft, double *tpot)
+{
+    if (!h || !q || !ttft || !tpot || nq == 0) return fail(QSIM_EINVAL, "null argument");
+    if (!h->bound) return fail(QSIM_ESTATE, "qsim_latency_percentiles before qsim_bind");
+    if (!h->cfg.hist) return fail(QSIM_EINVAL, "percentiles need cfg.hist = 1");
+    for (uint32_t k = 0; k < nq; ++k)
+        if (!(q[k] > 0.0 && q[k] <= 1.0)) return fail(QSIM_EINVAL, "quantiles must lie in (0, 1]");
+    const uint32_t R = h->cfg.R, I = h->cfg.I;
+    std::vector<uint32_t> raw((size_t)R * I * 2 * NBIN);
+    CUDA_TRY(cudaMemcpyAsync(raw.data(), h->par.hist_mem, raw.size() * 4, cudaMemcpyDeviceToHost, h->stream));
+    CUDA_TRY(cudaStreamSynchronize(h->stream));
+    std::vector<uint64_t> sum(NBIN);
+    for (uint32_t i = 0; i < I; ++i)
+        for (int kind = 0; kind < 2; ++kind) {
+            std::fill(sum.begin(), sum.end(), 0ull);
+            uint64_t total = 0;
+            for (uint32_t r = 0; r < R; ++r) {
+                const uint32_t *src = raw.data() + (((size_t)r * I + i) * 2 + kind) * NBIN;
+                for (int b = 0; b < NBIN; ++b) { sum[b] += src[b]; total += src[b]; }
+            }
+            double *out = kind == 0 ? ttft : tpot;
+            for (uint32_t k = 0; k < nq; ++k) {
+                double v = std::nan("");
+                if (total > 0) {
+                    uint64_t need = (uint64_t)std::ceil(q[k] * (double)total);
+                    if (need < 1) need = 1;
+                    if (need > total) need = total;
+                    uint64_t cum = 0;
+                    int b = 0;
+                    for (; b < NBIN; ++b) { cum += sum[b]; if (cum >= need) break; }
+                    // lower edge of bin b: the double whose top bits are b + ((1023 - 20) << 5)
+                    const uint64_t bits = ((uint64_t)b + ((uint64_t)(1023 - 20) << 5)) << 47;
+                    std::memcpy(&v, &bits, sizeof v);
+                }
+                out[(size_t)i * nq + k] = v;
+            }
+        }
+    return QSIM_OK;
+}
+
 int qsim_launch_count(const qsim_t *h, uint64_t *launches)
 {
     if (!h || !launches) return fail(QSIM_EINVAL, "null argument");

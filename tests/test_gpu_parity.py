@@ -122,6 +122,25 @@ def test_cfg3_subset_block_tables_and_histograms():
     assert st["hist_tpot"].sum() == (st["done_mixed"] + st["done_solo"]).sum()
 
 
+def test_latency_percentiles_from_the_histograms():
+    from oracle import OracleSim, hist_percentiles
+    from paper_2602_02987_b200 import QSim, QSimError
+    inp = presets.cfg3(N=96, R=4, block_len=1.0)
+    H = inp.meta["horizon_iters"]
+    q = [0.5, 0.95, 0.99]
+    sim = QSim(inp); sim.run(H)
+    ttft, tpot = sim.latency_percentiles(q)
+    sim.close()
+    o = OracleSim(inp); o.run(H); st = o.stats(); o.close()
+    assert np.array_equal(ttft, hist_percentiles(st["hist_ttft"], q))
+    assert np.array_equal(tpot, hist_percentiles(st["hist_tpot"], q))
+    assert (ttft[:, 0] <= ttft[:, 2]).all() and (tpot > 0).all()
+    nohist = QSim(presets.cfg0(R=2)); nohist.run(100)
+    with pytest.raises(QSimError):
+        nohist.latency_percentiles(q)
+    nohist.close()
+
+
 def test_cfg4_subset_sli_router_constrained_targets():
     for N in (16, 256):
         inp = presets.cfg4(N=N, R=3)

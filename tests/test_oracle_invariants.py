@@ -147,3 +147,30 @@ def test_reset_stats_discards_warm_up_but_keeps_state():
     assert np.allclose(s0["area_X"] + s1["area_X"], s2["area_X"], rtol=1e-12)
     assert np.allclose(s0["T_elapsed"] + s1["T_elapsed"], s2["T_elapsed"], rtol=1e-15)
     a.close(); b.close()
+
+
+def test_histogram_percentiles_bracket_the_exact_order_statistics():
+    # TTFT / TPOT of every request re-derived from the event trace; the histogram percentile is the lower edge of the
+    # bin that holds the ceil(q n)-th smallest latency
+    from oracle import bin_lower_edge, hist_percentiles
+    inp = presets.cfg0(R=2, horizon_iters=1500).with_(hist=1)
+    sim = OracleSim(inp, trace_cap=2_000_000)
+    sim.run(1500)
+    tr, st = sim.trace(), sim.stats()
+    q = [0.5, 0.9, 0.99, 1.0]
+    pt, pp = hist_percentiles(st["hist_ttft"], q), hist_percentiles(st["hist_tpot"], q)
+    jobs = {}
+    for r in range(inp.R):
+        rp = Replay(inp, tr, rep=r).run(None)
+        for (c, j), rec in rp.jobs.items():
+            jobs[(r, c, j)] = rec
+    for i in range(inp.I):
+        ttft = sorted(v["t_pf"] - v["t_arr"] for (r, c, j), v in jobs.items() if c == i and "t_pf" in v)
+        tpot = sorted((v["t_done"] - v["t_pf"]) / v["D"] for (r, c, j), v in jobs.items() if c == i and "t_done" in v)
+        assert len(ttft) == st["hist_ttft"][:, i].sum() and len(tpot) == st["hist_tpot"][:, i].sum()
+        for k, qq in enumerate(q):
+            for xs, p in ((ttft, pt[i, k]), (tpot, pp[i, k])):
+                x = xs[int(np.ceil(qq * len(xs))) - 1]
+                b = int(np.searchsorted(bin_lower_edge(np.arange(1024)), p, side="right")) - 1
+                assert bin_lower_edge(np.array([b]))[0] == p
+                assert p <= x < bin_lower_edge(np.array([b + 1]))[0] and x / p < 1.0 + 1.0 / 32 + 1e-12
