@@ -36,6 +36,14 @@ JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue ent
 # launch (dram__bytes_read.sum + dram__bytes_write.sum = 734.9 MB for 1.415e8 iterations); traffic grows with the
 # iterations of a launch, so a full launch is that figure times its iterations
 NCU_DRAM_BYTES_PER_ITER = 734.9e6 / 1.415e8
+# warp instructions per simulated server-iteration of the same capture (smsp__inst_executed.sum = 3.224e10)
+NCU_WARP_INST_PER_ITER = 3.224e10 / 1.415e8
+# exponential-service kernel, capture of a 1-second launch at R = 28416: 3.195e9 warp instructions and
+# 118.3 MB + 41.1 MB of DRAM traffic (the replication records, independent of the simulated time) for 6.254e7 jumps
+NCU_CTMC_WARP_INST_PER_JUMP = 3.195e9 / 6.254e7
+NCU_CTMC_DRAM_BYTES_PER_LAUNCH = 159.4e6
+# issue peak of the GPU: 148 SMs x 4 schedulers x one warp instruction per cycle at the maximum SM clock
+ISSUE_PEAK = 148 * 4 * 1.965e9
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
 R_PER_GPU = 1024
 
@@ -195,6 +203,12 @@ def run_ctmc(args):
                "unit": "jumps/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
                "ms_per_step": float(tmax[0]) / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                "dtype": "f64", "data": "synthetic", "gpu_launches": int(my[2]),
+               # no memory or tensor roofline applies: the records are read and written once per launch; the kernel is
+               # bound by instruction issue of dependent chains, so the fraction is taken against the issue peak
+               "roofline": {"bound": "alu", "achieved": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3),
+                            "peak": ISSUE_PEAK, "unit": "warp-inst/s",
+                            "frac": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3) / ISSUE_PEAK,
+                            "traffic": NCU_CTMC_DRAM_BYTES_PER_LAUNCH if (count == 28416 and world == 1) else None},
                "config": {"workload": f"exponential-service model, paper synthetic instance, n={n}, SLI-aware router, "
                                       f"{R} replications per GPU, {dT} s of simulated time per step"}}
         if not args.no_cpu_baseline and world == 1:
@@ -363,7 +377,9 @@ def main():
                          "traffic_source": "no capture for this workload" if other else "ncu capture of a 2000-iteration launch, scaled by iterations",
                          "peak_kind": peak_kind,
                          "bytes_per_iteration": JOB_BYTES * jobs / iters,
-                         "note": "latency/issue-bound event chain; HBM fraction is the contract figure"},
+                         "note": "latency/issue-bound event chain; HBM fraction is the contract figure",
+                         "issue": None if other else {"achieved": NCU_WARP_INST_PER_ITER * value / world, "peak": ISSUE_PEAK,
+                                                      "unit": "warp-inst/s", "frac": NCU_WARP_INST_PER_ITER * value / world / ISSUE_PEAK}},
             "clocks": clocks, "gpu_launches": int(n_launch), "wall_s": wall,
         }
         if e2e:
