@@ -38,10 +38,11 @@ JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue ent
 NCU_DRAM_BYTES_PER_ITER = 734.9e6 / 1.415e8
 # warp instructions per simulated server-iteration of the same capture (smsp__inst_executed.sum = 3.224e10)
 NCU_WARP_INST_PER_ITER = 3.224e10 / 1.415e8
-# exponential-service kernel, capture of a 1-second launch at R = 28416: 3.195e9 warp instructions and
-# 118.3 MB + 41.1 MB of DRAM traffic (the replication records, independent of the simulated time) for 6.254e7 jumps
-NCU_CTMC_WARP_INST_PER_JUMP = 3.195e9 / 6.254e7
-NCU_CTMC_DRAM_BYTES_PER_LAUNCH = 159.4e6
+# exponential-service kernel, capture of a 1-second launch at R = 37888: 4.238e9 warp instructions for 8.339e7 jumps and
+# 160.5 MB + 191.4 MB of DRAM traffic (the replication records once, plus the counters and integrals that are added to in
+# place; the latter grows with the simulated time, so a longer launch has no traffic figure)
+NCU_CTMC_WARP_INST_PER_JUMP = 4.238e9 / 8.339e7
+NCU_CTMC_DRAM_BYTES_PER_LAUNCH = 351.9e6
 # issue peak of the GPU: 148 SMs x 4 schedulers x one warp instruction per cycle at the maximum SM clock
 ISSUE_PEAK = 148 * 4 * 1.965e9
 HORIZON = 100_000          # iterations of horizon per step (cfg1)
@@ -163,7 +164,7 @@ def run_reference(args, workload):
 
 def run_ctmc(args):
     """Second workload: the exponential-service model of Section 2.3 on the paper's two-class synthetic instance,
-    n = 1000 GPUs, SLI-aware router, 28416 replications per GPU (one resident wave: 148 SMs x 6 blocks x 32 threads);
+    n = 1000 GPUs, SLI-aware router, 37888 replications per GPU (one resident wave: 148 SMs x 8 blocks x 32 threads);
     one step advances every replication by 10 s."""
     import torch
     import torch.distributed as dist
@@ -177,7 +178,7 @@ def run_ctmc(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    n, R, dT = 1000, 28416, args.ctmc_seconds
+    n, R, dT = 1000, 37888, args.ctmc_seconds
     count, offset = shard(R * world, world, rank)
     inp = presets.ctmc_instance(n=n, R=count, router=ROUTER_SLI).with_(rep_offset=offset)
     sim = QSimCTMC(inp, device=f"cuda:{local}")
@@ -208,7 +209,7 @@ def run_ctmc(args):
                "roofline": {"bound": "alu", "achieved": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3),
                             "peak": ISSUE_PEAK, "unit": "warp-inst/s",
                             "frac": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3) / ISSUE_PEAK,
-                            "traffic": NCU_CTMC_DRAM_BYTES_PER_LAUNCH if (count == 28416 and world == 1) else None},
+                            "traffic": NCU_CTMC_DRAM_BYTES_PER_LAUNCH if (count == 37888 and world == 1 and dT == 1.0) else None},
                "config": {"workload": f"exponential-service model, paper synthetic instance, n={n}, SLI-aware router, "
                                       f"{R} replications per GPU, {dT} s of simulated time per step"}}
         if not args.no_cpu_baseline and world == 1:

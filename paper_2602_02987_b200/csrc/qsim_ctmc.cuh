@@ -51,7 +51,9 @@ struct CtmcParams {
 };
 
 // Working copy of one replication in shared memory: 8-byte words, word w of thread t at [w * blockDim + t]
-// (consecutive threads hit consecutive banks).  Only the I classes in use take space: 5 + 62 I words.
+// (consecutive threads hit consecutive banks).  Only the I classes in use take space: 5 + 47 I words.  The event
+// counters and the time integrals are only ever added to, so they stay in the global record and take
+// fire-and-forget additions (one thread, one address: applied in program order, so the sums are deterministic).
 struct CtmcWords {
     unsigned long long *base;   // this thread's word 0
     uint32_t stride, I;
@@ -59,10 +61,8 @@ struct CtmcWords {
     __device__ __forceinline__ uint32_t clk(uint32_t k, uint32_t i, uint32_t f) const { return W_BASE + (k * I + i) * 5u + f; }   // f: acc, lvl, t_last, t_fire, m
     __device__ __forceinline__ uint32_t count(uint32_t c, uint32_t i) const { return W_BASE + 35u * I + c * I + i; }             // c: Qp, X, Qd0, Qd1, Ym, Ys
     __device__ __forceinline__ uint32_t sli(uint32_t i) const { return W_BASE + 41u * I + i; }
-    __device__ __forceinline__ uint32_t area(uint32_t a, uint32_t i) const { return W_BASE + 42u * I + a * I + i; }
-    __device__ __forceinline__ uint32_t area_t(uint32_t a, uint32_t i) const { return W_BASE + 47u * I + a * I + i; }
-    __device__ __forceinline__ uint32_t cnt(uint32_t i, uint32_t c) const { return W_BASE + 52u * I + i * 10u + c; }
-    __host__ __device__ static uint32_t words(uint32_t I) { return 5u + 62u * I; }
+    __device__ __forceinline__ uint32_t area_t(uint32_t a, uint32_t i) const { return W_BASE + 42u * I + a * I + i; }
+    __host__ __device__ static uint32_t words(uint32_t I) { return 5u + 47u * I; }
     __device__ __forceinline__ unsigned long long u(uint32_t w) const { return base[(size_t)w * stride]; }
     __device__ __forceinline__ void su(uint32_t w, unsigned long long v) const { base[(size_t)w * stride] = v; }
     __device__ __forceinline__ double d(uint32_t w) const { return __longlong_as_double((long long)u(w)); }
@@ -73,12 +73,13 @@ enum { CQ_QP = 0, CQ_X = 1, CQ_QD0 = 2, CQ_QD1 = 3, CQ_YM = 4, CQ_YS = 5 };
 struct CtmcSim {
     const CtmcParams &p;
     const CtmcWords W;
+    CtmcRep &G;                 // the record in global memory: counters and integrals are added to in place
     uint8_t *ring0, *ring1;
     const uint32_t rep;
     uint32_t totX, totYm, totYs, err;
 
-    __device__ CtmcSim(const CtmcParams &p_, const CtmcWords &W_, uint32_t rep_)
-        : p(p_), W(W_), ring0(p_.rings + (size_t)rep_ * 2 * p_.qcap), ring1(ring0 + p_.qcap), rep(rep_), totX(0), totYm(0), totYs(0), err(0) {}
+    __device__ CtmcSim(const CtmcParams &p_, const CtmcWords &W_, CtmcRep &G_, uint32_t rep_)
+        : p(p_), W(W_), G(G_), ring0(p_.rings + (size_t)rep_ * 2 * p_.qcap), ring1(ring0 + p_.qcap), rep(rep_), totX(0), totYm(0), totYs(0), err(0) {}
 
     __device__ __forceinline__ uint32_t stream_of(uint32_t k, uint32_t i) const
     {
@@ -100,7 +101,7 @@ struct CtmcSim {
     __device__ __forceinline__ uint32_t cq(uint32_t c, uint32_t i) const { return (uint32_t)W.u(W.count(c, i)); }
     __device__ __forceinline__ void touch(uint32_t a, uint32_t i, uint32_t count, double t)
     {
-        W.sd(W.area(a, i), __dadd_rn(W.d(W.area(a, i)), __dmul_rn((double)count, __dsub_rn(t, W.d(W.area_t(a, i))))));
+        atomicAdd(&G.area[a][i], __dmul_rn((double)count, __dsub_rn(t, W.d(W.area_t(a, i)))));
         W.sd(W.area_t(a, i), t);
     }
     // the count that process k of class i runs on changes from n_old to n_new at time t
@@ -153,7 +154,7 @@ struct CtmcSim {
         touch(CA_QD, i, q0 + q1, t);
         W.su(W.count(pool ? CQ_QD1 : CQ_QD0, i), v);
     }
-    __device__ __forceinline__ void bump(uint32_t i, uint32_t c) { W.su(W.cnt(i, c), W.u(W.cnt(i, c)) + 1ull); }
+    __device__ __forceinline__ void bump(uint32_t i, uint32_t c) { atomicAdd(&G.cnt[i][c], 1ull); }
 
     // Section 4.1 occupancy gate (xi_i = (X_i - n x*_i)/x*_i, ties to the largest Q_p,i - n q*_p,i) or the
     // Section 5.1.1 priority gate (smallest static rank); ties to the lowest class index
@@ -337,8 +338,7 @@ struct CtmcSim {
             W.su(W.count(CQ_QP, i), S.Qp[i]); W.su(W.count(CQ_X, i), S.X[i]); W.su(W.count(CQ_QD0, i), S.Qd[0][i]);
             W.su(W.count(CQ_QD1, i), S.Qd[1][i]); W.su(W.count(CQ_YM, i), S.Ym[i]); W.su(W.count(CQ_YS, i), S.Ys[i]);
             W.su(W.sli(i), S.sli_ord[i]);
-            for (uint32_t a = 0; a < CA_N; ++a) { W.sd(W.area(a, i), S.area[a][i]); W.sd(W.area_t(a, i), S.area_t[a][i]); }
-            for (uint32_t c = 0; c < CC_N; ++c) W.su(W.cnt(i, c), S.cnt[i][c]);
+            for (uint32_t a = 0; a < CA_N; ++a) W.sd(W.area_t(a, i), S.area_t[a][i]);
         }
     }
     __device__ void store(CtmcRep &S) const
@@ -355,8 +355,7 @@ struct CtmcSim {
             S.Qp[i] = cq(CQ_QP, i); S.X[i] = cq(CQ_X, i); S.Qd[0][i] = cq(CQ_QD0, i); S.Qd[1][i] = cq(CQ_QD1, i);
             S.Ym[i] = cq(CQ_YM, i); S.Ys[i] = cq(CQ_YS, i);
             S.sli_ord[i] = W.u(W.sli(i));
-            for (uint32_t a = 0; a < CA_N; ++a) { S.area[a][i] = W.d(W.area(a, i)); S.area_t[a][i] = W.d(W.area_t(a, i)); }
-            for (uint32_t c = 0; c < CC_N; ++c) S.cnt[i][c] = W.u(W.cnt(i, c));
+            for (uint32_t a = 0; a < CA_N; ++a) S.area_t[a][i] = W.d(W.area_t(a, i));
         }
     }
 };
@@ -371,7 +370,7 @@ __global__ void __launch_bounds__(64) qsim_ctmc_kernel(CtmcParams p)
     CtmcRep &S = p.reps[rep];
     CtmcWords W;
     W.base = ctmc_sm + threadIdx.x; W.stride = blockDim.x; W.I = p.I;
-    CtmcSim sim(p, W, rep);
+    CtmcSim sim(p, W, S, rep);
     if (p.init) {
         uint32_t *w = reinterpret_cast<uint32_t *>(&S);
         for (uint32_t o = 0; o < sizeof(CtmcRep) / 4; ++o) w[o] = 0;
@@ -431,7 +430,7 @@ CtmcSections ctmc_sections(const qsim_ctmc_config &c)
 }
 
 // one warp per block: many small blocks spread the replications over all SMs; the working copies of a block's
-// replications take 32 (5 + 62 I) 8-byte words of shared memory
+// replications take 32 (5 + 47 I) 8-byte words of shared memory
 int ctmc_launch_shape(uint32_t I, uint32_t &threads, size_t &smem)
 {
     threads = 32;

@@ -44,10 +44,10 @@ def test_ctmc_parity_element_by_element(router, gate, theta, lam):
 
 def test_ctmc_full_size_in_the_bench_launch_configuration():
     from oracle import run_ctmc_oracle
-    inp = presets.ctmc_instance(n=1000, R=28416, router=ROUTER_SLI)       # what `bench.py --workload ctmc` times
+    inp = presets.ctmc_instance(n=1000, R=37888, router=ROUTER_SLI)       # what `bench.py --workload ctmc` times
     gpu = gpu_run(inp, [10.0, 20.0])
     # sampled replications against the oracle (the Philox counter holds the global replication index)
-    for r in (0, 14209, 28415):
+    for r in (0, 18945, 37887):
         ref = run_ctmc_oracle(inp.with_(rep_offset=r, R=1), 20.0)
         for k in CTMC_COUNTERS + CTMC_STATE + ("events",):
             assert np.array_equal(gpu[k][r:r + 1], ref[k]), (r, k)
