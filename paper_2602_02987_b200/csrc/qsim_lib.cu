@@ -162,6 +162,11 @@ void add_variants(std::vector<RunVariant> &v)
     v.push_back({SPL, F_SLOTS | F_OCC, qsim_run_kernel<SPL, F_SLOTS | F_OCC>});
     v.push_back({SPL, F_SLOTS | F_OCC | F_ABANDON, qsim_run_kernel<SPL, F_SLOTS | F_OCC | F_ABANDON>});
     v.push_back({SPL, F_SLOTS | F_OCC | F_ABANDON | F_RANDOM, qsim_run_kernel<SPL, F_SLOTS | F_OCC | F_ABANDON | F_RANDOM>});
+    // occupancy gate with abandonment when the finish stamps do not fit on chip (large B), and the SLI-aware router with
+    // histograms in both slot modes
+    v.push_back({SPL, F_OCC | F_ABANDON, qsim_run_kernel<SPL, F_OCC | F_ABANDON>});
+    v.push_back({SPL, F_OCC | F_ABANDON | F_SLI | F_HIST, qsim_run_kernel<SPL, F_OCC | F_ABANDON | F_SLI | F_HIST>});
+    v.push_back({SPL, F_SLOTS | F_OCC | F_ABANDON | F_SLI | F_HIST, qsim_run_kernel<SPL, F_SLOTS | F_OCC | F_ABANDON | F_SLI | F_HIST>});
     v.push_back({SPL, F_GENERIC, qsim_run_kernel<SPL, F_GENERIC>});
 }
 
@@ -172,6 +177,9 @@ const std::vector<RunVariant> &run_variants()
         add_variants<1>(v);
         add_variants<2>(v);
         add_variants<4>(v);
+        // one warp, run-time row count (129..511 GPUs)
+        v.push_back({0, F_OCC | F_ABANDON, qsim_run_kernel<0, F_OCC | F_ABANDON>});
+        v.push_back({0, F_OCC | F_ABANDON | F_SLI | F_HIST, qsim_run_kernel<0, F_OCC | F_ABANDON | F_SLI | F_HIST>});
         v.push_back({0, F_GENERIC, qsim_run_kernel<0, F_GENERIC>});
         // several warps per replication (large clusters): instances for the occupancy gate with abandonment under
         // the solo-first and (with histograms) the SLI-aware router, the priority gate with blocks and histograms, and the generic one
@@ -242,10 +250,10 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
     for (const RunVariant &v : run_variants()) {
         if (v.spl < 0) continue;                            // the multi-warp instance is chosen by the caller
         if (v.spl != 0 && v.spl < rows) continue;          // too few GPUs per lane
-        if (v.spl == 0 && !generic) generic = &v;
-        if (v.spl == 0) continue;
-        // smallest row count that fits; among those the feature set with the fewest extras
-        int spl_fit = rows <= 1 ? 1 : (rows <= 2 ? 2 : 4);
+        if (v.spl == 0 && (v.feat & F_GENERIC)) { generic = &v; continue; }
+        // smallest row count that fits (0 = run-time row count, beyond four rows); among those the feature set with
+        // the fewest extras
+        int spl_fit = rows <= 1 ? 1 : (rows <= 2 ? 2 : (rows <= 4 ? 4 : 0));
         if (v.spl != spl_fit) continue;
         if (v.feat & F_GENERIC) { if (!best) { best = &v; best_bits = 98; } continue; }
         // mode bits (router, placement, gate, histograms) select code and must match exactly; capability bits

@@ -142,9 +142,10 @@ def test_latency_percentiles_from_the_histograms():
 
 
 def test_cfg4_subset_sli_router_constrained_targets():
-    for N in (16, 256):
+    # N = 16: finish stamps on chip; N = 64, 128: global slot lists with 2 and 4 GPUs per lane; N = 256: run-time row count
+    for N, H in ((16, 1200), (64, 800), (128, 500), (256, 500)):
         inp = presets.cfg4(N=N, R=3)
-        check(inp, 1200 if N == 16 else 500)
+        check(inp, H)
 
 
 def test_multi_warp_instances_large_clusters():
