@@ -165,6 +165,14 @@ def test_multi_warp_instances_large_clusters():
     assert_parity(g2, g, what="generic multi-warp instance")
 
 
+@pytest.mark.parametrize("preset,N,H", [("cfg4", 40, 900), ("cfg4", 100, 600), ("cfg4", 300, 300), ("cfg2", 33, 900),
+                                         ("cfg2", 129, 500), ("cfg2", 520, 200)])
+def test_ragged_cluster_sizes(preset, N, H):
+    # cluster sizes that do not fill their last row of 32 GPUs, on every row-count variant of the specialised instances
+    inp = getattr(presets, preset)(N=N, R=3)
+    check(inp, H)
+
+
 def test_large_n_one_replication():
     inp = presets.cfg4(N=4096, R=1)
     check(inp, 60)
