@@ -95,3 +95,22 @@ def test_ctmc_degenerate_cases():
     # an end time of zero processes nothing
     z = gpu_run(base, [0.0])
     assert z["events"].sum() == 0 and z["T_elapsed"].max() == 0.0
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_ctmc_random_configuration(seed):
+    # random rates, targets and capacities (not an LP plan): parity does not depend on the inputs making sense
+    from oracle import run_ctmc_oracle
+    from qsim_inputs.spec import CtmcInputs
+    rng = np.random.default_rng(700 + seed)
+    I = int(rng.integers(1, 9)); N = int(rng.integers(1, 40)); M = int(rng.integers(0, N + 1)); B = int(rng.integers(1, 20))
+    inp = CtmcInputs(name=f"rnd{seed}", I=I, N=N, M=M, B=B, R=int(rng.choice([1, 31, 33, 65])), gate=int(rng.integers(0, 2)),
+                     router=int(rng.integers(0, 2)), qcap=int(rng.choice([1, 3, 64])), seed=seed,
+                     lam=rng.random(I) * 0.6, theta=rng.choice([0.0, 0.1, 1.0], I), mu_p=0.5 + rng.random(I) * 3,
+                     mu_m=0.05 + rng.random(I), mu_s=0.1 + rng.random(I) * 2, P=np.full(I, 100.0), D=np.full(I, 50.0),
+                     prices=np.array([1.0, 2.0]), prio_rank=rng.permutation(I).astype(np.uint32),
+                     xstar=rng.choice([0.0, 0.05, 0.2], I), n_xstar=rng.random(I) * N * 0.2, n_qpstar=rng.random(I) * 3,
+                     p_solo=rng.choice([0.0, 0.3, 1.0], I))
+    inp.validate()
+    ref = run_ctmc_oracle(inp, 40.0)
+    compare(gpu_run(inp, [11.0, 40.0]), ref, inp.name)
