@@ -28,7 +28,10 @@
  * Parity pins: Philox against its published known-answer vectors; qlog against libm; the event
  * dynamics against hand-computed trajectories, flow-balance identities (Eq. (15)-(20)), capacity
  * constraints (Eq. (12)-(14)), a finite-horizon Little identity, a no-contention closed form and
- * convergence of revenue to the LP optimum.  The trace-replay revenue tables the paper prints need
+ * convergence of revenue to the LP optimum; the KV-token bookkeeping of the KV slope and the role change of
+ * a GPU at a block end against hand-computed trajectories and the request-by-request replay; the uniformity
+ * of random placement and of the abandoning request by chi-square; broken copies of this file must fail
+ * these pins (tests/test_oracle_kv_and_block_switch.py).  The trace-replay revenue tables the paper prints need
  * its production traces: parity unpinned for those numbers.
  */
 #ifndef QSIM_ORACLE_H

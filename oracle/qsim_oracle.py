@@ -62,23 +62,29 @@ class TraceRec(C.Structure):
                 ("cls", C.c_int32), ("server", C.c_int32), ("rep", C.c_int32)]
 
 
+def compile_oracle(src: str, out: str) -> str:
+    """gcc command of the oracle: every fp operation stays a single rounded IEEE double operation."""
+    cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+           "-Wall", "-Wextra", "-I", _HERE, "-o", out, src, "-lm"]
+    subprocess.run(cmd, check=True, cwd=_HERE)
+    return out
+
+
 def build_oracle(force: bool = False) -> str:
-    """Compile the oracle with gcc; every fp operation stays a single rounded IEEE double operation."""
+    """Compile the oracle with gcc when its source is newer than the library."""
     stale = (not os.path.exists(_LIB)) or any(os.path.getmtime(p) > os.path.getmtime(_LIB) for p in (_SRC, _HDR))
     if force or stale:
-        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
-               "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
-        subprocess.run(cmd, check=True, cwd=_HERE)
+        compile_oracle(_SRC, _LIB)
     return _LIB
 
 
 _lib = None
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        L = C.CDLL(build_oracle())
+def load_oracle(path: str):
+    """Load an oracle library and declare its entry points (tests load deliberately broken copies this way)."""
+    if True:
+        L = C.CDLL(path)
         L.orc_create.restype = C.c_int
         L.orc_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Config), C.POINTER(Class), C.c_void_p,
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Targets), C.c_void_p, C.c_void_p]
@@ -107,7 +113,13 @@ def lib():
         L.orc_table_length.argtypes = [C.c_void_p, C.c_uint32]
         L.orc_hist_bin.restype = C.c_uint32
         L.orc_hist_bin.argtypes = [C.c_double]
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = load_oracle(build_oracle())
     return _lib
 
 

@@ -31,6 +31,10 @@ class Replay:
         self.jobs = {}                                 # (cls, job) -> dict of timestamps and lengths
         self.sojourn = defaultdict(float)              # stage -> sum over jobs of time in stage (up to T)
         self.n_events = 0
+        # (rank, size) of every choice the paper makes uniformly at random: the GPU inside the eligible tier
+        # (Section 4.1) and the request that abandons a queue (memoryless patience, Section 2.3)
+        self.place_ranks, self.admit_ranks, self.abandon_p_ranks, self.abandon_d_ranks = [], [], [], []
+        self.max_load_seen = [0] * self.N              # most decodes ever held, per GPU
 
     # -- helpers -----------------------------------------------------------------------------
     def M(self):
@@ -39,10 +43,18 @@ class Replay:
     def cap(self, g):
         return self.B - 1 if (g < self.M() or self.pf[g] is not None) else self.B
 
-    def tau(self, p, d):
+    def tau(self, p, d, K=0):
+        """Eq. (1)-(3) plus the KV slope of the Section 6.1 solo fit: K = KV tokens resident in the batch."""
         am, beta, dm, a_s, ds, kappa = (float(x) for x in self.inp.coeffs)
-        assert kappa == 0.0
-        return am + beta * p + dm * d if p > 0 else a_s + ds * d
+        return (am + beta * p + dm * d if p > 0 else a_s + ds * d) + kappa * K
+
+    def kv_tokens(self, g, members):
+        """KV tokens held by the decodes of a batch: each one's prompt plus the tokens it has emitted so far."""
+        K = 0
+        for key in members:
+            P, D = self.lengths(*key)
+            K += P + (D - self.dec[g][key][0])
+        return K
 
     def lengths(self, cls, job):
         j = self.jobs[(cls, job)]
@@ -53,7 +65,8 @@ class Replay:
         if self.iter_start[g] is None and (self.pf[g] is not None or self.dec[g]):
             p = min(self.C, self.pf[g][2]) if self.pf[g] is not None else 0
             self.iter_start[g] = t
-            self.batch[g] = (p, len(self.dec[g]), set(self.dec[g].keys()))
+            members = set(self.dec[g].keys())
+            self.batch[g] = (p, len(members), members, self.kv_tokens(g, members))
 
     # -- the walk ----------------------------------------------------------------------------
     def run(self, known_lengths=None):
@@ -93,10 +106,13 @@ class Replay:
                         self.jobs[(cls, job)]["dropped"] = True
                 elif typ == "ABANDON_P":
                     assert job in self.pq[cls]
+                    self.abandon_p_ranks.append((self.pq[cls].index(job), len(self.pq[cls])))
                     self.pq[cls].remove(job)
                     self.jobs[(cls, job)]["t_leave_q"] = t
                 elif typ == "ABANDON_D":
                     assert (cls, job) in self.dq
+                    same = [e for e in self.dq if e[0] == cls]
+                    self.abandon_d_ranks.append((same.index((cls, job)), len(same)))
                     self.dq.remove((cls, job))
                     self.jobs[(cls, job)]["t_leave_dq"] = t
                 elif typ == "ITER_END":
@@ -132,8 +148,8 @@ class Replay:
 
     def _iter_end(self, g, t, tau_logged, group):
         assert self.iter_start[g] is not None, "iteration end on an idle GPU"
-        p, d, members = self.batch[g]
-        assert abs(tau_logged - self.tau(p, d)) < 1e-15, ("iteration time", tau_logged, self.tau(p, d), p, d)
+        p, d, members, K = self.batch[g]
+        assert abs(tau_logged - self.tau(p, d, K)) < 1e-15, ("iteration time", tau_logged, self.tau(p, d, K), p, d, K)
         assert abs((self.iter_start[g] + tau_logged) - t) < 1e-9
         for key in members:                       # every decode frozen into the batch emits one token
             self.dec[g][key][0] -= 1
@@ -164,11 +180,13 @@ class Replay:
         mix_free = [h for h in range(0, M) if loads[h] < self.cap(h)]
         tier = solo_free if solo_free else mix_free
         assert g in tier, "router must fill solo GPUs first (Section 4.1)"
+        self.place_ranks.append((tier.index(g), len(tier)))
         if self.inp.placement == 1:
             best = min(tier, key=lambda h: (loads[h], h))
             assert g == best, "least-loaded placement violated"
         P, D = self.lengths(cls, job)
         self.dec[g][(cls, job)] = [D, t]
+        self.max_load_seen[g] = max(self.max_load_seen[g], len(self.dec[g]))
         self.jobs[(cls, job)]["t_place"] = t
 
     def _check_admit(self, cls, job, g, t):
@@ -190,6 +208,7 @@ class Replay:
             assert cls == min(waiting, key=lambda i: (int(inp.prio_rank[i]), i)), "priority gate violated"
         cands = [h for h in range(M) if self.pf[h] is None and len(self.dec[h]) <= self.B - 1]
         assert g in cands
+        self.admit_ranks.append((cands.index(g), len(cands)))
         if inp.placement == 1:
             assert g == min(cands, key=lambda h: (len(self.dec[h]), h))
         self.pq[cls].pop(0)
