@@ -290,6 +290,19 @@ def single_class(N=1, B=3, C=256, P=512, D=2, lam=1.0, R=1, seed=7, coeffs=COEFF
     return inp
 
 
+def crowded(kind="decode", N=4, R=1, placement=PLACE_RANDOM, seed=None, M=None, router=ROUTER_SOLO_FIRST) -> SimInputs:
+    """Two fixed-length classes with short patience, half of the GPUs mixed.  kind "decode": decode slots are the scarce
+    resource (requests wait in, and abandon, the decode buffer); kind "prefill": prefill slots are scarce (requests
+    abandon the prefill queues).  Per-GPU rates are fixed, so the congestion is the same at every cluster size."""
+    P, D, lam, B, sd = ([300, 700], [60, 30], [9.0, 6.0], 4, 5) if kind == "decode" else ([1500, 2500], [10, 6], [8.0, 5.0], 8, 6)
+    inp = build(f"crowded_{kind}_N{N}", N=N, R=R, B=B, C=256, Pm=P, Dm=D, lam_blocks=[lam], theta=[0.6, 0.9],
+                prices=[1.0, 2.0], coeffs=COEFFS_BENCH, gate=GATE_OCCUPANCY, router=router,
+                placement=placement, pricing=PRICING_BUNDLED, P_fixed=P, D_fixed=D, seed=sd if seed is None else seed,
+                qcap=max(1024, _next_pow2(2.0 * N)))
+    inp.M[:] = N // 2 if M is None else M
+    return inp
+
+
 def trace_replay(n=10, R=2, T=90.0, seed=42, placement=PLACE_RANDOM, coeffs=COEFFS_PAPER_KV):
     """Matched synthetic stand-in for the paper's trace replay (Section 6.2; the Azure traces are not
     redistributable): two classes ("code": long prompts, short outputs; "conversation": the reverse) with

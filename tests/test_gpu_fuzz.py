@@ -63,14 +63,14 @@ def test_random_configuration(seed):
             assert np.array_equal(a[k], b[k]), (inp.name, "GPU state", k)
 
 
-@pytest.mark.parametrize("seed", range(18))
+@pytest.mark.parametrize("seed", range(24))
 def test_random_sizes_on_the_benchmark_feature_sets(seed):
     # the feature sets that have their own kernel instances (cfg1, cfg2, cfg4 recipes) on random cluster sizes and decode caps
     from oracle import OracleSim
     from paper_2602_02987_b200 import QSim
     rng = np.random.default_rng(5000 + seed)
     recipe = [presets.cfg1, presets.cfg2, presets.cfg4][seed % 3]
-    N = int(rng.choice([1, 5, 32, 33, 64, 70, 128, 129, 200, 512, 530]))
+    N = int(rng.choice([1, 5, 32, 33, 64, 70, 128, 129, 200, 512, 530, 1024, 2049]))
     B = int(rng.choice([2, 17, 32, 100, 128, 256]))
     kw = {} if recipe is presets.cfg1 else {"N": N}
     inp = recipe(R=2, **kw)
@@ -78,7 +78,22 @@ def test_random_sizes_on_the_benchmark_feature_sets(seed):
         N = int(rng.choice([1, 5, 33, 64, 100]))
         inp = inp.with_(N=N, M=np.array([max(1, N // 3)], np.uint32), n_xstar=inp.xstar * N, n_qpstar=inp.n_qpstar * N / 64)
     inp = inp.with_(B=B, seed=seed)
-    H = int(60_000 / max(N, 20))
+    H = max(int(60_000 / max(N, 20)), 150)
+    sim = QSim(inp); sim.run(H); got = sim.stats(); gstate = [sim.server_state(r) for r in range(inp.R)]; sim.close()
+    o = OracleSim(inp); o.run(H); ref = o.stats(); ostate = [o.server_state(r) for r in range(inp.R)]; o.close()
+    assert_parity(got, ref, what=f"{inp.name}: N={inp.N} B={inp.B}")
+    for a, b in zip(gstate, ostate):
+        for k in a:
+            assert np.array_equal(a[k], b[k]), (inp.name, "GPU state", k)
+
+
+@pytest.mark.parametrize("recipe,N,B", [("cfg2", 1024, 100), ("cfg4", 2049, 17), ("cfg2", 2049, 33), ("cfg4", 1023, 256)])
+def test_sizes_around_the_warp_count_thresholds(recipe, N, B):
+    # 1024 GPUs = 32 rows (four warps per replication), 2049 = 65 rows (eight warps, last row holds one GPU)
+    from oracle import OracleSim
+    from paper_2602_02987_b200 import QSim
+    inp = getattr(presets, recipe)(N=N, R=2).with_(B=B, seed=N + B)
+    H = 150
     sim = QSim(inp); sim.run(H); got = sim.stats(); gstate = [sim.server_state(r) for r in range(inp.R)]; sim.close()
     o = OracleSim(inp); o.run(H); ref = o.stats(); ostate = [o.server_state(r) for r in range(inp.R)]; o.close()
     assert_parity(got, ref, what=f"{inp.name}: N={inp.N} B={inp.B}")

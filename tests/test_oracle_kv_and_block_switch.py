@@ -145,24 +145,13 @@ def _chi2_uniform(ranks, rng, bins=10):
     return float(((obs - exp) ** 2 / exp).sum()), r.size
 
 
-def crowded_case(kind):
-    """Two classes with short patience on four GPUs: "decode" keeps the decode slots scarce (requests abandon the decode
-    buffer), "prefill" keeps the prefill slots scarce (requests abandon the prefill queues)."""
-    P, D, lam, B, seed = ([300, 700], [60, 30], [9.0, 6.0], 4, 5) if kind == "decode" else ([1500, 2500], [10, 6], [8.0, 5.0], 8, 6)
-    inp = presets.build(f"crowded_{kind}", N=4, R=1, B=B, C=256, Pm=P, Dm=D, lam_blocks=[lam], theta=[0.6, 0.9],
-                        prices=[1.0, 2.0], coeffs=presets.COEFFS_BENCH, gate=GATE_OCCUPANCY, router=ROUTER_SOLO_FIRST,
-                        placement=PLACE_RANDOM, pricing=PRICING_BUNDLED, P_fixed=P, D_fixed=D, seed=seed, qcap=1024)
-    inp.M[:] = 2
-    return inp
-
-
 def check_uniform_choices():
     # Section 4.1 places a request on a GPU chosen uniformly among those of the tier that have room; memoryless
     # patience (Section 2.3) makes every waiting request of a class equally likely to be the one that leaves
     rng = np.random.default_rng(12345)
     place, ab_p, ab_d = [], [], []
     cases = [(presets.paper_instance(n=8, R=1, horizon_iters=12_000, placement=PLACE_RANDOM, seed=100), 12_000),
-             (crowded_case("decode"), 20_000), (crowded_case("prefill"), 20_000)]
+             (presets.crowded("decode"), 20_000), (presets.crowded("prefill"), 20_000)]
     for inp, H in cases:
         tr, _ = _run(inp, H, cap=4_000_000)
         rp = Replay(inp, tr, rep=0).run()
