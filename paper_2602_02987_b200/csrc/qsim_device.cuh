@@ -46,15 +46,13 @@ constexpr int TOUCH_CAP = 48;
 // compiled out.  SPL > 0 fixes the number of simulated GPUs per lane (N <= 32 SPL) so the per-GPU loops unroll.
 constexpr uint32_t F_GENERIC = 1, F_ABANDON = 2, F_SLI = 4, F_KAPPA = 8, F_HIST = 16, F_BLOCKS = 32, F_RANDOM = 64,
                    F_OCC = 128, F_SLOTS = 256, F_MW = 512, F_FCFS = 1024, F_SLIG = 2048, F_IMM = 4096;
-// F_MW: several warps per replication (large clusters).  Warp 0 (the master) runs the round loop and every event
-// handler; all warps share the local iteration ends of a round, row by row (a row = 32 consecutive GPUs).  Per-row
-// summaries in shared memory (earliest end, earliest non-local ends, least-loaded keys, eligible counts) are refreshed
-// by whoever changes a GPU of the row, so that the master's searches touch one entry per row instead of every GPU.
-enum { MW_ENDS = 2, MW_EXIT = 3 };
+// F_MW: several warps per replication.  Warp 0 (the master) runs the round loop and every event handler; the
+// other warps (helpers) wait at a block barrier for commands and take their share of the per-GPU work of a
+// round: rows r = warp, warp + W, ... of the candidate scan and of the local iteration ends / retirements.
+enum { MW_SCAN = 1, MW_ENDS = 2, MW_EXIT = 3 };
+struct MwCmd { unsigned long long lim_t; uint32_t op, lim_s, buffered, M, force, pad; };
+struct MwRes { unsigned long long bt, tmin; uint32_t bs, progressed; };
 constexpr int MW_MAX = 16;
-constexpr int MW_ROWS = 128;          // at most 4096 GPUs per replication
-struct MwCmd { unsigned long long lim_t; uint32_t op, lim_s, buffered, M, force, overcap, prog, pad; uint32_t todo[MW_ROWS / 32]; };
-constexpr uint32_t NOHINT = 0xffffu;
 
 // source ids: smaller id wins an exact tie in time
 constexpr uint32_t SRC_BLOCK = 0, SRC_ARRIVAL = 1, SRC_ABP = 9, SRC_ABD0 = 17, SRC_ABD1 = 25, SRC_SERVER = 33;
@@ -94,8 +92,7 @@ static_assert(sizeof(ClassState) % 8 == 0 && (sizeof(ClassState) * MAXI) % 16 ==
 static_assert(sizeof(RepHeader) % 16 == 0 && offsetof(RepHeader, cs) % 16 == 0, "RepHeader layout");
 
 struct SlotRec { double tpf; uint32_t pk; uint32_t pad; };  // request in a decode slot: prefill end time, packed lengths/class/group
-constexpr int STAGE_CAP = 64;                                 // finished-request records waiting for their accounting (one warp per replication)
-constexpr int STAGE_CAP_MW = 24;                              // the same, per warp, when several warps share a replication
+constexpr int STAGE_CAP = 64;                                 // finished-request records waiting for their accounting
 // Accounting of finished requests, one block per warp (merged into the class records at kernel exit)
 struct WarpClassStats { double sYm_out, sYs_out, sum_tpot; unsigned long long tok_in, tok_out; uint32_t done_mixed, done_solo; };
 struct ADraw { double E; uint32_t pk; uint32_t pad; };     // one arrival draw: unit exponential (divided by the rate already when there is one block) and packed lengths
@@ -119,14 +116,13 @@ struct Params {
     // workspace sections (all arrays are [R][...])
     RepHeader *hdr;
     char *srv;                   // per replication: server structure-of-arrays image, srv_bytes each
-    uint32_t *slot_fin;          // [R][N][Bp]
+    uint32_t *slot_fin;          // [R][N][B]
     SlotRec *slot_rec;           // [R][N][B]
     QEntry *pq;                  // [R][I][qcap]
     QEntry *dq;                  // [R][2][qcap]
     uint32_t *hist_mem;          // [R][I][2][NBIN] or null
     uint32_t *not_done;          // single counter: replications that stopped on the event budget
     uint32_t srv_bytes;
-    uint32_t Bp;                 // row stride (entries) of slot_fin: B rounded up to a multiple of 4
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -318,18 +314,12 @@ struct Sim {
     const uint32_t rep;
     int warp, nwarps;            // position in the block (F_MW); 0 / 1 otherwise
     MwCmd *cmd;
+    MwRes *res;
     WarpClassStats *wcs;         // [nwarps][MAXI]
-    // per-row summaries (F_MW): earliest end of the row with its GPU, earliest end that finishes a prefill, earliest end
-    // that finishes a decode only, least-loaded key (decodes << 16 | GPU) per kind of request, and packed counts of
-    // eligible GPUs (solo decode | mixed decode << 8 | prefill << 16 | mixed GPUs above the mixed cap << 24)
-    unsigned long long *rc_tmin, *rc_tpf, *rc_tdec;
-    uint32_t *rc_gmin, *rc_gpf, *rc_gdec, *rc_ksolo, *rc_kmix, *rc_kpf, *rc_cnt;
-    bool overcap;                // F_MW: some mixed GPU holds more than B-1 decodes (possible after M grew)
     // shared memory (lane-owned entries)
-    double *tnext, *pf_tarr;
+    double *tnext, *pf_tarr, *taucur;      // taucur: duration of the running iteration
     uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
     uint16_t *ndec, *nact, *pfcur;
-    uint16_t *hw, *hint;         // slot records in global memory: slots at or above hw[g] were never used; hint[g] = a free slot or NOHINT
     uint16_t *sfin16;            // [Npad][B]  low 16 bits of each slot's finish iteration (f_slots)
     uint32_t *socc;              // [Npad][ceil(B/32)]  slot occupancy bits; bits past B are set for good
     uint32_t *touch;
@@ -343,7 +333,7 @@ struct Sim {
     SlotRec *st_rec;
     double *st_te;
     QEntry *pqh;
-    uint32_t n_pend, stage_cap;
+    uint32_t n_pend;
     uint32_t rec_after;          // per lane: record copies committed since this lane's last queue-head copy
     QEntry *pq, *dq;
     uint32_t *hist;
@@ -480,7 +470,6 @@ struct Sim {
 
     __device__ uint32_t count_idle_pf()
     {
-        if (F & F_MW) return count_idle_pf_rows();
         // per-lane count over the lane's rows (branch-free), one warp-wide sum
         uint32_t cnt = 0;
 #pragma unroll 4
@@ -571,134 +560,6 @@ struct Sim {
         }
     }
 
-    // --- per-row summaries (F_MW) -------------------------------------------------------------------
-    // warp minimum of a 64-bit key together with the lowest id among the lanes that hold it
-    __device__ __forceinline__ void min_key_id(unsigned long long v, uint32_t id, unsigned long long &vmin, uint32_t &idmin) const
-    {
-        const uint32_t hi = (uint32_t)(v >> 32), lo = (uint32_t)v;
-        const uint32_t mhi = __reduce_min_sync(FULL, hi);
-        const uint32_t mlo = __reduce_min_sync(FULL, hi == mhi ? lo : NONE32);
-        idmin = __reduce_min_sync(FULL, (hi == mhi && lo == mlo) ? id : NONE32);
-        vmin = ((unsigned long long)mhi << 32) | mlo;
-    }
-
-    // Times of row k (whole warp): earliest end, earliest end that finishes a prefill, earliest end that finishes decodes only.
-    __device__ void refresh_time(uint32_t k)
-    {
-        const unsigned long long INF = 0x7ff0000000000000ull;
-        const uint32_t g = (k << 5) + (uint32_t)lane;
-        const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-        const uint32_t na = nact[g];
-        const bool run = v < INF;
-        unsigned long long a, b, c;
-        uint32_t ga, gb, gc;
-        min_key_id(v, g, a, ga);
-        min_key_id((run && (na & 0x8000u)) ? v : INF, g, b, gb);
-        min_key_id((run && (na & 0xc000u) == 0x4000u) ? v : INF, g, c, gc);
-        if (lane == 0) {
-            rc_tmin[k] = a; rc_gmin[k] = ga; rc_tpf[k] = b; rc_gpf[k] = gb; rc_tdec[k] = c; rc_gdec[k] = gc;
-        }
-    }
-
-    // Loads of row k (whole warp): least-loaded key and count of the GPUs eligible for a solo decode, a mixed decode, a prefill.
-    __device__ void refresh_load(uint32_t k)
-    {
-        const uint32_t g = (k << 5) + (uint32_t)lane;
-        const uint32_t nd = ndec[g];
-        const bool pf = (pfjob[g] >> 31) != 0, mix = g < M, in = g < p.N;
-        const uint32_t cap = (mix || pf) ? p.B - 1 : p.B;
-        const bool es = in && !mix && nd < cap, em = in && mix && nd < cap, ep = in && mix && !pf && nd <= p.B - 1;
-        const uint32_t key = (nd << 16) | g;
-        const uint32_t ks = __reduce_min_sync(FULL, es ? key : NONE32);
-        const uint32_t km = __reduce_min_sync(FULL, em ? key : NONE32);
-        const uint32_t kp = __reduce_min_sync(FULL, ep ? key : NONE32);
-        const uint32_t cs_ = (uint32_t)__popc(__ballot_sync(FULL, es)), cm = (uint32_t)__popc(__ballot_sync(FULL, em)),
-                       cp = (uint32_t)__popc(__ballot_sync(FULL, ep));
-        const uint32_t over = __ballot_sync(FULL, in && mix && nd > p.B - 1) ? 1u : 0u;
-        if (lane == 0) { rc_ksolo[k] = ks; rc_kmix[k] = km; rc_kpf[k] = kp; rc_cnt[k] = cs_ | (cm << 8) | (cp << 16) | (over << 24); }
-    }
-
-    __device__ void refresh_all_rows()
-    {
-        __syncwarp();
-        for (uint32_t k = 0; k < n_rows(); ++k) { refresh_time(k); refresh_load(k); }
-        __syncwarp();
-    }
-
-    __device__ __forceinline__ uint32_t row_key(uint32_t r, int want) const
-    {
-        return want == WANT_SOLO ? rc_ksolo[r] : (want == WANT_MIX ? rc_kmix[r] : rc_kpf[r]);
-    }
-
-    // F_MW: the searches over all GPUs read one summary per row
-    __device__ uint32_t choose_server_rows(int want)
-    {
-        const uint32_t rows = n_rows();
-        __syncwarp();
-        if (!f_random()) {
-            uint32_t best = NONE32;
-            for (uint32_t r = (uint32_t)lane; r < rows; r += 32) best = min(best, row_key(r, want));
-            best = __reduce_min_sync(FULL, best);
-            return best == NONE32 ? NONE32 : (best & 0xffffu);
-        }
-        const uint32_t sh = want == WANT_SOLO ? 0u : (want == WANT_MIX ? 8u : 16u);
-        uint32_t mine = 0;
-        for (uint32_t r = (uint32_t)lane; r < rows; r += 32) mine += (rc_cnt[r] >> sh) & 0xffu;
-        const uint32_t cnt = __reduce_add_sync(FULL, mine);
-        if (cnt == 0) return NONE32;
-        uint32_t idx = 0;
-        if (cnt > 1) {
-            uint32_t w0, w1, w2, w3;
-            draw(p, rep, STREAM_PLACEMENT << 8, place_ord++, w0, w1, w2, w3);
-            idx = __umulhi(w0, cnt);
-        }
-        // the idx-th eligible GPU in index order: rows j*32 .. j*32+31 at a time
-        for (uint32_t j = 0; j < rows; j += 32) {
-            const uint32_t r = j + (uint32_t)lane;
-            const uint32_t c = r < rows ? (rc_cnt[r] >> sh) & 0xffu : 0u;
-            uint32_t incl = c;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t up = __shfl_up_sync(FULL, incl, d);
-                if (lane >= d) incl += up;
-            }
-            const uint32_t tot = __shfl_sync(FULL, incl, 31);
-            if (idx >= tot) { idx -= tot; continue; }
-            const uint32_t excl = incl - c;
-            const uint32_t holder = __ballot_sync(FULL, idx >= excl && idx < incl);
-            const int hl = __ffs((int)holder) - 1;
-            const uint32_t row = j + (uint32_t)hl;
-            const uint32_t within = idx - __shfl_sync(FULL, excl, hl);
-            const uint32_t b = __ballot_sync(FULL, eligible((row << 5) + (uint32_t)lane, want));
-            return (row << 5) + (uint32_t)__fns(b, 0, (int)within + 1);
-        }
-        err = ERR_INTERNAL;
-        return NONE32;
-    }
-
-    __device__ uint32_t choose_solo_first_rows()
-    {
-        __syncwarp();
-        uint32_t best = NONE32;
-        for (uint32_t r = (uint32_t)lane; r < n_rows(); r += 32) {
-            const uint32_t a = rc_ksolo[r], b = rc_kmix[r];
-            best = min(best, a);
-            best = min(best, b == NONE32 ? NONE32 : (b | 0x40000000u));
-        }
-        best = __reduce_min_sync(FULL, best);
-        return best == NONE32 ? NONE32 : (best & 0xffffu);
-    }
-
-    // idle prefill slots, and whether some mixed GPU is above the mixed cap
-    __device__ uint32_t count_idle_pf_rows()
-    {
-        __syncwarp();
-        uint32_t mine = 0, over = 0;
-        for (uint32_t r = (uint32_t)lane; r < n_rows(); r += 32) { const uint32_t c = rc_cnt[r]; mine += (c >> 16) & 0xffu; over |= c >> 24; }
-        overcap = __any_sync(FULL, over != 0);
-        return __reduce_add_sync(FULL, mine);
-    }
-
     // --- GPU choice ----------------------------------------------------------------------------
     __device__ __forceinline__ bool eligible(uint32_t g, int want) const
     {
@@ -716,7 +577,6 @@ struct Sim {
     // Solo-first target of a decode under least-loaded placement in one reduction: key = tier, load, index.
     __device__ __forceinline__ uint32_t choose_solo_first()
     {
-        if (F & F_MW) return choose_solo_first_rows();
         uint32_t best = NONE32;
 #pragma unroll 4
         for (uint32_t k = 0; k < n_rows(); ++k) {
@@ -733,7 +593,6 @@ struct Sim {
 
     __device__ uint32_t choose_server(int want)
     {
-        if (F & F_MW) return choose_server_rows(want);
         const uint32_t rows = n_rows();
         if (!f_random()) {
             uint32_t best = NONE32;
@@ -817,50 +676,6 @@ struct Sim {
         return 0;
     }
 
-    // Slot records in global memory (large N*B): every GPU has B fixed slots; the finish stamp of a free slot is NONE32.
-    // All lanes: a free slot of GPU g for a new request.  The owner lane first tries the slot it remembers as free
-    // (freed by the last retirement, or found by the last search), then a slot that was never used; only when both fail
-    // does the warp read the GPU's stamps and look for free slots.  Record copies of finished requests that are still in
-    // flight are awaited first: the new request's record may go where one of them reads.
-    __device__ uint32_t take_slot(uint32_t g)
-    {
-        const int owner = (int)(g & 31u);
-        cp_async_wait_all();
-        __syncwarp();
-        uint32_t slot = NONE32;
-        if (lane == owner) {
-            const uint32_t h = hint[g], w = hw[g];
-            if (h != NOHINT) { slot = h; hint[g] = (uint16_t)NOHINT; }
-            else if (w < p.B) { slot = w; hw[g] = (uint16_t)(w + 1u); }
-        }
-        slot = __shfl_sync(FULL, slot, owner);
-        if (slot != NONE32) return slot;
-        const uint32_t *row = s_fin + (size_t)g * p.Bp;
-        uint32_t first = NONE32, second = NONE32;
-        for (uint32_t c = 0; c < p.B && second == NONE32; c += 128) {
-            const uint32_t j0 = c + ((uint32_t)lane << 2);
-            uint32_t fe[4] = { 0u, 0u, 0u, 0u };
-            if (j0 < p.B) {
-                const uint4 f = *reinterpret_cast<const uint4 *>(row + j0);
-                fe[0] = f.x; fe[1] = f.y; fe[2] = f.z; fe[3] = f.w;
-            }
-            uint32_t a = NONE32, b = NONE32;          // the two lowest free slots of this lane's four
-#pragma unroll
-            for (uint32_t e = 0; e < 4; ++e)
-                if (j0 + e < p.B && fe[e] == NONE32) { if (a == NONE32) a = j0 + e; else if (b == NONE32) b = j0 + e; }
-            const uint32_t m1 = __reduce_min_sync(FULL, a);
-            if (first == NONE32) {
-                first = m1;
-                second = __reduce_min_sync(FULL, a == m1 ? b : a);
-            } else {
-                second = m1;
-            }
-        }
-        if (first == NONE32) { err = ERR_INTERNAL; return 0; }
-        if (lane == owner) hint[g] = (uint16_t)(second == NONE32 ? NOHINT : second);
-        return first;
-    }
-
     // entry pos (0 = head) of the pool's buffer goes to GPU g
     __device__ void place_decode(uint32_t pool, uint32_t g, uint32_t pos = 0)
     {
@@ -885,9 +700,6 @@ struct Sim {
     __device__ void place_job(uint32_t pool, uint32_t g, uint32_t i, uint32_t P, uint32_t D, double tpf, bool from_buffer)
     {
         const bool mixed = g < M;
-        uint32_t gslot = 0;
-        if (!f_slots()) gslot = take_slot(g);
-        else if (n_pend) { cp_async_wait_all(); __syncwarp(); }   // a record copy in flight may read the slot this request takes
         if (lane == (int)i) {
             ClassState &c = cs[i];
             const uint32_t Qd = pool ? c.Qd1 : c.Qd0;
@@ -920,8 +732,8 @@ struct Sim {
                 sfin16[g * p.B + slot] = (uint16_t)fin;
                 o = (size_t)g * p.B + slot;
             } else {
-                o = (size_t)g * p.B + gslot;
-                s_fin[(size_t)g * p.Bp + gslot] = fin;
+                o = (size_t)g * p.B + sl;
+                s_fin[o] = fin;
             }
             SlotRec r; r.tpf = tpf; r.pk = pack_job(P, D, i, mixed ? 1u : 0u); r.pad = 0;
             s_rec[o] = r;
@@ -930,7 +742,6 @@ struct Sim {
             if (f_kappa()) Kpend[g] += P;
         }
         touch_server(g);
-        if (F & F_MW) { __syncwarp(); refresh_load(g >> 5); }
     }
 
     // --- prefill gate ------------------------------------------------------------------------------
@@ -1007,7 +818,6 @@ struct Sim {
             pf_tarr[g] = e.t;
         }
         touch_server(g);
-        if (F & F_MW) { __syncwarp(); refresh_load(g >> 5); }
     }
 
     // Called by the owner: a GPU with work that is between iterations starts one at time ts.  The batch
@@ -1030,6 +840,7 @@ struct Sim {
             if (f_kappa()) { K[g] = Kg; Kpend[g] = 0; }
             pfcur[g] = (uint16_t)pc;
             nact[g] = (uint16_t)(nd | fl);
+            taucur[g] = tau;
             tnext[g] = __dadd_rn(ts, tau);
         }
     }
@@ -1100,20 +911,6 @@ struct Sim {
             for (uint32_t k = 0; k < n_touch; ++k) {
                 const uint32_t g = touch[k];
                 if (lane == (int)(g & 31u)) start_if_needed(g);
-            }
-        }
-        if (F & F_MW) {
-            // the rows of the GPUs that may have started an iteration get their times summarised again
-            __syncwarp();
-            if (touch_all) {
-                for (uint32_t k = 0; k < n_rows(); ++k) refresh_time(k);
-            } else {
-                uint32_t last = NONE32;
-                for (uint32_t k = 0; k < n_touch; ++k) {
-                    const uint32_t row = touch[k] >> 5;
-                    if (row != last) refresh_time(row);
-                    last = row;
-                }
             }
         }
         n_touch = 0;
@@ -1204,77 +1001,38 @@ struct Sim {
         __syncwarp();
     }
 
-    // One group of four stamps (slots j0 .. j0+3 of GPU g, valid below hwm) of the retirement scan.
-    __device__ __forceinline__ void retire_four(uint32_t g, const uint4 f, uint32_t j0, uint32_t hwm, uint32_t itg, double te,
-                                                uint32_t &newmin, uint32_t &done, uint32_t &Kdrop, uint32_t &freed)
-    {
-        const uint32_t fe[4] = { f.x, f.y, f.z, f.w };
-        bool hit[4];
-#pragma unroll
-        for (uint32_t e = 0; e < 4; ++e) {
-            const bool valid = j0 + e < hwm;
-            hit[e] = valid && fe[e] == itg;
-            if (valid && !hit[e]) newmin = min(newmin, fe[e]);      // a free slot holds NONE32, the identity of the minimum
-        }
-        if (!__ballot_sync(FULL, hit[0] || hit[1] || hit[2] || hit[3])) return;
-        uint32_t *row = s_fin + (size_t)g * p.Bp;
-#pragma unroll
-        for (uint32_t e = 0; e < 4; ++e) {
-            uint32_t hits = __ballot_sync(FULL, hit[e]);
-            if (!hits) continue;
-            const uint32_t j = j0 + e, nh = (uint32_t)__popc(hits);
-            done += nh;
-            if (hit[e]) { row[j] = NONE32; freed = min(freed, j); }
-            if (!f_kappa()) {
-                // the records only feed statistics: copy them on chip asynchronously, account later
-                if (n_pend + nh > stage_cap) flush_done();
-                if (hit[e]) {
-                    const uint32_t pos = n_pend + (uint32_t)__popc(hits & ((1u << lane) - 1u));
-                    cp_async16(&st_rec[pos], &s_rec[(size_t)g * p.B + j]);
-                    cp_async_commit();
-                    rec_after++;
-                    st_te[pos] = te;
-                }
-                n_pend += nh;
-            } else {
-                SlotRec r; r.tpf = 0.0; r.pk = 0;
-                if (hit[e]) r = s_rec[(size_t)g * p.B + j];
-                while (hits) {
-                    const int hl = __ffs((int)hits) - 1;
-                    hits &= hits - 1;
-                    const uint32_t pkh = __shfl_sync(FULL, r.pk, hl);
-                    const double tpfh = __shfl_sync(FULL, r.tpf, hl);
-                    account_done(pkh, tpfh, te);
-                    Kdrop += job_P(pkh) + job_D(pkh);
-                }
-            }
-        }
-    }
-
-    // Some decode on GPU g emitted its last token in the iteration that ended at te (its itg-th).  Slot records in global
-    // memory: every lane reads four stamps per load (256 slots = two loads in flight), the slots that hit are marked
-    // free and their records are fetched asynchronously for the accounting; nothing is moved.
     __device__ void retire_decodes(uint32_t g, uint32_t itg, uint32_t nd, double te)
     {
         if (f_slots()) { retire_slots(g, itg, nd, te); return; }
         const int owner = (int)(g & 31u);
-        const uint32_t hwm = hw[g];
-        const uint32_t *row = s_fin + (size_t)g * p.Bp;
-        uint32_t newmin = NONE32, done = 0, Kdrop = 0, freed = NONE32;
-        for (uint32_t c = 0; c < hwm; c += 256) {
-            const uint32_t j0 = c + ((uint32_t)lane << 2), j1 = j0 + 128u;
-            uint4 f0 = make_uint4(0u, 0u, 0u, 0u), f1 = f0;
-            if (j0 < hwm) f0 = *reinterpret_cast<const uint4 *>(row + j0);
-            if (j1 < hwm) f1 = *reinterpret_cast<const uint4 *>(row + j1);
-            retire_four(g, f0, j0, hwm, itg, te, newmin, done, Kdrop, freed);
-            retire_four(g, f1, j1, hwm, itg, te, newmin, done, Kdrop, freed);
+        uint32_t n = nd, newmin = NONE32, Kdrop = 0;
+        const size_t base = (size_t)g * p.B;
+        for (int k = (int)((nd - 1) >> 5); k >= 0; --k) {
+            const uint32_t j = ((uint32_t)k << 5) + (uint32_t)lane;
+            const uint32_t f = j < nd ? s_fin[base + j] : NONE32;
+            const bool hit = f == itg;
+            if (!hit) newmin = min(newmin, f);
+            uint32_t hits = __ballot_sync(FULL, hit);
+            while (hits) {
+                const int hl = 31 - __clz(hits);
+                hits &= ~(1u << hl);
+                const uint32_t h = ((uint32_t)k << 5) + (uint32_t)hl;
+                const SlotRec rh = s_rec[base + h];
+                account_done(rh.pk, rh.tpf, te);
+                Kdrop += job_P(rh.pk) + job_D(rh.pk);
+                const uint32_t last = n - 1;
+                __syncwarp();
+                if (lane == 0 && h != last) {
+                    s_fin[base + h] = s_fin[base + last];
+                    s_rec[base + h] = s_rec[base + last];
+                }
+                n = last;
+            }
         }
         newmin = __reduce_min_sync(FULL, newmin);
-        freed = __reduce_min_sync(FULL, freed);
         if (lane == owner) {
-            ndec[g] = (uint16_t)(nd - done);
+            ndec[g] = (uint16_t)n;
             nfin[g] = newmin;
-            if (freed != NONE32) hint[g] = (uint16_t)freed;
             if (f_kappa()) K[g] -= Kdrop;
         }
         __syncwarp();
@@ -1296,7 +1054,7 @@ struct Sim {
                 itg = it[g] + 1;
                 it[g] = itg;
                 const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
-                const double tau = iter_time(p, pc, na, Kg, f_kappa());     // duration of the iteration that ends (same chain as at its start)
+                const double tau = taucur[g];
                 if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
                 else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
                 if (f_kappa()) K[g] = Kg + na;
@@ -1321,7 +1079,6 @@ struct Sim {
             drain_dirty = true;
             gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
             recount_idle = true;
-            if (F & F_MW) { __syncwarp(); refresh_load(g >> 5); }
         }
         if (flags & 2u) {
             // prefill finished: account, then hand the request to the decode stage
@@ -1351,7 +1108,6 @@ struct Sim {
             __syncwarp();   // every lane has read the finished job before its owner clears it
             if (lane == owner) pfjob[g] = 0;
             __syncwarp();
-            if (F & F_MW) refresh_load(g >> 5);
             // No router (immediate same-slot decoding, an ablation of the paper's EC): the request goes on decoding on
             // g, in the slot it holds; it passes through the empty buffer at this instant.
             const bool immediate = (F & F_GENERIC) && p.router == 3;
@@ -1418,9 +1174,9 @@ struct Sim {
     {
         // straight-line: all fields are read first and the stores are predicated on `act` (see start_at)
         const uint32_t it0 = it[g], na_raw = nact[g], pc = pfcur[g], nd = ndec[g], pj = pfjob[g], pr = pfrem[g], nf = nfin[g];
+        const double tau = taucur[g];
         uint32_t K0 = 0, Kp = 0;
         if (f_kappa()) { K0 = K[g]; Kp = Kpend[g]; }
-        const double tau = iter_time(p, pc, na_raw & 0x3fffu, K0, f_kappa());   // duration of the iteration that ends (same chain as at its start)
         const uint32_t itg = it0 + 1u;
         const uint32_t rem = pr - pc;                       // prompt tokens left after this iteration's chunk
         const bool retire = (na_raw & 0x4000u) != 0;        // a decode finished: the GPU waits for retire_decodes
@@ -1439,7 +1195,7 @@ struct Sim {
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
             if (f_kappa()) { K[g] = restart ? Kg : Kend; if (restart) Kpend[g] = 0; }
             pfcur[g] = restart ? (uint16_t)pc2 : (uint16_t)0;
-            if (restart) nact[g] = (uint16_t)(nd | fl);
+            if (restart) { nact[g] = (uint16_t)(nd | fl); taucur[g] = tau2; }
             tnext[g] = restart ? __dadd_rn(te, tau2) : dinf();
         }
         return act && retire;
@@ -1462,61 +1218,45 @@ struct Sim {
         }
     }
 
-    // The local iteration ends of row k below the limit key, with their retirements (whole warp).  Returns true when
-    // some GPU of the row ended an iteration.
-    __device__ bool ends_row(uint32_t k, unsigned long long lim_t, uint32_t lim_s, bool buffered)
+    // This warp's share (rows warp, warp + nwarps, ...) of the candidate scan; run-time row count.
+    __device__ void scan_share(bool buffered, unsigned long long &bt, uint32_t &bs, unsigned long long &tmin)
     {
         const unsigned long long INF = 0x7ff0000000000000ull;
-        const uint32_t g = (k << 5) + (uint32_t)lane;
-        const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-        bool retire = false, did = false;
-        if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
-            retire = local_end(g, __longlong_as_double((long long)v));
-            did = true;
+#pragma unroll 4
+        for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
+            // straight-line (INF is the identity of the minimum; padded GPUs never run)
+            const uint32_t g = (k << 5) + (uint32_t)lane;
+            const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+            const uint32_t na = nact[g], nd = ndec[g];
+            const bool nl = force_nonlocal || (na & 0x8000u) != 0 ||
+                            ((na & 0x4000u) != 0 && (buffered || (g < M && nd > p.B - 1)));
+            tmin = min(tmin, v);
+            if (v < INF && nl && v < bt) { bt = v; bs = SRC_SERVER + g; }
         }
-        uint32_t need = __ballot_sync(FULL, retire);
-        __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
-        while (need) {
-            const int l = __ffs((int)need) - 1;
-            need &= need - 1;
-            const uint32_t gg = (k << 5) + (uint32_t)l;
-            const double te = __longlong_as_double((long long)__shfl_sync(FULL, v, l));
-            retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
-            if (lane == l) start_at(gg, te);
-        }
-        return did;
     }
 
-    // One warp per replication, run-time row count: every row in turn.
-    __device__ bool ends_all(unsigned long long lim_t, uint32_t lim_s, bool buffered)
+    // This warp's share of the local iteration ends below the limit key, with their retirements.
+    __device__ bool ends_share(unsigned long long lim_t, uint32_t lim_s, bool buffered)
     {
+        const unsigned long long INF = 0x7ff0000000000000ull;
         bool progressed = false;
-        for (uint32_t k = 0; k < n_rows(); ++k)
-            if (ends_row(k, lim_t, lim_s, buffered)) progressed = true;
-        return progressed;
-    }
-
-    // F_MW: this warp's share of the rows that the master listed in the command (rows with an end at or below the
-    // limit): the j-th listed row goes to warp (j + 1) mod W, so the master takes one only when every helper has one.
-    // A row that ended an iteration gets its summaries refreshed by the warp that handled it.
-    __device__ bool ends_rows(unsigned long long lim_t, uint32_t lim_s, bool buffered)
-    {
-        bool progressed = false;
-        uint32_t j = 0;
-        for (uint32_t w = 0; w < (n_rows() + 31u) >> 5; ++w) {
-            uint32_t word = cmd->todo[w];
-            while (word) {
-                const uint32_t k = (w << 5) + (uint32_t)__ffs((int)word) - 1u;
-                word &= word - 1;
-                ++j;
-                if ((int)(j % (uint32_t)nwarps) != warp) continue;
-                const bool did = ends_row(k, lim_t, lim_s, buffered);
-                if (__any_sync(FULL, did)) {
-                    __syncwarp();
-                    refresh_time(k);
-                    refresh_load(k);
-                    progressed = true;
-                }
+        for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
+            const uint32_t g = (k << 5) + (uint32_t)lane;
+            const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+            bool retire = false;
+            if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+                retire = local_end(g, __longlong_as_double((long long)v));
+                progressed = true;
+            }
+            uint32_t need = __ballot_sync(FULL, retire);
+            __syncwarp();   // the owners' updates of it / n_dec are visible to the whole warp
+            while (need) {
+                const int l = __ffs((int)need) - 1;
+                need &= need - 1;
+                const uint32_t gg = (k << 5) + (uint32_t)l;
+                const double te = __longlong_as_double((long long)__shfl_sync(FULL, v, l));
+                retire_decodes(gg, it[gg], (uint32_t)ndec[gg], te);
+                if (lane == l) start_at(gg, te);
             }
         }
         return progressed;
@@ -1537,117 +1277,36 @@ struct Sim {
         tmin_all = ((unsigned long long)tmh << 32) | tml;
     }
 
-    // Helper warps (F_MW): every round the master publishes a command, all warps meet at a block barrier, handle their
-    // share of the local iteration ends and meet again; the master alone then handles the round's non-local event.
+    // Helper warps (F_MW): serve the master's commands until it says stop.  Every command is bracketed by two
+    // block barriers; the master executes the same two.
     __device__ void helper_loop()
     {
+        const unsigned long long INF = 0x7ff0000000000000ull;
         for (;;) {
             __syncthreads();
-            if (cmd->op == MW_EXIT) break;
+            const uint32_t op = cmd->op;
+            if (op == MW_EXIT) return;
+            const bool buffered = cmd->buffered != 0;
             M = cmd->M;
             force_nonlocal = cmd->force != 0;
-            overcap = cmd->overcap != 0;
-            const bool pr = ends_rows(cmd->lim_t, cmd->lim_s, cmd->buffered != 0);
-            cp_async_wait_all();     // a slot freed here may be taken by the master's next placement: its record has been read
-            if (__any_sync(FULL, pr) && lane == 0) cmd->prog = 1u;
+            if (op == MW_SCAN) {
+                unsigned long long bt = INF, tmin = INF, tint, tall;
+                uint32_t bs = NONE32, src;
+                scan_share(buffered, bt, bs, tmin);
+                warp_keys(bt, bs, tmin, tint, src, tall);
+                if (lane == 0) { MwRes r; r.bt = tint; r.bs = src; r.tmin = tall; r.progressed = 0; res[warp] = r; }
+            } else {
+                const bool pr = ends_share(cmd->lim_t, cmd->lim_s, buffered);
+                const uint32_t any = __ballot_sync(FULL, pr);
+                if (lane == 0) res[warp].progressed = any != 0;
+            }
             __syncthreads();
         }
-        flush_done();
     }
 
     // --- round loop ----------------------------------------------------------------------------------
-    // Earliest non-local event among the sources this lane owns besides its GPUs (sources scanned in id order with '<'
-    // keep the tie order); an arrival is local while no prefill slot is idle: it only joins its class queue.
-    __device__ __forceinline__ void class_candidates(unsigned long long &bt, uint32_t &bs, unsigned long long &tmin) const
-    {
-        if (f_blocks() && lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
-        if (lane < (int)p.I) {
-            const ClassState &c = cs[lane];
-            unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
-            tmin = v;
-            if ((n_idle_pf > 0 || force_nonlocal) && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
-            if (f_abandon()) {
-                v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABP + lane; }
-                v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABD0 + lane; }
-                v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
-                if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
-            }
-        }
-    }
-
-    // Local arrivals of this lane's class, in time order, up to the limit key and up to the class's own next abandonment
-    // (which each arrival moves).
-    __device__ __forceinline__ bool local_arrivals(unsigned long long lim_t, uint32_t lim_s)
-    {
-        bool progressed = false;
-        if (lane < (int)p.I && n_idle_pf == 0 && !force_nonlocal) {
-            ClassState &c = cs[lane];
-            for (int guard = 0; guard < 64; ++guard) {
-                const unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
-                if (!(v < lim_t || (v == lim_t && SRC_ARRIVAL + (uint32_t)lane < lim_s))) break;
-                if (f_abandon() && v > (unsigned long long)__double_as_longlong(c.abp.t_ab)) break;
-                arrival_local();
-                progressed = true;
-            }
-        }
-        return progressed;
-    }
-
-    // A class that ran out of draws has an unknown next arrival, possibly before T_int, and a local arrival may have
-    // pulled its class's next abandonment before T_int: then T_int is not the next non-local event after all.
-    __device__ __forceinline__ bool must_redo(unsigned long long tint, uint32_t src) const
-    {
-        bool redo = sched_pending;
-        if (f_abandon() && lane < (int)p.I) {
-            const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
-            redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
-        }
-        return __any_sync(FULL, redo);
-    }
-
-    // The round's non-local event on the warp-wide path, followed by the dispatch.
-    __device__ __forceinline__ void handle_event(unsigned long long tint, uint32_t src)
-    {
-        t = __longlong_as_double((long long)tint);
-        if (src >= SRC_SERVER) {
-            on_server(src - SRC_SERVER);
-        } else {
-            if (f_abandon() && src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
-            else if (f_abandon() && src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
-            else if (f_abandon() && src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
-            else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
-            else {
-                ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true;
-                if (F & F_MW) refresh_all_rows();      // eligibility depends on M
-                n_idle_pf = count_idle_pf(); idle_hint = NONE32;
-            }
-        }
-        if (err) return;
-        dispatch();
-        force_nonlocal = false;
-    }
-
-    // Limit key of the local ends of a round: min{(T_int, src), (T_min + tau_min, 0), (T_end, max)}; wt = T_min + tau_min
-    // (no iteration that starts in this round can end before it).
-    __device__ __forceinline__ void round_limit(unsigned long long tint, uint32_t src, unsigned long long tmin_all, unsigned long long tend_bits,
-                                                unsigned long long &wt, unsigned long long &lim_t, uint32_t &lim_s) const
-    {
-        const unsigned long long INF = 0x7ff0000000000000ull;
-        wt = INF;
-        if (tmin_all < INF)
-            wt = (unsigned long long)__double_as_longlong(__dadd_rn(__longlong_as_double((long long)tmin_all), tau_min));
-        lim_t = tint;
-        lim_s = src;
-        if (wt <= lim_t) { lim_t = wt; lim_s = 0; }
-        if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
-    }
-
-    // One warp per replication.
     __device__ bool run()
     {
-        if (F & F_MW) return run_mw();
         const uint32_t rows = n_rows();
         const unsigned long long INF = 0x7ff0000000000000ull;
         const unsigned long long tend_bits = (unsigned long long)__double_as_longlong(T_end);
@@ -1657,48 +1316,112 @@ struct Sim {
             // classes that ran out of arrival draws get 32 new ones
             for (uint32_t need = __ballot_sync(FULL, sched_pending); need; need &= need - 1)
                 refill((uint32_t)__ffs((int)need) - 1u);
+            // next non-local event of this lane (sources scanned in id order with '<' keep the tie order);
+            // an arrival is local while no prefill slot is idle: it only joins its class queue
             unsigned long long bt = INF, tmin = INF;
             uint32_t bs = NONE32;
-            class_candidates(bt, bs, tmin);
+            if (f_blocks() && lane == 0 && T_blk_next < dinf()) { bt = (unsigned long long)__double_as_longlong(T_blk_next); bs = SRC_BLOCK; }
+            if (lane < (int)p.I) {
+                const ClassState &c = cs[lane];
+                unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
+                tmin = v;
+                if ((n_idle_pf > 0 || force_nonlocal) && v < bt) { bt = v; bs = SRC_ARRIVAL + lane; }
+                if (f_abandon()) {
+                    v = (unsigned long long)__double_as_longlong(c.abp.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABP + lane; }
+                    v = (unsigned long long)__double_as_longlong(c.abd0.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABD0 + lane; }
+                    v = (unsigned long long)__double_as_longlong(c.abd1.t_ab);
+                    if (v < bt) { bt = v; bs = SRC_ABD1 + lane; }
+                }
+            }
             const bool buffered = (dq_n0 | dq_n1) != 0;
             constexpr int NC = SPL > 0 ? SPL : 1;       // per-row values kept in registers when the rows unroll
             unsigned long long vrow[NC];
             bool lrow[NC];
             unsigned long long tint, tmin_all;
             uint32_t src;
+            if (F & F_MW) {
+                // every warp scans its rows; the partial results meet in shared memory
+                if (lane == 0) { cmd->op = MW_SCAN; cmd->buffered = buffered; cmd->M = M; cmd->force = force_nonlocal; }
+                __syncthreads();
+                scan_share(buffered, bt, bs, tmin);
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
+                if (lane == 0) { MwRes r; r.bt = tint; r.bs = src; r.tmin = tmin_all; r.progressed = 0; res[0] = r; }
+                __syncthreads();
+                bt = INF; bs = NONE32; tmin = INF;
+                if (lane < nwarps) { bt = res[lane].bt; bs = res[lane].bs; tmin = res[lane].tmin; }
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
+            } else {
 #pragma unroll
-            for (uint32_t k = 0; k < rows; ++k) {
-                // straight-line (INF is the identity of the minimum; padded GPUs never run)
-                const uint32_t g = (k << 5) + (uint32_t)lane;
-                const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
-                const uint32_t na = nact[g], nd = ndec[g];
-                const bool nl = force_nonlocal || (na & 0x8000u) != 0 ||
-                                ((na & 0x4000u) != 0 && (buffered || (g < M && nd > p.B - 1)));
-                const bool loc = v < INF && !nl;
-                if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
-                tmin = min(tmin, v);
-                if (v < INF && nl && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                for (uint32_t k = 0; k < rows; ++k) {
+                    // straight-line (INF is the identity of the minimum; padded GPUs never run)
+                    const uint32_t g = (k << 5) + (uint32_t)lane;
+                    const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
+                    const uint32_t na = nact[g], nd = ndec[g];
+                    const bool nl = force_nonlocal || (na & 0x8000u) != 0 ||
+                                    ((na & 0x4000u) != 0 && (buffered || (g < M && nd > p.B - 1)));
+                    const bool loc = v < INF && !nl;
+                    if (SPL > 0) { vrow[k] = v; lrow[k] = loc; }
+                    tmin = min(tmin, v);
+                    if (v < INF && nl && v < bt) { bt = v; bs = SRC_SERVER + g; }
+                }
+                // warp argmin of (time bits, source id) over non-local events; warp min over all pending times
+                warp_keys(bt, bs, tmin, tint, src, tmin_all);
             }
-            // warp argmin of (time bits, source id) over non-local events; warp min over all pending times
-            warp_keys(bt, bs, tmin, tint, src, tmin_all);
             if (tint > tend_bits && tmin_all > tend_bits) return true;     // nothing left up to T_end
             if (budget == 0) return false;
             --budget;
             ++rounds;
-            unsigned long long wt, lim_t;
-            uint32_t lim_s;
-            round_limit(tint, src, tmin_all, tend_bits, wt, lim_t, lim_s);
-            bool progressed = local_arrivals(lim_t, lim_s);
+            // no iteration that starts in this round can end before T_min + tau_min
+            unsigned long long wt = INF;
+            if (tmin_all < INF)
+                wt = (unsigned long long)__double_as_longlong(__dadd_rn(__longlong_as_double((long long)tmin_all), tau_min));
+            // local ends strictly before the limit key min{(T_int, src), (W, 0), (T_end, max)}
+            unsigned long long lim_t = tint;
+            uint32_t lim_s = src;
+            if (wt <= lim_t) { lim_t = wt; lim_s = 0; }
+            if (tend_bits < lim_t) { lim_t = tend_bits; lim_s = NONE32; }
+            bool progressed = false;
+            if (F & F_MW) {
+                if (lane == 0) { cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M; cmd->force = force_nonlocal; }
+                __syncthreads();
+            }
+            if (lane < (int)p.I && n_idle_pf == 0 && !force_nonlocal) {
+                // local arrivals of this lane's class, in time order, up to the limit and up to the class's own
+                // next abandonment (which each arrival moves)
+                ClassState &c = cs[lane];
+                for (int guard = 0; guard < 64; ++guard) {
+                    const unsigned long long v = (unsigned long long)__double_as_longlong(c.ta);
+                    if (!(v < lim_t || (v == lim_t && SRC_ARRIVAL + (uint32_t)lane < lim_s))) break;
+                    if (f_abandon() && v > (unsigned long long)__double_as_longlong(c.abp.t_ab)) break;
+                    arrival_local();
+                    progressed = true;
+                }
+            }
+            // a class that ran out of draws has an unknown next arrival, possibly before T_int, and a local
+            // arrival may have pulled its class's next abandonment before T_int: then T_int is not next after all
+            bool redo = sched_pending;
+            if (f_abandon() && lane < (int)p.I) {
+                const unsigned long long v = (unsigned long long)__double_as_longlong(cs[lane].abp.t_ab);
+                redo = redo || v < tint || (v == tint && SRC_ABP + (uint32_t)lane < src);
+            }
             // the non-local event happens in this round if it comes before anything a new iteration could bring
-            const bool any_redo = must_redo(tint, src);
+            const bool any_redo = __any_sync(FULL, redo);
             const bool do_event = !any_redo && tint < wt && tint <= tend_bits;
             // with unrolled rows the event GPU's iteration ends in pass 1 and its decodes retire in pass 2
             const uint32_t ev_g = (SPL > 0 && do_event && src >= SRC_SERVER) ? src - SRC_SERVER : NONE32;
             // pass 1: every lane ends the local iterations of its own GPUs (straight-line over the rows)
             uint32_t retire_rows = 0;
             if (SPL == 0) {
-                // run-time row count: ends and retirements row by row
-                if (ends_all(lim_t, lim_s, buffered)) progressed = true;
+                // run-time row count (and, with helpers, only this warp's rows): ends and retirements row by row
+                if (ends_share(lim_t, lim_s, buffered)) progressed = true;
+                if (F & F_MW) {
+                    const uint32_t mine = __ballot_sync(FULL, progressed);
+                    if (lane == 0) res[0].progressed = mine != 0;
+                    __syncthreads();
+                    if (lane < nwarps && res[lane].progressed) progressed = true;
+                }
             }
             if (SPL > 0) {
 #pragma unroll
@@ -1734,89 +1457,21 @@ struct Sim {
                 }
             }
             if (do_event) {
-                handle_event(tint, src);
+                t = __longlong_as_double((long long)tint);
+                if (src >= SRC_SERVER) {
+                    on_server(src - SRC_SERVER);
+                } else {
+                    if (f_abandon() && src >= SRC_ABD1) on_abandon_d(1, src - SRC_ABD1);
+                    else if (f_abandon() && src >= SRC_ABD0) on_abandon_d(0, src - SRC_ABD0);
+                    else if (f_abandon() && src >= SRC_ABP) on_abandon_p(src - SRC_ABP);
+                    else if (src >= SRC_ARRIVAL) on_arrival(src - SRC_ARRIVAL);
+                    else { ++events; load_block(blk + 1); drain_dirty = true; gate_dirty = true; n_idle_pf = count_idle_pf(); idle_hint = NONE32; }
+                }
                 if (err) return true;
+                dispatch();
+                force_nonlocal = false;
             } else if (!any_redo && !__any_sync(FULL, progressed)) {
                 err = ERR_INTERNAL;     // a round that neither ended an iteration nor handled an event: never spin
-                return true;
-            }
-        }
-    }
-
-    // Several warps per replication (master only; the helpers run helper_loop).  The candidates of a round come from the
-    // per-row summaries; the rows that hold an end at or below the limit are listed in the command and shared out.
-    __device__ bool run_mw()
-    {
-        const uint32_t rows = n_rows();
-        const unsigned long long INF = 0x7ff0000000000000ull;
-        const unsigned long long tend_bits = (unsigned long long)__double_as_longlong(T_end);
-        unsigned long long budget = p.event_budget;
-        for (;;) {
-            __syncwarp();
-            for (uint32_t need = __ballot_sync(FULL, sched_pending); need; need &= need - 1)
-                refill((uint32_t)__ffs((int)need) - 1u);
-            unsigned long long bt = INF, tmin = INF;
-            uint32_t bs = NONE32;
-            class_candidates(bt, bs, tmin);
-            const bool buffered = (dq_n0 | dq_n1) != 0;
-            const bool dec_nonlocal = buffered || overcap;
-            unsigned long long trow[MW_ROWS / 32];
-#pragma unroll
-            for (uint32_t j = 0; j < MW_ROWS / 32; ++j) {
-                const uint32_t r = (j << 5) + (uint32_t)lane;
-                trow[j] = INF;
-                if (r < rows) {
-                    trow[j] = rc_tmin[r];
-                    tmin = min(tmin, trow[j]);
-                    unsigned long long v;
-                    uint32_t sid;
-                    if (force_nonlocal) {
-                        v = trow[j]; sid = SRC_SERVER + rc_gmin[r];
-                        if (v < INF && (v < bt || (v == bt && sid < bs))) { bt = v; bs = sid; }
-                    } else {
-                        v = rc_tpf[r]; sid = SRC_SERVER + rc_gpf[r];
-                        if (v < INF && (v < bt || (v == bt && sid < bs))) { bt = v; bs = sid; }
-                        if (dec_nonlocal) {
-                            v = rc_tdec[r]; sid = SRC_SERVER + rc_gdec[r];
-                            if (v < INF && (v < bt || (v == bt && sid < bs))) { bt = v; bs = sid; }
-                        }
-                    }
-                }
-            }
-            unsigned long long tint, tmin_all;
-            uint32_t src;
-            warp_keys(bt, bs, tmin, tint, src, tmin_all);
-            if (tint > tend_bits && tmin_all > tend_bits) return true;     // nothing left up to T_end
-            if (budget == 0) return false;
-            --budget;
-            ++rounds;
-            unsigned long long wt, lim_t;
-            uint32_t lim_s;
-            round_limit(tint, src, tmin_all, tend_bits, wt, lim_t, lim_s);
-            // rows with an end at or below the limit time
-#pragma unroll
-            for (uint32_t j = 0; j < MW_ROWS / 32; ++j) {
-                const uint32_t todo = __ballot_sync(FULL, trow[j] <= lim_t && trow[j] < INF);
-                if (lane == 0) cmd->todo[j] = todo;
-            }
-            if (lane == 0) {
-                cmd->op = MW_ENDS; cmd->lim_t = lim_t; cmd->lim_s = lim_s; cmd->buffered = buffered; cmd->M = M;
-                cmd->force = force_nonlocal; cmd->overcap = overcap; cmd->prog = 0;
-            }
-            __syncthreads();
-            bool progressed = local_arrivals(lim_t, lim_s);
-            if (ends_rows(lim_t, lim_s, buffered)) progressed = true;
-            cp_async_wait_all();
-            if (__any_sync(FULL, progressed) && lane == 0) cmd->prog = 1u;
-            __syncthreads();
-            progressed = cmd->prog != 0;
-            const bool any_redo = must_redo(tint, src);
-            const bool do_event = !any_redo && tint < wt && tint <= tend_bits;
-            if (do_event) {
-                handle_event(tint, src);
-                if (err) return true;
-            } else if (!any_redo && !progressed) {
-                err = ERR_INTERNAL;
                 return true;
             }
         }
@@ -1830,26 +1485,25 @@ struct Sim {
         if (force_nonlocal) return false;
         const uint32_t na = nact[g];
         if (na & 0x8000u) return false;
-        if ((na & 0x4000u) && (buffered || ((F & F_MW) ? overcap : (g < M && ndec[g] > p.B - 1)))) return false;
+        if ((na & 0x4000u) && (buffered || (g < M && ndec[g] > p.B - 1))) return false;
         return true;
     }
 };
 
-// shared-memory carve-up for one replication (one block)
+// shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
-    uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
-        off_pfcur, off_hw, off_hint, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte,
-        off_pqh, off_wcs, off_cmd, off_rc, total;
+    uint32_t off_tnext, off_tarr, off_tau, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
+        off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, off_wcs, off_cmd, off_res, total;
 };
 
-// mw: the block runs the several-warps instance (per-row summaries and the command block exist)
 __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps = 1,
-                                                  bool kappa = true, bool mw = false)
+                                                  bool kappa = true)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.off_tnext = o; o += 8 * Npad;
     L.off_tarr = o; o += 8 * Npad;
+    L.off_tau = o; o += 8 * Npad;
     L.off_it = o; o += 4 * Npad;
     L.off_nfin = o; o += 4 * Npad;
     L.off_pfrem = o; o += 4 * Npad;
@@ -1859,8 +1513,6 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_ndec = o; o += 2 * Npad;
     L.off_nact = o; o += 2 * Npad;
     L.off_pfcur = o; o += 2 * Npad;
-    L.off_hw = o; if (!slots_smem) o += 2 * Npad;     // slot records in global memory: never-used mark and free-slot hint
-    L.off_hint = o; if (!slots_smem) o += 2 * Npad;
     o = (o + 15u) & ~15u;
     L.off_sfin16 = o; if (slots_smem) o += 2 * Npad * B;
     o = (o + 15u) & ~15u;
@@ -1874,15 +1526,14 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
     o = (o + 15u) & ~15u;
     L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * MAXI;
-    const uint32_t cap = mw ? (uint32_t)STAGE_CAP_MW : (uint32_t)STAGE_CAP;
-    L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * cap * nwarps;
-    L.off_stte = o; o += 8 * cap * nwarps;
+    L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * STAGE_CAP;
+    L.off_stte = o; o += 8 * STAGE_CAP;
     L.off_pqh = o; o += (uint32_t)sizeof(QEntry) * MAXI;
     L.off_wcs = o; o += (uint32_t)sizeof(WarpClassStats) * MAXI * nwarps;
     o = (o + 15u) & ~15u;
-    L.off_cmd = o; if (mw) o += (uint32_t)sizeof(MwCmd);
+    L.off_cmd = o; o += (uint32_t)sizeof(MwCmd);
     o = (o + 15u) & ~15u;
-    L.off_rc = o; if (mw) o += (3u * 8u + 7u * 4u) * (Npad >> 5);
+    L.off_res = o; o += (uint32_t)sizeof(MwRes) * MW_MAX;
     L.total = (o + 15u) & ~15u;
     return L;
 }
@@ -1892,6 +1543,7 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
 {
     s.tnext = reinterpret_cast<double *>(sm + L.off_tnext);
     s.pf_tarr = reinterpret_cast<double *>(sm + L.off_tarr);
+    s.taucur = reinterpret_cast<double *>(sm + L.off_tau);
     s.it = reinterpret_cast<uint32_t *>(sm + L.off_it);
     s.nfin = reinterpret_cast<uint32_t *>(sm + L.off_nfin);
     s.pfrem = reinterpret_cast<uint32_t *>(sm + L.off_pfrem);
@@ -1901,8 +1553,6 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.ndec = reinterpret_cast<uint16_t *>(sm + L.off_ndec);
     s.nact = reinterpret_cast<uint16_t *>(sm + L.off_nact);
     s.pfcur = reinterpret_cast<uint16_t *>(sm + L.off_pfcur);
-    s.hw = reinterpret_cast<uint16_t *>(sm + L.off_hw);
-    s.hint = reinterpret_cast<uint16_t *>(sm + L.off_hint);
     s.sfin16 = reinterpret_cast<uint16_t *>(sm + L.off_sfin16);
     s.socc = reinterpret_cast<uint32_t *>(sm + L.off_socc);
     s.touch = reinterpret_cast<uint32_t *>(sm + L.off_touch);
@@ -1911,33 +1561,18 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.gate_ok = reinterpret_cast<uint32_t *>(s.gate_dq + MAXI);
     s.cs = reinterpret_cast<ClassState *>(sm + L.off_cs);
     s.aring = reinterpret_cast<ADraw *>(sm + L.off_ring);
-    // every warp stages the records of the requests it retires in its own part
-    s.stage_cap = (F & F_MW) ? (uint32_t)STAGE_CAP_MW : (uint32_t)STAGE_CAP;
-    s.st_rec = reinterpret_cast<SlotRec *>(sm + L.off_strec) + (size_t)s.warp * s.stage_cap;
-    s.st_te = reinterpret_cast<double *>(sm + L.off_stte) + (size_t)s.warp * s.stage_cap;
+    s.st_rec = reinterpret_cast<SlotRec *>(sm + L.off_strec);
+    s.st_te = reinterpret_cast<double *>(sm + L.off_stte);
     s.pqh = reinterpret_cast<QEntry *>(sm + L.off_pqh);
     s.wcs = reinterpret_cast<WarpClassStats *>(sm + L.off_wcs);
     s.cmd = reinterpret_cast<MwCmd *>(sm + L.off_cmd);
-    {
-        const uint32_t rows = s.p.Npad >> 5;
-        s.rc_tmin = reinterpret_cast<unsigned long long *>(sm + L.off_rc);
-        s.rc_tpf = s.rc_tmin + rows;
-        s.rc_tdec = s.rc_tpf + rows;
-        s.rc_gmin = reinterpret_cast<uint32_t *>(s.rc_tdec + rows);
-        s.rc_gpf = s.rc_gmin + rows;
-        s.rc_gdec = s.rc_gpf + rows;
-        s.rc_ksolo = s.rc_gdec + rows;
-        s.rc_kmix = s.rc_ksolo + rows;
-        s.rc_kpf = s.rc_kmix + rows;
-        s.rc_cnt = s.rc_kpf + rows;
-    }
-    s.overcap = false;
+    s.res = reinterpret_cast<MwRes *>(sm + L.off_res);
     s.n_pend = 0;
     s.rec_after = 0;
     s.ring_n = 0; s.ring_pos = 0; s.sched_pending = false; s.t0_pending = 0.0;
     const Params &p = s.p;
     const size_t r = s.rep;
-    s.s_fin = p.slot_fin + r * (size_t)p.N * p.Bp;
+    s.s_fin = p.slot_fin + r * (size_t)p.N * p.B;
     s.s_rec = p.slot_rec + r * (size_t)p.N * p.B;
     s.pq = p.pq + r * (size_t)p.I * p.qcap;
     s.dq = p.dq + r * (size_t)2 * p.qcap;
@@ -1959,8 +1594,6 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
         for (uint32_t o = lane * 4; o < L.total; o += 128) *reinterpret_cast<uint32_t *>(sm + o) = 0;
         __syncwarp();
         for (uint32_t g = lane; g < p.Npad; g += 32) { s.tnext[g] = dinf(); s.nfin[g] = NONE32; }
-        if (!p.slots_smem)
-            for (uint32_t g = lane; g < p.Npad; g += 32) s.hint[g] = (uint16_t)NOHINT;     // hw = 0: no slot used yet
         if (p.slots_smem && (p.B & 31u)) {
             const uint32_t bw = (p.B + 31u) >> 5;
             for (uint32_t g = lane; g < p.Npad; g += 32) s.socc[g * bw + bw - 1] = ~0u << (p.B & 31u);
@@ -2014,7 +1647,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_ke
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0, (FT & F_MW) != 0);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0);
         Sim<SPLT, FT> s(p, lane, rep);
         s.warp = warp;
         s.nwarps = (int)(nthr >> 5);
@@ -2051,11 +1684,6 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_ke
         s.idle_hint = NONE32;
         s.it_mixed = 0; s.it_solo = 0; s.busy_mixed = 0.0; s.busy_solo = 0.0;
         bool finished = true;
-        if (FT & F_MW) {
-            // the per-row summaries are derived state: every warp builds its share
-            for (uint32_t k = (uint32_t)warp; k < (p.Npad >> 5); k += (uint32_t)s.nwarps) { s.refresh_time(k); s.refresh_load(k); }
-            __syncthreads();
-        }
         if (warp == 0) {
             s.n_idle_pf = s.count_idle_pf();
             if (lane < (int)p.I && s.cs[lane].pq_n > 0) s.pqh[lane] = s.pq[(size_t)lane * p.qcap + s.cs[lane].pq_head];

@@ -45,8 +45,7 @@ struct qsim {
     qsim_class cls[QSIM_MAXI]{};
     double prices[2]{};
     Params par{};
-    SmemLayout lay{};             // shared memory of the run kernel's block
-    uint32_t init_smem = 0;       // shared memory of the init kernel's block (one warp, same per-GPU image)
+    SmemLayout lay{};
     Sections sec{};
     BlockPar *d_blocks = nullptr;
     uint32_t *d_lengths = nullptr;
@@ -63,7 +62,6 @@ struct qsim {
     int device = 0;
     void (*run_fn)(qsimdev::Params) = nullptr;
     uint32_t nwarps = 1;          // warps per replication (block size / 32)
-    bool mw = false;              // the several-warps instance runs this handle
 };
 
 namespace {
@@ -72,10 +70,10 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
 {
     Sections s{};
     size_t o = 0;
-    const size_t R = c.R, NB = (size_t)c.N * c.B, NBp = (size_t)c.N * ((c.B + 3u) & ~3u);
+    const size_t R = c.R, NB = (size_t)c.N * c.B;
     s.hdr = o; o = align256(o + R * sizeof(RepHeader));
     s.srv = o; o = align256(o + R * (size_t)srv_bytes);
-    s.fin = o; o = align256(o + R * NBp * 4);     // finish stamps: rows of B rounded up to four entries (16-byte loads)
+    s.fin = o; o = align256(o + R * NB * 4);
     s.rec = o; o = align256(o + R * NB * sizeof(SlotRec));
     s.pq = o; o = align256(o + R * (size_t)c.I * c.qcap * sizeof(QEntry));
     s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
@@ -211,18 +209,17 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
     return f;
 }
 
-// Large clusters run the several-warps instance: the master warp handles the events, all warps share the local
-// iteration ends row by row, and per-row summaries keep the master's searches short.  QSIM_WARPS overrides the number of
-// warps per replication (0 = always the one-warp instances).
-void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps, bool &mw)
+// Large clusters: per-replication shared memory allows only a few blocks per SM, so each replication gets
+// several warps (master + helpers) that share the per-GPU scans.  QSIM_WARPS overrides the choice (1 = off).
+void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
-    uint32_t W = rows >= 64 ? 8u : (rows >= 16 ? 4u : 0u);
+    uint32_t W = rows >= 64 ? 16u : (rows >= 16 ? 4u : 1u);
     if (const char *e = std::getenv("QSIM_WARPS")) {
         const int v = std::atoi(e);
-        if (v >= 0 && v <= MW_MAX) W = (uint32_t)v;
+        if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
     }
-    if (W == 0 || rows < 2) return;
+    if (W <= 1 || rows < 2) return;
     const char *force = std::getenv("QSIM_KERNEL");
     const bool generic_only = force && std::strcmp(force, "generic") == 0;
     // mode bits must match exactly, capability bits may be present unused (as in pick_run_kernel)
@@ -238,9 +235,8 @@ void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint3
     }
     fn = best->fn;
     nwarps = W;
-    mw = true;
     p.Npad = rows * 32u;
-    p.slots_smem = 0;       // every warp retires through the slot records in global memory
+    p.slots_smem = 0;       // helpers retire through the global slot lists
 }
 
 RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
@@ -301,14 +297,10 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     if (p.slots_smem) v = pick_run_kernel(cfg.N, feat | F_SLOTS);
     h.run_fn = v.fn;
     h.nwarps = 1;
-    bool mw = false;
-    choose_multiwarp(cfg.N, feat, p, h.run_fn, h.nwarps, mw);
-    h.mw = mw;
-    p.Bp = (cfg.B + 3u) & ~3u;
-    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa, mw);
-    h.init_smem = smem_layout(p.Npad, p.B, p.slots_smem, 1, kappa, false).total;
+    choose_multiwarp(cfg.N, feat, p, h.run_fn, h.nwarps);
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa);
     p.srv_bytes = h.lay.srv_bytes;
-    if (h.lay.total > 227u * 1024u || h.init_smem > 227u * 1024u)
+    if (h.lay.total > 227u * 1024u)
         return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     h.sec = layout_sections(cfg, p.srv_bytes);
     return QSIM_OK;
@@ -439,7 +431,7 @@ int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
 {
     int rc = attach_workspace(h, ws, bytes, cuda_stream);
     if (rc != QSIM_OK) return rc;
-    qsim_init_kernel<<<h->cfg.R, 32, h->init_smem, h->stream>>>(h->par);
+    qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     h->bound = true;
@@ -515,7 +507,7 @@ int qsim_set_injected(qsim_t *h, const double *t, const uint32_t *job, uint64_t 
     h->par.n_inject = (uint32_t)n;
     // the trace source lives in the run-time-configured instance
     RunVariant v = pick_run_kernel(h->cfg.N, ~0u);
-    if (h->mw)
+    if (h->nwarps > 1)
         for (const RunVariant &mw : run_variants())
             if (mw.spl < 0 && (mw.feat & F_GENERIC)) v = mw;
     h->run_fn = v.fn;
@@ -870,7 +862,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     CUDA_TRY(allow_large_smem(reinterpret_cast<const void *>(qsim_init_kernel)));
     // the array keeps the previous call's contents: the init kernel rewrites every header and GPU image;
     // queue rings and slot lists are never read before they are written, the flag is cleared per launch
-    qsim_init_kernel<<<cfg->R, 32, h.init_smem, stream>>>(p);
+    qsim_init_kernel<<<cfg->R, 32, h.lay.total, stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     bool advance = true;
     for (;;) {
