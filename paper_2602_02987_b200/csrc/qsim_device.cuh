@@ -81,6 +81,7 @@ struct RepHeader {
     double T_end, T_reset;
     unsigned long long place_ord, events, H_total, rounds;
     uint32_t blk, done, err, force;    // force: the next event must be followed by a dispatch (targets were replaced)
+    double t_now, t_pad;               // time of the last event handled (one-thread-per-replication kernels)
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
     unsigned long long sel_ord0, sel_ord1;   // class selections drawn so far in the solo / mixed pool (general SLI router)
     unsigned long long iters_mixed[32], iters_solo[32];
@@ -100,6 +101,25 @@ struct QEntry { double t; uint32_t pk; uint32_t cls; };   // 16 bytes: prefill q
 
 struct ClassPar { double theta; uint32_t P, D, prio, pad; };
 struct BlockPar { uint32_t M, pad; double xstar[MAXI], nx[MAXI], nq[MAXI], ps[MAXI], rate[MAXI], ws[MAXI], wm[MAXI]; };
+
+// Shapes and arrays of the one-thread-per-replication family (qsim_lane.cuh); arrays are [R][...]
+struct LaneSrv;
+struct LanePar {
+    uint32_t on;                 // this handle runs that family
+    uint32_t nbk;                // calendar buckets (power of two); every pending iteration end lies less than nbk buckets ahead
+    uint32_t tlev, toff[6], tsize;   // eligibility trees: internal levels, offset of every level (0 = leaves) and entries per tree
+    uint32_t b8, slev, soff[5], ssize;   // slot trees: leaves per GPU, internal levels, offsets of levels 1.. and nodes per GPU
+    double inv_w;                // buckets per second
+    LaneSrv *srv;                // [N] GPU records
+    double *tarr;                // [N] arrival time of the request in prefill
+    uint16_t *cal_head;          // [nbk] first GPU of every bucket
+    uint32_t *cal_bm;            // [nbk/32] non-empty buckets
+    uint32_t *tree;              // [3][tsize] solo decode, mixed decode, prefill
+    uint32_t *sfin;              // [N][b8] finish iteration per slot (NONE32 = free)
+    unsigned long long *snode;   // [N][ssize] minimum of finish << 16 | slot per group of eight
+    SlotRec *srec;               // [N][B] request in each slot
+    uint16_t *sfree;             // [N][B] entries at and above the GPU's decode count are its free slots
+};
 
 struct Params {
     uint32_t I, N, Npad, R, B, C, nblk, gate, router, placement, length_mode, qcap, hist, advance, any_theta, slots_smem;
@@ -123,6 +143,7 @@ struct Params {
     uint32_t *hist_mem;          // [R][I][2][NBIN] or null
     uint32_t *not_done;          // single counter: replications that stopped on the event budget
     uint32_t srv_bytes;
+    LanePar lane;
 };
 
 // ---------------------------------------------------------------------------------------------

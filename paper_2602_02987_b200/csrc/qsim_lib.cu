@@ -4,6 +4,7 @@
 // without a CUDA device every entry point that needs one fails with QSIM_ECUDA.
 #include "qsim.h"
 #include "qsim_device.cuh"
+#include "qsim_lane.cuh"
 
 #include <cmath>
 #include <cstdio>
@@ -36,6 +37,8 @@ size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 struct Sections {
     size_t hdr, srv, fin, rec, pq, dq, hist, flag, total;
+    // one-thread-per-replication family
+    size_t l_srv, l_tarr, l_head, l_bm, l_tree, l_sfin, l_snode, l_srec, l_sfree;
 };
 
 }  // namespace
@@ -62,6 +65,8 @@ struct qsim {
     int device = 0;
     void (*run_fn)(qsimdev::Params) = nullptr;
     uint32_t nwarps = 1;          // warps per replication (block size / 32)
+    bool allow_lane = true;       // the one-thread-per-replication family may run this handle
+    double coef[6]{};
 };
 
 namespace {
@@ -81,6 +86,75 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
     s.flag = o; o = align256(o + 256);
     s.total = o;
     return s;
+}
+
+Sections lane_sections(const qsim_config &c, const LanePar &q)
+{
+    Sections s{};
+    size_t o = 0;
+    const size_t R = c.R, N = c.N;
+    s.hdr = o; o = align256(o + R * sizeof(RepHeader));
+    s.l_srv = o; o = align256(o + R * N * sizeof(LaneSrv));
+    s.l_tarr = o; o = align256(o + R * N * 8);
+    s.l_head = o; o = align256(o + R * (size_t)q.nbk * 2);
+    s.l_bm = o; o = align256(o + R * (size_t)(q.nbk / 32u) * 4);
+    s.l_tree = o; o = align256(o + R * 3 * (size_t)q.tsize * 4);
+    s.l_sfin = o; o = align256(o + R * N * (size_t)q.b8 * 4);
+    s.l_snode = o; o = align256(o + R * N * (size_t)q.ssize * 8);
+    s.l_srec = o; o = align256(o + R * N * (size_t)c.B * sizeof(SlotRec));
+    s.l_sfree = o; o = align256(o + R * N * (size_t)c.B * 2);
+    s.pq = o; o = align256(o + R * (size_t)c.I * c.qcap * sizeof(QEntry));
+    s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
+    s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
+    s.flag = o; o = align256(o + 256);
+    s.total = o;
+    return s;
+}
+
+// 8-ary tree over n leaves: number of internal levels, offset of every level (level 0 = leaves) and total entries;
+// every level is padded to a multiple of eight entries.
+void tree_shape(uint32_t n, uint32_t &lev, uint32_t *off, uint32_t &size)
+{
+    uint32_t m = (n + 7u) & ~7u, o = 0;
+    lev = 0;
+    off[0] = 0;
+    for (;;) {
+        o += m;
+        const uint32_t parents = (m + 7u) / 8u;
+        ++lev;
+        off[lev] = o;
+        if (parents == 1) { size = o + 8u; return; }
+        m = (parents + 7u) & ~7u;
+    }
+}
+
+// Which configurations the one-thread-per-replication family simulates: every gate, the solo-first and the SLI-aware
+// router with least-loaded placement, abandonment, blocks, histograms; no KV slope, no trace replay.
+bool lane_supports(const qsim_config &c, const double *coef)
+{
+    return (c.router == QSIM_ROUTER_SOLO_FIRST || c.router == QSIM_ROUTER_SLI) && c.placement == QSIM_PLACE_LEAST_LOADED &&
+           coef[5] == 0.0 && c.N <= 4096 && c.B <= 4096;
+}
+
+// Shapes of the family's structures (no pointers yet)
+void lane_shapes(const qsim_config &c, const double *coef, LanePar &q)
+{
+    std::memset(&q, 0, sizeof q);
+    q.on = 1;
+    uint32_t nbk = 64;
+    while (nbk < 4u * c.N) nbk <<= 1;
+    q.nbk = nbk;
+    // no iteration lasts longer than tau_max, so with (nbk - 2) buckets per 1.01 tau_max every pending end lies less
+    // than one revolution of the calendar ahead of the current time
+    const double tau_mix = coef[0] + coef[1] * (double)c.C + coef[2] * (double)c.B, tau_solo = coef[3] + coef[4] * (double)c.B;
+    const double tau_max = tau_mix > tau_solo ? tau_mix : tau_solo;
+    q.inv_w = (double)(nbk - 2u) / (1.01 * tau_max);
+    tree_shape(c.N, q.tlev, q.toff, q.tsize);
+    q.b8 = (c.B + 7u) & ~7u;
+    uint32_t off[6], size = 0;
+    tree_shape(c.B, q.slev, off, size);
+    for (uint32_t l = 0; l < q.slev; ++l) q.soff[l] = off[l + 1] - off[1];      // internal levels only: the leaves are a separate array
+    q.ssize = size - off[1];
 }
 
 int validate(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
@@ -271,7 +345,7 @@ RunVariant pick_run_kernel(uint32_t N, uint32_t feat)
 int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const double *prices, const double *coef)
 {
     h.cfg = cfg;
-    std::memcpy(h.cls, classes, cfg.I * sizeof(qsim_class));
+    if (classes != h.cls) std::memcpy(h.cls, classes, cfg.I * sizeof(qsim_class));
     h.prices[0] = prices[0];
     h.prices[1] = prices[1];
     Params &p = h.par;
@@ -303,6 +377,20 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     if (h.lay.total > 227u * 1024u)
         return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     h.sec = layout_sections(cfg, p.srv_bytes);
+    for (int k = 0; k < 6; ++k) h.coef[k] = coef[k];
+    // Kernel family.  One thread per replication pays when there are enough replications to fill the device with
+    // independent chains; a warp per replication is faster for few replications.  QSIM_FAMILY=lane / warp overrides.
+    std::memset(&p.lane, 0, sizeof p.lane);
+    bool lane = h.allow_lane && lane_supports(cfg, coef) && cfg.R >= 2048u;
+    if (const char *e = std::getenv("QSIM_FAMILY")) {
+        if (std::strcmp(e, "lane") == 0) lane = h.allow_lane && lane_supports(cfg, coef);
+        else if (std::strcmp(e, "warp") == 0) lane = false;
+    }
+    if (lane) {
+        lane_shapes(cfg, coef, p.lane);
+        h.sec = lane_sections(cfg, p.lane);
+        h.nwarps = 0;
+    }
     return QSIM_OK;
 }
 
@@ -339,7 +427,8 @@ int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
     p.force_dispatch = h->targets_changed ? 1u : 0u;
     h->targets_changed = false;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
+    if (p.lane.on) qsim_lane_run_kernel<<<(h->cfg.R + 31u) / 32u, 32, 0, h->stream>>>(p);
+    else h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
@@ -424,6 +513,18 @@ static int attach_workspace(qsim_t *h, void *ws, size_t bytes, void *cuda_stream
     p.dq = reinterpret_cast<QEntry *>(base + h->sec.dq);
     p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h->sec.flag);
+    if (p.lane.on) {
+        LanePar &q = p.lane;
+        q.srv = reinterpret_cast<LaneSrv *>(base + h->sec.l_srv);
+        q.tarr = reinterpret_cast<double *>(base + h->sec.l_tarr);
+        q.cal_head = reinterpret_cast<uint16_t *>(base + h->sec.l_head);
+        q.cal_bm = reinterpret_cast<uint32_t *>(base + h->sec.l_bm);
+        q.tree = reinterpret_cast<uint32_t *>(base + h->sec.l_tree);
+        q.sfin = reinterpret_cast<uint32_t *>(base + h->sec.l_sfin);
+        q.snode = reinterpret_cast<unsigned long long *>(base + h->sec.l_snode);
+        q.srec = reinterpret_cast<SlotRec *>(base + h->sec.l_srec);
+        q.sfree = reinterpret_cast<uint16_t *>(base + h->sec.l_sfree);
+    }
     return QSIM_OK;
 }
 
@@ -431,7 +532,8 @@ int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
 {
     int rc = attach_workspace(h, ws, bytes, cuda_stream);
     if (rc != QSIM_OK) return rc;
-    qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
+    if (h->par.lane.on) qsim_lane_init_kernel<<<(h->cfg.R + 31u) / 32u, 32, 0, h->stream>>>(h->par);
+    else qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     h->bound = true;
@@ -492,6 +594,16 @@ int qsim_set_injected(qsim_t *h, const double *t, const uint32_t *job, uint64_t 
     if (!h || !t || !job || n == 0 || n > 0x7fffffffull) return fail(QSIM_EINVAL, "bad injected arrival list");
     if (h->bound) return fail(QSIM_ESTATE, "qsim_set_injected must come before qsim_bind");
     if (h->cfg.nblk != 1) return fail(QSIM_EINVAL, "injected arrivals need nblk == 1");
+    if (h->par.lane.on) {
+        // trace replay lives in the warp-per-replication family: lay the handle out again for it
+        h->allow_lane = false;
+        int rc = configure(*h, h->cfg, h->cls, h->prices, h->coef);
+        if (rc != QSIM_OK) return rc;
+        h->par.blocks = h->d_blocks;
+        h->par.lengths = h->d_lengths;
+        cudaError_t e = allow_large_smem(reinterpret_cast<const void *>(h->run_fn));
+        if (e != cudaSuccess) return fail(QSIM_ECUDA, cudaGetErrorString(e));
+    }
     for (uint64_t k = 0; k < n; ++k) {
         if (!(t[k] >= 0.0) || !std::isfinite(t[k]) || (k > 0 && t[k] < t[k - 1])) return fail(QSIM_EINVAL, "injected times must be ascending and >= 0");
         if (job[3 * k] >= h->cfg.I || job[3 * k + 1] < 1 || job[3 * k + 1] > QSIM_LMAX || job[3 * k + 2] < 1 || job[3 * k + 2] > QSIM_LMAX)
@@ -556,7 +668,7 @@ int qsim_layout_info(const qsim_t *h, uint64_t out[4])
 {
     if (!h || !out) return fail(QSIM_EINVAL, "null argument");
     out[0] = sizeof(RepHeader);          // bytes per replication copied to the host by qsim_stats
-    out[1] = h->lay.srv_bytes;           // bytes of per-GPU state staged per replication at kernel entry and exit
+    out[1] = h->par.lane.on ? 0 : h->lay.srv_bytes;   // bytes of per-GPU state staged per replication at kernel entry and exit
     out[2] = h->lay.total;               // shared memory per block
     out[3] = h->nwarps;                  // warps per replication
     return QSIM_OK;
@@ -734,6 +846,18 @@ int qsim_server_state(qsim_t *h, uint32_t r, uint32_t *n_dec, uint32_t *it, doub
     if (!h) return fail(QSIM_EINVAL, "null handle");
     if (!h->bound) return fail(QSIM_ESTATE, "qsim_server_state before qsim_bind");
     if (r >= h->cfg.R) return fail(QSIM_EINVAL, "replication index out of range");
+    if (h->par.lane.on) {
+        std::vector<LaneSrv> rec(h->cfg.N);
+        CUDA_TRY(cudaMemcpyAsync(rec.data(), h->par.lane.srv + (size_t)r * h->cfg.N, rec.size() * sizeof(LaneSrv), cudaMemcpyDeviceToHost, h->stream));
+        CUDA_TRY(cudaStreamSynchronize(h->stream));
+        for (uint32_t g = 0; g < h->cfg.N; ++g) {
+            if (n_dec) n_dec[g] = rec[g].ndec;
+            if (it) it[g] = rec[g].it;
+            if (t_next) t_next[g] = rec[g].tnext;
+            if (pf_rem) pf_rem[g] = (rec[g].pfjob >> 31) ? rec[g].pfrem : 0u;
+        }
+        return QSIM_OK;
+    }
     std::vector<char> img(h->lay.srv_bytes);
     CUDA_TRY(cudaMemcpyAsync(img.data(), h->par.srv + (size_t)r * h->lay.srv_bytes, img.size(), cudaMemcpyDeviceToHost, h->stream));
     CUDA_TRY(cudaStreamSynchronize(h->stream));
@@ -823,6 +947,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
     qsim h;   // a handle that owns nothing: no table allocation, no pinned flag
+    h.allow_lane = false;                  // the built-in scratch is sized for the warp-per-replication layout
     qsim_config nohist = *cfg;
     nohist.hist = 0;                       // histograms are not recorded here
     rc = configure(h, nohist, classes, prices, coef);
