@@ -1,21 +1,25 @@
 #!/usr/bin/env python
-"""Benchmark: simulated GPU-server-iterations per second on the two-class lognormal workload (cfg1).
+"""Benchmark: simulated GPU-server-iterations per second.
 
-One step = one pass of the whole hot path (arrivals, next-event selection, iteration completion,
-accounting, decode routing, prefill gate, abandonment clocks, iteration starts, state staging) over one
-batch: all R = 1024 replications of N = 64 simulated GPUs advance by 10^5 iterations of horizon.  Steps
-continue the same simulation, so the timed steps run in steady state.
+Default workload: cfg2, the largest configuration that is resident whole on one GPU (four lognormal classes at 1.05 of
+the fluid capacity, N = 512 simulated GPUs, B = 256, R = 4096 replications per GPU).  One step = one pass of the whole
+hot path (arrivals, next-event selection, iteration completion, accounting, decode routing, prefill gate, abandonment
+clocks, iteration starts, statistics reduction) over one batch: all R replications advance by `--horizon` iterations of
+horizon.  Steps continue the same simulation after a warm-up of at least 2000 iterations of horizon, so the timed steps
+run in steady state.
 
     python bench.py --gpus N --steps K --warmup W          (N > 1: launched under torchrun, one rank per GPU)
     python bench.py --impl reference ...                   (the CPU oracle, timed on the host cores)
+    python bench.py --workload cfg1 | cfg0 | cfg3 | cfg4 --cluster N | ctmc      (the other configurations)
 
-Prints one JSON line.  `value` is timed with CUDA events around qsim_run with all state resident in HBM;
-`e2e` is the same metric through qsim_simulate with host buffers (tables copied in, statistics copied out,
-device memory allocated and freed inside the timed region).
+Prints one JSON line.  `value` is timed with CUDA events around qsim_run with all state resident in HBM; `e2e` is the
+same metric through qsim_simulate with host buffers (tables copied in, totals copied out, device memory allocated and
+freed inside the timed region).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -32,21 +36,12 @@ METRIC = "simulated GPU-server-iterations/sec"
 UNIT = "server-iterations/s"
 JOB_BYTES = 128            # algorithmic bytes per request life cycle: queue entry, prefill record, decode slot,
                            # decode-buffer pass, each written and read once at 32-byte sector granularity
-# DRAM bytes per simulated server-iteration of qsim_run_kernel on cfg1, from an ncu capture of a 2000-iteration
-# launch (dram__bytes_read.sum + dram__bytes_write.sum = 734.9 MB for 1.415e8 iterations); traffic grows with the
-# iterations of a launch, so a full launch is that figure times its iterations
-NCU_DRAM_BYTES_PER_ITER = 734.9e6 / 1.415e8
-# warp instructions per simulated server-iteration of the same capture (smsp__inst_executed.sum = 3.224e10)
-NCU_WARP_INST_PER_ITER = 3.224e10 / 1.415e8
-# exponential-service kernel, capture of a 1-second launch at R = 37888: 4.238e9 warp instructions for 8.339e7 jumps and
-# 160.5 MB + 191.4 MB of DRAM traffic (the replication records once, plus the counters and integrals that are added to in
-# place; the latter grows with the simulated time, so a longer launch has no traffic figure)
-NCU_CTMC_WARP_INST_PER_JUMP = 4.238e9 / 8.339e7
-NCU_CTMC_DRAM_BYTES_PER_LAUNCH = 351.9e6
-# issue peak of the GPU: 148 SMs x 4 schedulers x one warp instruction per cycle at the maximum SM clock
-ISSUE_PEAK = 148 * 4 * 1.965e9
-HORIZON = 100_000          # iterations of horizon per step (cfg1)
-R_PER_GPU = 1024
+N_SM, SCHEDULERS = 148, 4  # issue peak of the GPU: SMs x schedulers x one warp instruction per cycle x SM clock
+PREWARM = 2000             # iterations of horizon before the warm-up steps (steady state)
+
+# workload -> (replications per GPU, iterations of horizon per step)
+DEFAULTS = {"cfg2": (4096, 400), "cfg1": (1024, 100_000), "cfg0": (16, 10_000), "cfg3": (2048, 300), "cfg4": (8192, 300)}
+CSRC = os.path.join(ROOT, "paper_2602_02987_b200", "csrc")
 
 
 def measured_peaks():
@@ -55,6 +50,28 @@ def measured_peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def kernel_source_id() -> str:
+    """Fingerprint of the kernel sources: profile counters are only quoted for the sources they were taken with."""
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(CSRC)):
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(name.encode()); h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def profile_counters(key: str):
+    """Counters of an ncu capture kept beside its summary under profiles/ (per simulated server-iteration, or per jump):
+    None when there is no capture for this workload or the kernels changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", "counters.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as f:
+        rec = json.load(f).get(key)
+    if not rec or rec.get("kernel_source_id") != kernel_source_id():
+        return None
+    return rec
 
 
 class ClockSampler:
@@ -104,10 +121,42 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def make_inputs(workload: str, reps: int, horizon: int, cluster: int):
+    from qsim_inputs import presets
+    kw = {"N": cluster} if cluster else {}
+    if workload == "cfg1":
+        return presets.cfg1(R=reps)
+    if workload == "cfg0":
+        return presets.cfg0(R=reps, horizon_iters=horizon)
+    if workload == "cfg3":
+        return presets.cfg3(R=reps, block_len=1.0, **kw)      # 24 blocks of 1 s instead of one hour each
+    return getattr(presets, workload)(R=reps, horizon_iters=horizon, **kw)
+
+
+def describe(workload: str, inp, reps: int, horizon: int) -> str:
+    what = {"cfg0": "2 fixed-length classes, occupancy gate, solo-first router, bundled pricing",
+            "cfg1": "2 lognormal classes, priority gate, solo-first router, separate pricing",
+            "cfg2": "4 lognormal classes at 1.05 of the fluid capacity, occupancy gate, solo-first router, abandonment, bundled pricing",
+            "cfg3": "4 lognormal classes, 24 blocks of 1 s (sinusoidal demand, per-block LP targets), priority gate, histograms",
+            "cfg4": "cfg2 workload under constrained-LP targets, SLI-aware router, histograms"}[workload]
+    return (f"{workload}: {what}; N={inp.N} GPUs, B={inp.B}, C={inp.C}, least-loaded placement, R={reps} replications per GPU, "
+            f"{horizon} iterations of horizon per step")
+
+
+def oracle_sample(workload: str, inp):
+    """Bounded sample of the workload for the CPU oracle: about 10-20 s of work for the host cores (the oracle scans
+    every GPU at every event).  Returns (replications, iterations of horizon each)."""
+    cores = os.cpu_count() or 1
+    h_s = 50_000 if workload == "cfg1" else max(100, int(1.0e6 / inp.N))
+    return 2 * cores, h_s, cores
+
+
 def oracle_throughput(inp, horizon_iters: int, n_reps: int, n_threads: int):
-    """The CPU oracle as it stands, one replication per thread (the C code runs without the GIL)."""
+    """The CPU oracle as it stands, one replication per thread (the C code runs without the interpreter lock).  Handles
+    are created before the clock starts; the clock covers the simulation only."""
     from oracle import OracleSim, build_oracle
     build_oracle()
+    sims = [OracleSim(inp.with_(R=1, rep_offset=inp.rep_offset + r)) for r in range(n_reps)]
     iters = [0] * n_reps
     nxt = [0]
     lock = threading.Lock()
@@ -119,11 +168,7 @@ def oracle_throughput(inp, horizon_iters: int, n_reps: int, n_threads: int):
                 nxt[0] += 1
             if r >= n_reps:
                 return
-            sim = OracleSim(inp.with_(R=1, rep_offset=inp.rep_offset + r))
-            sim.run(horizon_iters)
-            st = sim.stats()
-            iters[r] = int(st["iters_mixed"].sum() + st["iters_solo"].sum())
-            sim.close()
+            sims[r].run(horizon_iters)
 
     t0 = time.perf_counter()
     threads = [threading.Thread(target=work) for _ in range(min(n_threads, n_reps))]
@@ -132,30 +177,32 @@ def oracle_throughput(inp, horizon_iters: int, n_reps: int, n_threads: int):
     for t in threads:
         t.join()
     dt = time.perf_counter() - t0
+    for r, sim in enumerate(sims):
+        st = sim.stats()
+        iters[r] = int(st["iters_mixed"].sum() + st["iters_solo"].sum())
+        sim.close()
     return sum(iters) / dt, sum(iters), dt
 
 
-def run_reference(args, workload):
-    from qsim_inputs import presets
+def run_reference(args):
+    """The reference arm: the oracle on the host cores, on the same bounded sample as the `cpu_baseline` leg."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    cores = os.cpu_count() or 1
-    inp = presets.cfg1(R=R_PER_GPU)
-    # bounded sample of the workload per step: one replication per core, 2000 iterations of horizon each
-    h_sample, n_reps = 2000, cores
+    inp = make_inputs(args.workload, 1, args.horizon, args.cluster)
+    n_reps, h_s, cores = oracle_sample(args.workload, inp)
     vals, ms = [], []
     for s in range(args.warmup + args.steps):
-        v, iters, dt = oracle_throughput(inp.with_(rep_offset=s * n_reps), h_sample, n_reps, cores)
+        v, iters, dt = oracle_throughput(inp.with_(rep_offset=s * n_reps), h_s, n_reps, cores)
         if s >= args.warmup:
             vals.append(v); ms.append(dt * 1e3)
     value = sum(vals) / len(vals)
-    sample = f"{n_reps} replications x {h_sample} iterations of horizon of {workload} per step, one per thread"
+    sample = f"{n_reps} replications x {h_s} iterations of horizon of {args.workload} per step, one per thread"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sum(ms) / len(ms), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload, "sample": sample},
+        "config": {"workload": describe(args.workload, inp, args.reps, args.horizon), "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -169,7 +216,7 @@ def run_ctmc(args):
     import torch
     import torch.distributed as dist
     from paper_2602_02987_b200 import QSimCTMC
-    from paper_2602_02987_b200.sharding import shard
+    from paper_2602_02987_b200.sharding import combine_totals, shard
     from qsim_inputs import presets
     from qsim_inputs.spec import ROUTER_SLI
     world = int(os.environ.get("WORLD_SIZE", "1")); rank = int(os.environ.get("RANK", "0")); local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -186,30 +233,38 @@ def run_ctmc(args):
     for _ in range(max(args.warmup, 3)):
         T += dT; sim.run_until(T)
     ev0 = int(sim.stats()["events"].sum()); l0 = sim.launches
+    sampler = ClockSampler(local)
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
+    if rank == 0:
+        sampler.start()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
     for _ in range(args.steps):
         T += dT; sim.run_until(T)
     b.record()
-    torch.cuda.synchronize()
-    my = torch.tensor([a.elapsed_time(b), float(int(sim.stats()["events"].sum()) - ev0), float(sim.launches - l0)], dtype=torch.float64, device="cuda")
-    tmax = my[:1].clone()
     if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX); dist.all_reduce(my[1:], op=dist.ReduceOp.SUM)
+        dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    tot = combine_totals({"jumps": int(sim.stats()["events"].sum()) - ev0, "launches": int(sim.launches - l0)}, a.elapsed_time(b))
     if rank == 0:
-        out = {"metric": "simulated jumps of the exponential-service model/sec", "value": float(my[1]) / (float(tmax[0]) * 1e-3),
+        t_ms, jumps = tot["max_ms"], tot["jumps"]
+        rate = jumps / (t_ms * 1e-3)
+        prof = profile_counters("qsim_ctmc_kernel")
+        issue_peak = N_SM * SCHEDULERS * (clocks["sm_mhz"] or 1965.0) * 1e6
+        inst = prof["warp_inst_per_unit"] * rate / world if prof else None
+        out = {"metric": "simulated jumps of the exponential-service model/sec", "value": rate,
                "unit": "jumps/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-               "ms_per_step": float(tmax[0]) / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-               "dtype": "f64", "data": "synthetic", "gpu_launches": int(my[2]),
+               "ms_per_step": t_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+               "dtype": "f64", "data": "synthetic", "gpu_launches": tot["launches"], "clocks": clocks,
                # no memory or tensor roofline applies: the records are read and written once per launch; the kernel is
                # bound by instruction issue of dependent chains, so the fraction is taken against the issue peak
-               "roofline": {"bound": "alu", "achieved": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3),
-                            "peak": ISSUE_PEAK, "unit": "warp-inst/s",
-                            "frac": NCU_CTMC_WARP_INST_PER_JUMP * float(my[1]) / world / (float(tmax[0]) * 1e-3) / ISSUE_PEAK,
-                            "traffic": NCU_CTMC_DRAM_BYTES_PER_LAUNCH if (count == 37888 and world == 1 and dT == 1.0) else None},
+               "roofline": {"bound": "alu", "achieved": inst, "peak": issue_peak, "unit": "warp-inst/s",
+                            "frac": inst / issue_peak if inst else None,
+                            "traffic": prof["dram_bytes_per_launch"] if (prof and count == 37888 and world == 1 and dT == prof.get("seconds_per_launch")) else None,
+                            "counters": "profiles/counters.json" if prof else "no capture for the current kernel sources"},
                "config": {"workload": f"exponential-service model, paper synthetic instance, n={n}, SLI-aware router, "
                                       f"{R} replications per GPU, {dT} s of simulated time per step"}}
         if not args.no_cpu_baseline and world == 1:
@@ -242,30 +297,27 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="qsim", choices=["qsim", "reference"])
-    ap.add_argument("--horizon", type=int, default=HORIZON, help="iterations of horizon per step")
-    ap.add_argument("--reps", type=int, default=R_PER_GPU, help="replications per GPU")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg1", "ctmc", "cfg0", "cfg3", "cfg4"],
+                    help="cfg2 (default): the largest configuration resident whole on one GPU; cfg1 / cfg0 / cfg3 / cfg4: the "
+                         "other configurations (--cluster gives the simulated GPUs of cfg2-4); ctmc: the exponential-service "
+                         "model, reported in jumps/s")
+    ap.add_argument("--horizon", type=int, default=0, help="iterations of horizon per step (0 = the workload's default)")
+    ap.add_argument("--reps", type=int, default=0, help="replications per GPU (0 = the workload's default)")
+    ap.add_argument("--cluster", type=int, default=0, help="simulated GPUs per replication for cfg2 / cfg3 / cfg4 (0 = the preset's)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="cfg1", choices=["cfg1", "ctmc", "cfg0", "cfg2", "cfg3", "cfg4"],
-                    help="cfg1: the iteration-level benchmark (default); ctmc: the exponential-service model, reported in "
-                         "jumps/s; cfg0 / cfg2 / cfg3 / cfg4: the other configurations (give --reps and --horizon, and "
-                         "--cluster for the GPUs of cfg2-4), without the end-to-end leg")
-    ap.add_argument("--cluster", type=int, default=0, help="simulated GPUs per replication for cfg2 / cfg3 / cfg4 (0 = the preset's)")
     ap.add_argument("--ctmc-seconds", type=float, default=10.0, help="simulated seconds per step of the ctmc workload")
     args = ap.parse_args()
     if args.workload == "ctmc":
+        if args.impl == "reference":
+            raise SystemExit("the reference arm times the iteration-level workloads")
         run_ctmc(args)
         return
-    workload = (f"cfg1: 2 lognormal classes, N=64 GPUs, B=128, C=256, separate pricing, priority gate, solo-first "
-                f"router, least-loaded placement, R={args.reps} replications per GPU, {args.horizon} iterations "
-                f"of horizon per step")
-    other = args.workload != "cfg1"
-    if other:
-        args.no_e2e = True
-        workload = (f"{args.workload}" + (f" with N={args.cluster} GPUs" if args.cluster else "") +
-                    f", R={args.reps} replications per GPU, {args.horizon} iterations of horizon per step")
+    d_reps, d_h = DEFAULTS[args.workload]
+    args.reps = args.reps or d_reps
+    args.horizon = args.horizon or d_h
     if args.impl == "reference":
-        run_reference(args, workload)
+        run_reference(args)
         return
     if args.warmup < 3:
         args.warmup = 3
@@ -273,7 +325,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2602_02987_b200 import QSim, simulate_host
-    from qsim_inputs import presets
+    from paper_2602_02987_b200.sharding import combine_totals, shard
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -290,23 +342,16 @@ def main():
         torch.cuda.synchronize()
 
     # replications are independent: rank k simulates global replications [k R, (k+1) R)  (weak scaling)
-    from paper_2602_02987_b200.sharding import shard
     count, offset = shard(args.reps * world, world, rank)
-    if args.workload == "cfg1":
-        inp = presets.cfg1(R=count)
-    elif args.workload == "cfg0":
-        inp = presets.cfg0(R=count, horizon_iters=args.horizon)
-    elif args.workload == "cfg3":
-        inp = presets.cfg3(R=count, block_len=1.0, **({"N": args.cluster} if args.cluster else {}))
-    else:
-        inp = getattr(presets, args.workload)(R=count, horizon_iters=args.horizon, **({"N": args.cluster} if args.cluster else {}))
-    inp = inp.with_(rep_offset=offset)
+    inp = make_inputs(args.workload, count, args.horizon, args.cluster).with_(rep_offset=offset)
     sim = QSim(inp, device=f"cuda:{local}")
     info = sim.layout_info()
+    family = "one thread per replication" if info["warps"] == 0 else f"{info['warps']} warp(s) per replication"
+    if args.workload not in ("cfg1", "cfg3"):
+        sim.run(PREWARM)          # steady state before the warm-up steps (cfg1's steps are 10^5 iterations each; cfg3 is one day)
     for _ in range(args.warmup):
         sim.run(args.horizon)
-    it0, ev0, tot0 = sim.totals()
-    jobs0 = sum(int(tot0.cls[i].done_mixed + tot0.cls[i].done_solo) for i in range(inp.I))
+    sim.reset_stats()             # the statistics below cover the timed region only
     launches0 = sim.launch_count()
     sampler = ClockSampler(local)
     barrier()
@@ -322,76 +367,79 @@ def main():
     wall = time.perf_counter() - t_wall0
     clocks = sampler.stop() if rank == 0 else None
     step_ms = [a.elapsed_time(b) for a, b in evs]
-    it1, ev1, tot1 = sim.totals()
-    jobs1 = sum(int(tot1.cls[i].done_mixed + tot1.cls[i].done_solo) for i in range(inp.I))
     launches = sim.launch_count() - launches0
-    overflow = sum(int(tot1.cls[i].overflow + tot1.cls[i].overflow_d) for i in range(inp.I))
-    my = torch.tensor([sum(step_ms), float(it1 - it0), float(ev1 - ev0), float(jobs1 - jobs0), float(launches),
-                       float(overflow)], dtype=torch.float64, device="cuda")
-    tmax = my[:1].clone()
-    if world > 1:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(my[1:], op=dist.ReduceOp.SUM)
-    total_ms = float(tmax[0])
-    iters, events, jobs, n_launch, ovf = (float(x) for x in my[1:])
+    it1, ev1, tot1 = sim.totals()                 # reduced on the device: a few KB come back
+    bundled, separate = sim.revenue(tot1)
+    I = inp.I
+    mine = {"iters": it1, "events": ev1, "launches": launches,
+            "jobs": sum(int(tot1.cls[i].done_mixed + tot1.cls[i].done_solo) for i in range(I)),
+            "overflow": sum(int(tot1.cls[i].overflow + tot1.cls[i].overflow_d) for i in range(I)),
+            "abandoned": sum(int(tot1.cls[i].abandoned_p + tot1.cls[i].abandoned_d) for i in range(I)),
+            "revenue_x_T": (separate if inp.pricing == 1 else bundled) * float(tot1.T_elapsed), "T": float(tot1.T_elapsed)}
+    tot = combine_totals(mine, sum(step_ms))
+    total_ms = tot["max_ms"]
+    iters, events, jobs, n_launch = tot["iters"], tot["events"], tot["jobs"], tot["launches"]
     value = iters / (total_ms * 1e-3)
 
-    # end to end through the host-buffer entry point (fresh system each step)
+    # end to end through the host-buffer entry point (fresh system each step, totals reduced on the device)
     e2e = None
     if not args.no_e2e:
-        e_iters, e_t = 0.0, 0.0
-        h2d = int(inp.lengths.nbytes + inp.rates.nbytes + 8 * 6 + 8 * 2 + inp.nblk * 264 + inp.I * 24 + 80)
-        d2h = 0
-        simulate_host(inp.with_(R=8), 200)   # warm the context and allocator paths
+        h2d = int((inp.lengths.nbytes if inp.lengths is not None else 0) + inp.rates.nbytes + 8 * 6 + 8 * 2 + inp.nblk * 456 + inp.I * 24 + 80)
+        d2h = 2048 + 8
+        simulate_host(inp.with_(R=8), 50, per_rep=False)   # warm the context and allocator paths
         barrier()
+        e_t, e_iters = 0.0, 0
         for _ in range(args.steps):
             t0 = time.perf_counter()
-            st = simulate_host(inp, args.horizon)
+            st = simulate_host(inp, args.horizon, per_rep=False)["_totals"]
             e_t += time.perf_counter() - t0
-            e_iters += float(st["iters_mixed"].sum() + st["iters_solo"].sum())
-            d2h = inp.R * info["header_bytes"]
-        ev = torch.tensor([e_t, e_iters], dtype=torch.float64, device="cuda")
-        tm = ev[:1].clone()
-        if world > 1:
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            dist.all_reduce(ev[1:], op=dist.ReduceOp.SUM)
-        e2e = {"value": float(ev[1]) / float(tm[0]), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h}
+            e_iters += int(st["iters_mixed"].sum() + st["iters_solo"].sum())
+        et = combine_totals({"iters": e_iters}, e_t * 1e3)
+        e2e = {"value": et["iters"] / (et["max_ms"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "note": "fresh system each step (transient from empty, no warm-up): allocation, table upload, set-up, run, totals"}
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
-        # algorithmic HBM bytes of one launch of the dominant kernel (qsim_run_kernel): the server state is
-        # resident in shared memory, so what must move is the request life cycle plus the state staging
+        # algorithmic HBM bytes of one launch of the dominant kernel (the run kernel): what the method must move is the
+        # request life cycle; the warp-per-replication kernels also stage their per-GPU state once per launch
         stage = 2.0 * inp.R * (info["header_bytes"] + info["image_bytes"])
-        alg_bytes_per_launch = (JOB_BYTES * jobs / world + stage * args.steps) / max(n_launch / world, 1.0)
-        kernel_ms = total_ms / max(n_launch / world, 1.0)
+        n_l = max(n_launch / world, 1.0)
+        alg_bytes_per_launch = (JOB_BYTES * jobs / world + stage * args.steps) / n_l
+        kernel_ms = total_ms / n_l
         achieved = alg_bytes_per_launch / (kernel_ms * 1e-3) / 1e9
+        key = f"{args.workload}:{'lane' if info['warps'] == 0 else 'warp'}" + (f":N{inp.N}" if args.cluster else "")
+        prof = profile_counters(key)
+        issue_peak = N_SM * SCHEDULERS * (clocks["sm_mhz"] or 1965.0) * 1e6
+        lp_value = float(inp.meta["lp_value"][0]) if inp.nblk == 1 else None
+        rev = tot["revenue_x_T"] / tot["T"] if tot["T"] > 0 else None
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload, "l2": "state larger than L2 (workspace %.0f MB per GPU)" % (sim.workspace_bytes / 1e6),
+            "config": {"workload": describe(args.workload, inp, args.reps, args.horizon), "kernels": family,
+                       "l2": "state larger than L2 (workspace %.0f MB per GPU)" % (sim.workspace_bytes / 1e6),
+                       "prewarm_iterations": PREWARM if args.workload not in ("cfg1", "cfg3") else 0,
                        "events_per_iteration": events / iters, "requests_per_iteration": jobs / iters,
-                       "queue_overflow": ovf},
+                       "queue_overflow": tot["overflow"], "abandoned": tot["abandoned"],
+                       "revenue_per_gpu": rev, "lp_value": lp_value,
+                       "revenue_over_lp": (rev / lp_value) if (rev is not None and lp_value) else None},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": None if other else NCU_DRAM_BYTES_PER_ITER * iters / world / max(n_launch / world, 1.0),
-                         "traffic_source": "no capture for this workload" if other else "ncu capture of a 2000-iteration launch, scaled by iterations",
-                         "peak_kind": peak_kind,
-                         "bytes_per_iteration": JOB_BYTES * jobs / iters,
-                         "note": "latency/issue-bound event chain; HBM fraction is the contract figure",
-                         "issue": None if other else {"achieved": NCU_WARP_INST_PER_ITER * value / world, "peak": ISSUE_PEAK,
-                                                      "unit": "warp-inst/s", "frac": NCU_WARP_INST_PER_ITER * value / world / ISSUE_PEAK}},
+                         "traffic": prof["dram_bytes_per_unit"] * iters / world / n_l if prof else None,
+                         "traffic_source": (f"ncu capture scaled by iterations ({prof['capture']})" if prof else
+                                            "no capture for this workload with the current kernel sources"),
+                         "peak_kind": peak_kind, "bytes_per_iteration": JOB_BYTES * jobs / iters,
+                         "note": "latency/issue-bound event chains; the HBM fraction is the contract figure",
+                         "issue": ({"achieved": prof["warp_inst_per_unit"] * value / world, "peak": issue_peak, "unit": "warp-inst/s",
+                                    "frac": prof["warp_inst_per_unit"] * value / world / issue_peak} if prof else None)},
             "clocks": clocks, "gpu_launches": int(n_launch), "wall_s": wall,
         }
         if e2e:
             out["e2e"] = e2e
         if not args.no_cpu_baseline and world == 1:
-            cores = os.cpu_count() or 1
-            # about 10 s of work for the host cores: the oracle scans every GPU at every event
-            h_s = 50_000 if not other else max(100, int(1.0e6 / inp.N))
-            v, it_s, dt = oracle_throughput(inp, h_s, 2 * cores, cores)
+            n_reps, h_s, cores = oracle_sample(args.workload, inp)
+            v, it_s, dt = oracle_throughput(inp, h_s, n_reps, cores)
             out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                   "sample": f"{2 * cores} replications x {h_s} iterations of horizon of {args.workload}, one per thread, {dt:.1f} s"}
+                                   "sample": f"{n_reps} replications x {h_s} iterations of horizon of {args.workload}, one per thread, {dt:.1f} s"}
         print(json.dumps(out))
     sim.close()
     if world > 1:

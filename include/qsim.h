@@ -151,7 +151,8 @@ int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
  * qsim_bind.  Nothing is initialised; the next qsim_run continues where the checkpointed run stopped, with bit-identical
  * results [the time horizon of Eq. (21)-(23) composes: run(a); run(b) is run(a+b)].  Targets installed with
  * qsim_set_targets are part of the handle, not of the workspace: install them again.  QSIM_ESTATE if the bytes hold
- * no resumable state (a replication stopped on an internal error).
+ * no resumable state (some replication stopped on an internal error) or were saved by a handle of another configuration or
+ * layout (a fingerprint of both is kept in the workspace).
  */
 int qsim_bind_restore(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
 
@@ -230,6 +231,21 @@ int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const doubl
                   const uint32_t *lengths, const double *prices, const double *iter_time_coeffs,
                   const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
                   qsim_rep_stats *per_rep);
+
+/*
+ * qsim_simulate for more replications than the device can hold at once [the convergence experiments of the EC run the
+ * same instance for growing n; at n = 4096 GPUs with B = 256 one replication is tens of MB of state].  The R
+ * replications are simulated `wave` at a time (0 = the largest wave that fits in nine tenths of the free device
+ * memory), each wave from the empty system over horizon_iters, in one workspace that the call allocates once and
+ * frees; random streams are keyed by the global replication index, so the result does not depend on `wave`: integer
+ * statistics are identical and the totals are added in replication order.  [host] per_rep[R] and totals may be NULL;
+ * waves_run (may be NULL) receives the number of waves.  Only whole runs can be split into waves: a handle that is
+ * resumed by further qsim_run calls keeps all its replications resident.
+ */
+int qsim_simulate_waves(const qsim_config *cfg, const qsim_class *classes, const double *rates,
+                        const uint32_t *lengths, const double *prices, const double *iter_time_coeffs,
+                        const qsim_targets *lp_targets, uint64_t horizon_iters, uint32_t wave,
+                        qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint32_t *waves_run);
 
 /*
  * The same simulation as qsim_simulate for callers that must not allocate.  (The paper has no
@@ -327,6 +343,13 @@ int qsim_ctmc_run_until(const qsim_ctmc_config *cfg, const qsim_ctmc_class *clas
  * Synchronises the stream.  QSIM_EOVERFLOW if a replication stopped on an internal error. */
 int qsim_ctmc_stats(const qsim_ctmc_config *cfg, const void *dev_workspace, size_t bytes, void *cuda_stream,
                     qsim_ctmc_rep_stats *per_rep);
+
+/* Revenue per GPU per second of every replication of the exponential-service model from its counters [Eq. (21)-(23)]:
+ * bundled charging credits c_p P_i + c_d D_i when a request finishes decoding; separate charging (separate != 0) credits
+ * c_p P_i when its prefill finishes and c_d D_i when its decode finishes.  [host] per_rep[R] as filled by qsim_ctmc_stats,
+ * P[I], D[I] mean prompt / output tokens, prices {c_p, c_d}; rate[R] receives revenue / (N T_elapsed). */
+int qsim_ctmc_revenue(const qsim_ctmc_config *cfg, const qsim_ctmc_rep_stats *per_rep, const double *P, const double *D,
+                      const double *prices, int separate, double *rate);
 
 int qsim_destroy(qsim_t *h);
 

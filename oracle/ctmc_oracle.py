@@ -124,3 +124,14 @@ def run_ctmc_oracle(inp, T_end: float, rep_lo: int = 0, rep_hi: int | None = Non
     st = sim.stats()
     sim.close()
     return st
+
+
+def ctmc_revenue_rate(inp, st: dict, separate=None) -> np.ndarray:
+    """Per-GPU revenue rate of every replication from the oracle's integer counters: bundled charging credits
+    c_p P_i + c_d D_i at decode completion (Eq. (21)-(22)); separate charging credits c_p P_i at prefill
+    completion and c_d D_i at decode completion (Eq. (23))."""
+    sep = inp.meta.get("separate", False) if separate is None else separate
+    done = (st["done_mixed"] + st["done_solo"]).astype(float)
+    pf = st["prefill_done"].astype(float) if sep else done
+    rev = (inp.prices[0] * inp.P * pf + inp.prices[1] * inp.D * done).sum(axis=1)
+    return rev / (inp.N * st["T_elapsed"])

@@ -5,5 +5,5 @@ marshals arguments; every simulation step runs in the CUDA kernels.  PyTorch sup
 (the workspace tensor) and the stream.  There is no CPU fallback: without the built library or without
 a CUDA device the calls raise.
 """
-from .binding import QSim, QSimCTMC, QSimError, load_library, simulate_host, simulate_static  # noqa: F401
+from .binding import QSim, QSimCTMC, QSimError, load_library, simulate_host, simulate_static, simulate_waves  # noqa: F401
 from .build import build_library  # noqa: F401

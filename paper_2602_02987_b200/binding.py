@@ -18,9 +18,9 @@ _SUMS = ("area_Qp", "area_X", "area_Qd", "area_Ym", "area_Ys", "sum_ttft", "sum_
 
 EXPORTS = ("qsim_create", "qsim_workspace_bytes", "qsim_bind", "qsim_run", "qsim_run_until", "qsim_set_injected",
            "qsim_set_targets", "qsim_set_event_budget", "qsim_sync",
-           "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate",
+           "qsim_stats", "qsim_reset_stats", "qsim_revenue", "qsim_server_state", "qsim_simulate", "qsim_simulate_waves",
            "qsim_simulate_static", "qsim_launch_count", "qsim_round_count", "qsim_layout_info", "qsim_destroy", "qsim_last_error",
-           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats", "qsim_bind_restore", "qsim_latency_percentiles")
+           "qsim_ctmc_workspace_bytes", "qsim_ctmc_init", "qsim_ctmc_run_until", "qsim_ctmc_stats", "qsim_ctmc_revenue", "qsim_bind_restore", "qsim_latency_percentiles")
 
 
 class QSimError(RuntimeError):
@@ -106,10 +106,13 @@ def load_library():
         L.qsim_ctmc_run_until.argtypes = [C.POINTER(qsim_ctmc_config), C.POINTER(qsim_ctmc_class), vp, C.c_size_t, vp,
                                           C.c_double, C.POINTER(C.c_uint64)]
         L.qsim_ctmc_stats.argtypes = [C.POINTER(qsim_ctmc_config), vp, C.c_size_t, vp, vp]
+        L.qsim_ctmc_revenue.argtypes = [C.POINTER(qsim_ctmc_config), vp, vp, vp, vp, C.c_int, vp]
         L.qsim_revenue.argtypes = [vp, vp, C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.qsim_server_state.argtypes = [vp, C.c_uint32, vp, vp, vp, vp]
         L.qsim_simulate.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
                                     C.POINTER(qsim_targets), C.c_uint64, vp, vp]
+        L.qsim_simulate_waves.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
+                                          C.POINTER(qsim_targets), C.c_uint64, C.c_uint32, vp, vp, C.POINTER(C.c_uint32)]
         L.qsim_simulate_static.argtypes = [C.POINTER(qsim_config), C.POINTER(qsim_class), vp, vp, vp, vp,
                                            C.POINTER(qsim_targets), C.c_uint64, vp, vp, vp]
         L.qsim_launch_count.argtypes = [vp, C.POINTER(C.c_uint64)]
@@ -294,6 +297,12 @@ class QSim:
         _check(self.L.qsim_stats(self.h, C.byref(tot), None, None, None))
         return int(tot.iters_mixed + tot.iters_solo), int(tot.events), tot
 
+    def revenue(self, tot):
+        """(bundled, separate) revenue per GPU per second of a totals record, Eq. (22)-(23)."""
+        b, s = C.c_double(), C.c_double()
+        _check(self.L.qsim_revenue(self.h, C.byref(tot), C.byref(b), C.byref(s)))
+        return b.value, s.value
+
     def server_state(self, r: int) -> dict:
         N = self.inp.N
         n_dec = np.zeros(N, np.uint32); it = np.zeros(N, np.uint32)
@@ -314,16 +323,32 @@ class QSim:
             pass
 
 
-def simulate_host(inp, horizon_iters: int) -> dict:
-    """qsim_simulate: host buffers in, host statistics out (allocates and frees its own device memory)."""
+def simulate_host(inp, horizon_iters: int, per_rep: bool = True) -> dict:
+    """qsim_simulate: host buffers in, host statistics out (allocates and frees its own device memory).
+    per_rep=False asks for the totals only: they are reduced on the device and a few KB come back."""
+    L = load_library()
+    cfg, classes, rates, lengths, prices, coeffs, tg = marshal(inp)
+    per = (qsim_rep_stats * inp.R)() if per_rep else None
+    tot = qsim_rep_stats()
+    _check(L.qsim_simulate(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
+                           int(horizon_iters), C.byref(tot), per))
+    out = _unpack(per, inp.R, inp.I) if per_rep else {}
+    out["_totals"] = _unpack((tot,), 1, inp.I)
+    return out
+
+
+def simulate_waves(inp, horizon_iters: int, wave: int = 0) -> dict:
+    """qsim_simulate_waves: all R replications of a whole run, `wave` of them resident at a time (0 = as many as fit)."""
     L = load_library()
     cfg, classes, rates, lengths, prices, coeffs, tg = marshal(inp)
     per = (qsim_rep_stats * inp.R)()
     tot = qsim_rep_stats()
-    _check(L.qsim_simulate(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
-                           int(horizon_iters), C.byref(tot), per))
+    n = C.c_uint32()
+    _check(L.qsim_simulate_waves(C.byref(cfg), classes, _ptr(rates), _ptr(lengths), _ptr(prices), _ptr(coeffs), tg,
+                                 int(horizon_iters), int(wave), C.byref(tot), per, C.byref(n)))
     out = _unpack(per, inp.R, inp.I)
     out["_totals"] = _unpack((tot,), 1, inp.I)
+    out["_waves"] = int(n.value)
     return out
 
 
@@ -404,6 +429,14 @@ class QSimCTMC:
             out[n] = np.ascontiguousarray(area[:, :I, k])
         out["events"] = tail[:, :8].copy().view(np.uint64).reshape(R)
         out["T_elapsed"] = tail[:, 8:16].copy().view(np.float64).reshape(R)
+        # per-GPU revenue rate of every replication under the instance's charging scheme (qsim_ctmc_revenue)
+        rate = np.zeros(R, np.float64)
+        P = np.ascontiguousarray(self.inp.P, np.float64); D = np.ascontiguousarray(self.inp.D, np.float64)
+        prices = np.ascontiguousarray(self.inp.prices, np.float64)
+        if (out["T_elapsed"] > 0).all():
+            _check(self.L.qsim_ctmc_revenue(C.byref(self.cfg), per, _ptr(P), _ptr(D), _ptr(prices),
+                                            1 if self.inp.meta.get("separate", False) else 0, _ptr(rate)))
+        out["_revenue_rate"] = rate
         return out
 
     def close(self) -> None:

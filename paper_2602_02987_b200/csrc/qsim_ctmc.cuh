@@ -506,17 +506,17 @@ int qsim_ctmc_run_until(const qsim_ctmc_config *cfg, const qsim_ctmc_class *clas
     rc = ctmc_launch_shape(cfg->I, threads, smem);
     if (rc != QSIM_OK) return rc;
     // a replication that used up its per-launch event budget is continued by further launches
-    for (int guard = 0; guard < 100000; ++guard) {
-        uint32_t flag = 0;
+    uint32_t flag = 1;
+    for (int guard = 0; guard < 100000 && flag != 0; ++guard) {
         CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, st));
         qsim_ctmc_kernel<<<(cfg->R + threads - 1u) / threads, threads, smem, st>>>(p);
         CUDA_TRY(cudaGetLastError());
         ++n;
         CUDA_TRY(cudaMemcpyAsync(&flag, p.not_done, 4, cudaMemcpyDeviceToHost, st));
         CUDA_TRY(cudaStreamSynchronize(st));
-        if (flag == 0) break;
     }
     if (launches) *launches = n;
+    if (flag != 0) return fail(QSIM_EOVERFLOW, "replications still unfinished after 100000 launches: the end time was not reached");
     return QSIM_OK;
 }
 
@@ -546,6 +546,25 @@ int qsim_ctmc_stats(const qsim_ctmc_config *cfg, const void *dev_workspace, size
         }
         o.events = S.events;
         o.T_elapsed = T;
+    }
+    return QSIM_OK;
+}
+
+int qsim_ctmc_revenue(const qsim_ctmc_config *cfg, const qsim_ctmc_rep_stats *per_rep, const double *P, const double *D,
+                      const double *prices, int separate, double *rate)
+{
+    if (!cfg || !per_rep || !P || !D || !prices || !rate) return fail(QSIM_EINVAL, "null argument");
+    if (cfg->size != sizeof(qsim_ctmc_config) || cfg->I < 1 || cfg->I > QSIM_MAXI || cfg->N < 1) return fail(QSIM_EINVAL, "bad qsim_ctmc_config");
+    for (uint32_t r = 0; r < cfg->R; ++r) {
+        const qsim_ctmc_rep_stats &s = per_rep[r];
+        if (!(s.T_elapsed > 0.0)) return fail(QSIM_ESTATE, "no simulated time has elapsed");
+        double rev = 0.0;
+        for (uint32_t i = 0; i < cfg->I; ++i) {
+            const double done = (double)(s.cnt[i][CC_DONE_MIXED] + s.cnt[i][CC_DONE_SOLO]);
+            const double paid_in = separate ? (double)s.cnt[i][CC_PREFILL_DONE] : done;       // separate charging credits the prompt at prefill completion
+            rev += prices[0] * P[i] * paid_in + prices[1] * D[i] * done;
+        }
+        rate[r] = rev / ((double)cfg->N * s.T_elapsed);
     }
     return QSIM_OK;
 }

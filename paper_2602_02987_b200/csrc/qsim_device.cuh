@@ -68,7 +68,7 @@ struct Area { double area, t_last; };
 struct ClassState {
     double ta;
     unsigned long long adraw, sli_ord;
-    uint32_t ablk, nextP, nextD, pq_head, pq_n, X, Ym, Ys, Qd0, Qd1;
+    uint32_t ablk, nextP, nextD, pq_head, pq_n, X, Ym, Ys, Qd0, Qd1, pq_tail, pq_pad;   // pq_tail: one-thread-per-replication kernels
     AbClock abp, abd0, abd1;
     Area aQp, aX, aQd;
     double sYm_in, sYm_out, sYs_in, sYs_out;   // sums of (placement / completion time - T_reset): integral of Y = out - in + Y (T - T_reset)
@@ -110,6 +110,7 @@ struct LanePar {
     uint32_t tlev, toff[6], tsize;   // eligibility trees: internal levels, offset of every level (0 = leaves) and entries per tree
     uint32_t b8, slev, soff[5], ssize;   // slot trees: leaves per GPU, internal levels, offsets of levels 1.. and nodes per GPU
     double inv_w;                // buckets per second
+    uint32_t cs_stride, smem_bytes;  // shared memory per lane for the class records (32-bit words) and per block of 32 lanes (bytes)
     LaneSrv *srv;                // [N] GPU records
     double *tarr;                // [N] arrival time of the request in prefill
     uint16_t *cal_head;          // [nbk] first GPU of every bucket
@@ -119,6 +120,8 @@ struct LanePar {
     unsigned long long *snode;   // [N][ssize] minimum of finish << 16 | slot per group of eight
     SlotRec *srec;               // [N][B] request in each slot
     uint16_t *sfree;             // [N][B] entries at and above the GPU's decode count are its free slots
+    uint32_t *pql;               // [I][qw] live bits of the prefill-queue positions
+    uint32_t qw, qw_pad;         // words per class in pql (a multiple of four)
 };
 
 struct Params {

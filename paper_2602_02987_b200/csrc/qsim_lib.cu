@@ -35,10 +35,12 @@ int fail(int code, const std::string &msg)
 
 size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
+struct TotalsRecBytes { char b[2048]; };      // room for the device totals record (checked where the record is defined)
+
 struct Sections {
-    size_t hdr, srv, fin, rec, pq, dq, hist, flag, total;
+    size_t hdr, srv, fin, rec, pq, dq, hist, flag, red, total;
     // one-thread-per-replication family
-    size_t l_srv, l_tarr, l_head, l_bm, l_tree, l_sfin, l_snode, l_srec, l_sfree;
+    size_t l_srv, l_tarr, l_head, l_bm, l_tree, l_sfin, l_snode, l_srec, l_sfree, l_pql;
 };
 
 }  // namespace
@@ -84,6 +86,7 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
     s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
     s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
     s.flag = o; o = align256(o + 256);
+    s.red = o; o = align256(o + sizeof(TotalsRecBytes) + R * (size_t)(c.I * 7u + 3u) * 8);    // totals record + fp64 statistics per replication
     s.total = o;
     return s;
 }
@@ -103,10 +106,12 @@ Sections lane_sections(const qsim_config &c, const LanePar &q)
     s.l_snode = o; o = align256(o + R * N * (size_t)q.ssize * 8);
     s.l_srec = o; o = align256(o + R * N * (size_t)c.B * sizeof(SlotRec));
     s.l_sfree = o; o = align256(o + R * N * (size_t)c.B * 2);
+    s.l_pql = o; o = align256(o + R * (size_t)c.I * q.qw * 4);
     s.pq = o; o = align256(o + R * (size_t)c.I * c.qcap * sizeof(QEntry));
     s.dq = o; o = align256(o + R * (size_t)2 * c.qcap * sizeof(QEntry));
     s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
     s.flag = o; o = align256(o + 256);
+    s.red = o; o = align256(o + sizeof(TotalsRecBytes) + R * (size_t)(c.I * 7u + 3u) * 8);    // totals record + fp64 statistics per replication
     s.total = o;
     return s;
 }
@@ -155,6 +160,13 @@ void lane_shapes(const qsim_config &c, const double *coef, LanePar &q)
     tree_shape(c.B, q.slev, off, size);
     for (uint32_t l = 0; l < q.slev; ++l) q.soff[l] = off[l + 1] - off[1];      // internal levels only: the leaves are a separate array
     q.ssize = size - off[1];
+    q.qw = ((c.qcap + 127u) / 128u) * 4u;
+    // shared memory of a block of 32 lanes: per lane the class records, at a stride whose half is odd (the lanes' 8-byte
+    // accesses then fall into different banks), and one bit per calendar bucket
+    uint32_t stride = c.I * (uint32_t)(sizeof(ClassState) / 4);
+    if (((stride / 2u) & 1u) == 0) stride += 2u;
+    q.cs_stride = stride;
+    q.smem_bytes = 32u * (stride * 4u + q.nbk / 8u);
 }
 
 int validate(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
@@ -388,6 +400,7 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     }
     if (lane) {
         lane_shapes(cfg, coef, p.lane);
+        if (p.lane.smem_bytes > 227u * 1024u) return fail(QSIM_EINVAL, "class records and calendar do not fit shared memory");
         h.sec = lane_sections(cfg, p.lane);
         h.nwarps = 0;
     }
@@ -427,12 +440,120 @@ int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
     p.force_dispatch = h->targets_changed ? 1u : 0u;
     h->targets_changed = false;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    if (p.lane.on) qsim_lane_run_kernel<<<(h->cfg.R + 31u) / 32u, 32, 0, h->stream>>>(p);
+    if (p.lane.on) qsim_lane_run_kernel<<<(h->cfg.R + 31u) / 32u, 32, p.lane.smem_bytes, h->stream>>>(p);
     else h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
     return QSIM_OK;
+}
+
+}  // namespace
+
+namespace {
+
+// Statistics of one replication from its device record.  The same function runs on the host (qsim_stats with per-replication
+// output) and on the device (totals only): every operation is one rounded IEEE double operation on either side.
+__host__ __device__ inline void rep_stats_of(const RepHeader &H, uint32_t I, qsim_rep_stats &st)
+{
+    const double T = H.T_end;
+    st.T_elapsed = T - H.T_reset;
+    st.iters_mixed = 0; st.iters_solo = 0; st.busy_mixed = 0.0; st.busy_solo = 0.0;
+    for (int l = 0; l < 32; ++l) {
+        st.iters_mixed += H.iters_mixed[l];
+        st.iters_solo += H.iters_solo[l];
+        st.busy_mixed = st.busy_mixed + H.busy_mixed[l];
+        st.busy_solo = st.busy_solo + H.busy_solo[l];
+    }
+    st.events = H.events + st.iters_mixed + st.iters_solo;   // H.events counts block switches; class events are added below
+    for (uint32_t i = 0; i < I; ++i) {
+        const ClassState &c = H.cs[i];
+        qsim_class_stats &o = st.cls[i];
+        o.arrivals = c.arrivals; o.admitted = c.admitted; o.prefill_done = c.prefill_done;
+        o.placed_mixed = c.placed_mixed; o.placed_solo = c.placed_solo; o.done_mixed = c.done_mixed;
+        o.done_solo = c.done_solo; o.abandoned_p = c.abandoned_p; o.abandoned_d = c.abandoned_d;
+        o.overflow = c.overflow; o.overflow_d = c.overflow_d; o.tokens_in_prefilled = c.tok_in_pf;
+        o.tokens_in_completed = c.tok_in_done; o.tokens_out_completed = c.tok_out_done;
+        const uint32_t Qd = c.Qd0 + c.Qd1;
+        o.Qp = c.pq_n; o.X = c.X; o.Qd = Qd; o.Ym = c.Ym; o.Ys = c.Ys; o.reserved = 0;
+        // integrals are reported up to the end of the run without touching the stored state
+        o.area_Qp = c.aQp.area + (double)c.pq_n * (T - c.aQp.t_last);
+        o.area_X = c.aX.area + (double)c.X * (T - c.aX.t_last);
+        o.area_Qd = c.aQd.area + (double)Qd * (T - c.aQd.t_last);
+        o.area_Ym = (c.sYm_out - c.sYm_in) + (double)c.Ym * (T - H.T_reset);
+        o.area_Ys = (c.sYs_out - c.sYs_in) + (double)c.Ys * (T - H.T_reset);
+        o.sum_ttft = c.sum_ttft; o.sum_tpot = c.sum_tpot;
+        st.events += c.arrivals + c.abandoned_p + c.abandoned_d;
+    }
+}
+
+// One more replication into the totals (replications are added in index order, so the fp64 totals are reproducible)
+inline void add_rep_stats(qsim_rep_stats &tot, const qsim_rep_stats &st, uint32_t I)
+{
+    tot.iters_mixed += st.iters_mixed; tot.iters_solo += st.iters_solo; tot.events += st.events;
+    tot.busy_mixed += st.busy_mixed; tot.busy_solo += st.busy_solo; tot.T_elapsed += st.T_elapsed;
+    for (uint32_t i = 0; i < I; ++i) {
+        const qsim_class_stats &a = st.cls[i];
+        qsim_class_stats &b = tot.cls[i];
+        b.arrivals += a.arrivals; b.admitted += a.admitted; b.prefill_done += a.prefill_done;
+        b.placed_mixed += a.placed_mixed; b.placed_solo += a.placed_solo; b.done_mixed += a.done_mixed;
+        b.done_solo += a.done_solo; b.abandoned_p += a.abandoned_p; b.abandoned_d += a.abandoned_d;
+        b.overflow += a.overflow; b.overflow_d += a.overflow_d; b.tokens_in_prefilled += a.tokens_in_prefilled;
+        b.tokens_in_completed += a.tokens_in_completed; b.tokens_out_completed += a.tokens_out_completed;
+        b.Qp += a.Qp; b.X += a.X; b.Qd += a.Qd; b.Ym += a.Ym; b.Ys += a.Ys;
+        b.area_Qp += a.area_Qp; b.area_X += a.area_X; b.area_Qd += a.area_Qd; b.area_Ym += a.area_Ym;
+        b.area_Ys += a.area_Ys; b.sum_ttft += a.sum_ttft; b.sum_tpot += a.sum_tpot;
+    }
+}
+
+// Totals on the device (a11, statistics reduction).  Integer counters are summed with atomic additions (exact in any
+// order); the floating-point statistics of every replication go to a compact array and one thread per statistic adds
+// them in replication order, which is the order the host uses: the totals are bit-identical to the host's.
+constexpr uint32_t NF_CLASS = 7, NF_REP = 3;      // fp64 statistics per class and per replication
+struct TotalsRec { qsim_rep_stats tot; uint32_t err_rep, err_code; };
+static_assert(sizeof(TotalsRec) <= sizeof(TotalsRecBytes), "room for the totals record in the workspace");
+
+__global__ void qsim_totals_gather_kernel(const RepHeader *hdr, uint32_t R, uint32_t I, double *F, TotalsRec *out)
+{
+    const uint32_t r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= R) return;
+    const RepHeader &H = hdr[r];
+    if (H.err) { if (atomicCAS(&out->err_code, 0u, H.err) == 0u) out->err_rep = r; return; }
+    qsim_rep_stats st;
+    rep_stats_of(H, I, st);
+    const uint32_t nf = I * NF_CLASS + NF_REP;
+    double *f = F + (size_t)r * nf;
+    qsim_rep_stats &t = out->tot;
+    typedef unsigned long long u64;
+    atomicAdd((u64 *)&t.iters_mixed, (u64)st.iters_mixed); atomicAdd((u64 *)&t.iters_solo, (u64)st.iters_solo);
+    atomicAdd((u64 *)&t.events, (u64)st.events);
+    for (uint32_t i = 0; i < I; ++i) {
+        const qsim_class_stats &a = st.cls[i];
+        qsim_class_stats &b = t.cls[i];
+        const uint64_t *src = &a.arrivals;
+        uint64_t *dst = &b.arrivals;
+        for (int k = 0; k < 14; ++k) atomicAdd((u64 *)(dst + k), (u64)src[k]);      // the fourteen 64-bit counters are contiguous
+        atomicAdd(&b.Qp, a.Qp); atomicAdd(&b.X, a.X); atomicAdd(&b.Qd, a.Qd); atomicAdd(&b.Ym, a.Ym); atomicAdd(&b.Ys, a.Ys);
+        double *fc = f + i * NF_CLASS;
+        fc[0] = a.area_Qp; fc[1] = a.area_X; fc[2] = a.area_Qd; fc[3] = a.area_Ym; fc[4] = a.area_Ys; fc[5] = a.sum_ttft; fc[6] = a.sum_tpot;
+    }
+    f[I * NF_CLASS + 0] = st.busy_mixed; f[I * NF_CLASS + 1] = st.busy_solo; f[I * NF_CLASS + 2] = st.T_elapsed;
+}
+
+__global__ void qsim_totals_sum_kernel(uint32_t R, uint32_t I, const double *F, TotalsRec *out)
+{
+    const uint32_t nf = I * NF_CLASS + NF_REP, k = threadIdx.x;
+    if (k >= nf || out->err_code) return;
+    double acc = 0.0;
+    for (uint32_t r = 0; r < R; ++r) acc = acc + F[(size_t)r * nf + k];
+    qsim_rep_stats &t = out->tot;
+    if (k < I * NF_CLASS) {
+        qsim_class_stats &b = t.cls[k / NF_CLASS];
+        double *dst[NF_CLASS] = { &b.area_Qp, &b.area_X, &b.area_Qd, &b.area_Ym, &b.area_Ys, &b.sum_ttft, &b.sum_tpot };
+        *dst[k % NF_CLASS] = acc;
+    } else if (k == I * NF_CLASS) t.busy_mixed = acc;
+    else if (k == I * NF_CLASS + 1) t.busy_solo = acc;
+    else t.T_elapsed = acc;
 }
 
 }  // namespace
@@ -471,6 +592,7 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     if (e == cudaSuccess) e = cudaMallocHost(&h->h_flag, 256);
     if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(h->run_fn));
     if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(qsim_init_kernel));
+    if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(qsim_lane_run_kernel));
     if (e != cudaSuccess) {
         std::string msg = std::string("device set-up failed: ") + cudaGetErrorString(e);
         qsim_destroy(h);
@@ -524,14 +646,35 @@ static int attach_workspace(qsim_t *h, void *ws, size_t bytes, void *cuda_stream
         q.snode = reinterpret_cast<unsigned long long *>(base + h->sec.l_snode);
         q.srec = reinterpret_cast<SlotRec *>(base + h->sec.l_srec);
         q.sfree = reinterpret_cast<uint16_t *>(base + h->sec.l_sfree);
+        q.pql = reinterpret_cast<uint32_t *>(base + h->sec.l_pql);
     }
     return QSIM_OK;
+}
+
+// Fingerprint of everything that fixes the meaning of the workspace bytes: stored in the workspace at bind, checked when a
+// saved workspace is adopted.
+static void workspace_tag(const qsim_t *h, unsigned long long tag[2])
+{
+    const qsim_config &c = h->cfg;
+    const unsigned long long words[] = { c.I, c.N, c.R, c.B, c.C, c.nblk, c.gate, c.router, c.placement, c.length_mode, c.qcap, c.hist,
+                                         c.seed, c.rep_offset, h->par.Npad, h->par.slots_smem, h->par.srv_bytes, h->par.lane.on,
+                                         (unsigned long long)h->sec.total, (unsigned long long)sizeof(RepHeader) };
+    unsigned long long x = 0xcbf29ce484222325ull;       // FNV-1a over the bytes of the words
+    for (unsigned long long w : words)
+        for (int b = 0; b < 8; ++b) { x ^= (w >> (8 * b)) & 0xffull; x *= 0x100000001b3ull; }
+    tag[0] = 0x7173696d2d777331ull;                      // "qsim-ws1"
+    tag[1] = x;
 }
 
 int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
 {
     int rc = attach_workspace(h, ws, bytes, cuda_stream);
     if (rc != QSIM_OK) return rc;
+    {
+        unsigned long long tag[2];
+        workspace_tag(h, tag);
+        CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char *>(h->par.not_done) + 16, tag, sizeof tag, cudaMemcpyHostToDevice, h->stream));
+    }
     if (h->par.lane.on) qsim_lane_init_kernel<<<(h->cfg.R + 31u) / 32u, 32, 0, h->stream>>>(h->par);
     else qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
     CUDA_TRY(cudaGetLastError());
@@ -544,13 +687,21 @@ int qsim_bind_restore(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
 {
     int rc = attach_workspace(h, ws, bytes, cuda_stream);
     if (rc != QSIM_OK) return rc;
-    // the end time reached so far is in every replication's record; a state that stopped on an internal error
-    // cannot be resumed
-    RepHeader first;
-    CUDA_TRY(cudaMemcpyAsync(&first, h->par.hdr, sizeof first, cudaMemcpyDeviceToHost, h->stream));
+    // the bytes must come from a handle of the same configuration and layout
+    unsigned long long want[2], got[2] = { 0, 0 };
+    workspace_tag(h, want);
+    CUDA_TRY(cudaMemcpyAsync(got, reinterpret_cast<char *>(h->par.not_done) + 16, sizeof got, cudaMemcpyDeviceToHost, h->stream));
+    // the end time reached so far is in every replication's record; a state in which any replication stopped on an
+    // internal error cannot be resumed
+    std::vector<RepHeader> hdr(h->cfg.R);
+    CUDA_TRY(cudaMemcpyAsync(hdr.data(), h->par.hdr, hdr.size() * sizeof(RepHeader), cudaMemcpyDeviceToHost, h->stream));
     CUDA_TRY(cudaStreamSynchronize(h->stream));
-    if (first.err != 0 || !(first.T_end >= 0.0) || !std::isfinite(first.T_end))
-        return fail(QSIM_ESTATE, "the workspace does not hold a resumable state");
+    if (got[0] != want[0] || got[1] != want[1])
+        return fail(QSIM_ESTATE, "the workspace was not saved by a handle of this configuration");
+    for (uint32_t r = 0; r < h->cfg.R; ++r)
+        if (hdr[r].err != 0 || !(hdr[r].T_end >= 0.0) || !std::isfinite(hdr[r].T_end))
+            return fail(QSIM_ESTATE, "the workspace does not hold a resumable state (replication " + std::to_string(r) + ")");
+    const RepHeader &first = hdr[0];
     h->T_end_abs = first.T_end;
     h->bound = true;
     return QSIM_OK;
@@ -749,6 +900,25 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
     if (!h) return fail(QSIM_EINVAL, "null handle");
     if (!h->bound) return fail(QSIM_ESTATE, "qsim_stats before qsim_bind");
     const uint32_t R = h->cfg.R, I = h->cfg.I;
+    if (!per_rep && !hist_ttft && !hist_tpot) {
+        // totals only: reduced on the device, a few KB come back
+        if (!totals) { CUDA_TRY(cudaStreamSynchronize(h->stream)); return QSIM_OK; }
+        char *base = static_cast<char *>(h->ws);
+        TotalsRec *d_out = reinterpret_cast<TotalsRec *>(base + h->sec.red);
+        double *d_F = reinterpret_cast<double *>(base + h->sec.red + sizeof(TotalsRecBytes));
+        CUDA_TRY(cudaMemsetAsync(d_out, 0, sizeof(TotalsRec), h->stream));
+        qsim_totals_gather_kernel<<<(R + 127u) / 128u, 128, 0, h->stream>>>(h->par.hdr, R, I, d_F, d_out);
+        qsim_totals_sum_kernel<<<1, 64, 0, h->stream>>>(R, I, d_F, d_out);
+        CUDA_TRY(cudaGetLastError());
+        h->launches += 2;
+        TotalsRec out;
+        CUDA_TRY(cudaMemcpyAsync(&out, d_out, sizeof out, cudaMemcpyDeviceToHost, h->stream));
+        CUDA_TRY(cudaStreamSynchronize(h->stream));
+        if (out.err_code)
+            return fail(QSIM_EOVERFLOW, "replication " + std::to_string(out.err_rep) + " hit an internal bound (code " + std::to_string(out.err_code) + ")");
+        *totals = out.tot;
+        return QSIM_OK;
+    }
     std::vector<RepHeader> hdr(R);
     CUDA_TRY(cudaMemcpyAsync(hdr.data(), h->par.hdr, (size_t)R * sizeof(RepHeader), cudaMemcpyDeviceToHost, h->stream));
     CUDA_TRY(cudaStreamSynchronize(h->stream));
@@ -759,49 +929,9 @@ int qsim_stats(qsim_t *h, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint6
         if (H.err) return fail(QSIM_EOVERFLOW, "replication " + std::to_string(r) + " hit an internal bound (code " + std::to_string(H.err) + ")");
         qsim_rep_stats st;
         std::memset(&st, 0, sizeof st);
-        const double T = H.T_end;
-        st.T_elapsed = T - H.T_reset;
-        for (int l = 0; l < 32; ++l) {
-            st.iters_mixed += H.iters_mixed[l];
-            st.iters_solo += H.iters_solo[l];
-            st.busy_mixed = st.busy_mixed + H.busy_mixed[l];
-            st.busy_solo = st.busy_solo + H.busy_solo[l];
-        }
-        st.events = H.events + st.iters_mixed + st.iters_solo;   // H.events counts block switches; class events are added below
-        for (uint32_t i = 0; i < I; ++i) {
-            const ClassState &c = H.cs[i];
-            qsim_class_stats &o = st.cls[i];
-            o.arrivals = c.arrivals; o.admitted = c.admitted; o.prefill_done = c.prefill_done;
-            o.placed_mixed = c.placed_mixed; o.placed_solo = c.placed_solo; o.done_mixed = c.done_mixed;
-            o.done_solo = c.done_solo; o.abandoned_p = c.abandoned_p; o.abandoned_d = c.abandoned_d;
-            o.overflow = c.overflow; o.overflow_d = c.overflow_d; o.tokens_in_prefilled = c.tok_in_pf;
-            o.tokens_in_completed = c.tok_in_done; o.tokens_out_completed = c.tok_out_done;
-            const uint32_t Qd = c.Qd0 + c.Qd1;
-            o.Qp = c.pq_n; o.X = c.X; o.Qd = Qd; o.Ym = c.Ym; o.Ys = c.Ys;
-            // integrals are reported up to the end of the run without touching the stored state
-            o.area_Qp = c.aQp.area + (double)c.pq_n * (T - c.aQp.t_last);
-            o.area_X = c.aX.area + (double)c.X * (T - c.aX.t_last);
-            o.area_Qd = c.aQd.area + (double)Qd * (T - c.aQd.t_last);
-            o.area_Ym = (c.sYm_out - c.sYm_in) + (double)c.Ym * (T - H.T_reset);
-            o.area_Ys = (c.sYs_out - c.sYs_in) + (double)c.Ys * (T - H.T_reset);
-            o.sum_ttft = c.sum_ttft; o.sum_tpot = c.sum_tpot;
-            st.events += c.arrivals + c.abandoned_p + c.abandoned_d;
-        }
+        rep_stats_of(H, I, st);
         if (per_rep) per_rep[r] = st;
-        tot.iters_mixed += st.iters_mixed; tot.iters_solo += st.iters_solo; tot.events += st.events;
-        tot.busy_mixed += st.busy_mixed; tot.busy_solo += st.busy_solo; tot.T_elapsed += st.T_elapsed;
-        for (uint32_t i = 0; i < I; ++i) {
-            const qsim_class_stats &a = st.cls[i];
-            qsim_class_stats &b = tot.cls[i];
-            b.arrivals += a.arrivals; b.admitted += a.admitted; b.prefill_done += a.prefill_done;
-            b.placed_mixed += a.placed_mixed; b.placed_solo += a.placed_solo; b.done_mixed += a.done_mixed;
-            b.done_solo += a.done_solo; b.abandoned_p += a.abandoned_p; b.abandoned_d += a.abandoned_d;
-            b.overflow += a.overflow; b.overflow_d += a.overflow_d; b.tokens_in_prefilled += a.tokens_in_prefilled;
-            b.tokens_in_completed += a.tokens_in_completed; b.tokens_out_completed += a.tokens_out_completed;
-            b.Qp += a.Qp; b.X += a.X; b.Qd += a.Qd; b.Ym += a.Ym; b.Ys += a.Ys;
-            b.area_Qp += a.area_Qp; b.area_X += a.area_X; b.area_Qd += a.area_Qd; b.area_Ym += a.area_Ym;
-            b.area_Ys += a.area_Ys; b.sum_ttft += a.sum_ttft; b.sum_tpot += a.sum_tpot;
-        }
+        add_rep_stats(tot, st, I);
     }
     if (totals) *totals = tot;
     if (hist_ttft || hist_tpot) {
@@ -911,6 +1041,70 @@ int qsim_simulate(const qsim_config *cfg, const qsim_class *classes, const doubl
     return rc;
 }
 
+int qsim_simulate_waves(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
+                        const double *prices, const double *coef, const qsim_targets *tg, uint64_t horizon_iters,
+                        uint32_t wave, qsim_rep_stats *totals, qsim_rep_stats *per_rep, uint32_t *waves_run)
+{
+    int rc = validate(cfg, classes, rates, lengths, prices, coef, tg);
+    if (rc != QSIM_OK) return rc;
+    const uint32_t R = cfg->R, I = cfg->I;
+    // bytes of state for w resident replications (a handle is cheap: it only holds the tables)
+    auto bytes_for = [&](uint32_t w, size_t &bytes) -> int {
+        qsim_config c = *cfg;
+        c.R = w;
+        qsim_t *h = nullptr;
+        int r = qsim_create(&h, &c, classes, rates, lengths, prices, coef, tg);
+        if (r != QSIM_OK) return r;
+        bytes = h->sec.total;
+        qsim_destroy(h);
+        return QSIM_OK;
+    };
+    uint32_t W = wave == 0 || wave > R ? R : wave;
+    size_t need = 0;
+    rc = bytes_for(W, need);
+    if (rc != QSIM_OK) return rc;
+    if (wave == 0) {
+        // the largest wave whose state fits in nine tenths of the free device memory
+        size_t free_b = 0, total_b = 0;
+        CUDA_TRY(cudaMemGetInfo(&free_b, &total_b));
+        while (need > free_b / 10 * 9 && W > 1) {
+            W = (W + 1) / 2;
+            rc = bytes_for(W, need);
+            if (rc != QSIM_OK) return rc;
+        }
+    }
+    void *ws = nullptr;
+    cudaError_t e = cudaMalloc(&ws, need);
+    if (e != cudaSuccess) return fail(QSIM_ENOMEM, std::string("cudaMalloc(workspace of one wave): ") + cudaGetErrorString(e));
+    qsim_rep_stats tot;
+    std::memset(&tot, 0, sizeof tot);
+    std::vector<qsim_rep_stats> buf(per_rep ? 0 : W);
+    uint32_t n_waves = 0;
+    for (uint32_t done = 0; done < R && rc == QSIM_OK; done += W, ++n_waves) {
+        qsim_config c = *cfg;
+        c.R = R - done < W ? R - done : W;
+        c.rep_offset = cfg->rep_offset + done;        // random streams are keyed by the global replication index
+        qsim_t *h = nullptr;
+        rc = qsim_create(&h, &c, classes, rates, lengths, prices, coef, tg);
+        if (rc != QSIM_OK) break;
+        qsim_rep_stats *out = per_rep ? per_rep + done : buf.data();
+        if (h->sec.total > need) rc = fail(QSIM_EWORKSPACE, "a later wave needs more state than the first");
+        if (rc == QSIM_OK) rc = qsim_bind(h, ws, need, nullptr);
+        if (rc == QSIM_OK) rc = qsim_run(h, horizon_iters);
+        if (rc == QSIM_OK) rc = qsim_stats(h, nullptr, out, nullptr, nullptr);
+        if (rc == QSIM_OK)
+            for (uint32_t r = 0; r < c.R; ++r) add_rep_stats(tot, out[r], I);
+        const std::string keep = g_err;
+        qsim_destroy(h);
+        if (rc != QSIM_OK) g_err = keep;
+    }
+    cudaFree(ws);
+    if (rc != QSIM_OK) return rc;
+    if (totals) *totals = tot;
+    if (waves_run) *waves_run = n_waves;
+    return QSIM_OK;
+}
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------------
@@ -954,6 +1148,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     if (rc != QSIM_OK) return rc;
     h.device = dev;
     h.stream = stream;
+    h.ws = base;
     Params &p = h.par;
     // scratch = [state sections | block table | length tables]
     const size_t off_blocks = h.sec.total;

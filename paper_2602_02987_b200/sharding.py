@@ -49,3 +49,28 @@ def totals(stats: dict) -> dict:
         else:
             out[k] = v.sum(axis=0, dtype=np.uint64)
     return out
+
+
+def combine_totals(mine: dict, my_ms: float, group=None) -> dict:
+    """End-of-run exchange of a sharded run: every rank contributes its own totals (a dict of numbers) and its device
+    time.  Integers are summed exactly, floats are added in rank order (a fixed order), and the time is the maximum over
+    ranks ("max_ms").  With one process (no process group) the input comes back unchanged.  This is the only exchange of
+    the multi-GPU layout: the simulation itself never communicates."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return dict(mine, max_ms=float(my_ms))
+    world = dist.get_world_size(group)
+    parts = [None] * world
+    dist.all_gather_object(parts, (dict(mine), float(my_ms)), group=group)
+    out = {}
+    for k in mine:
+        vals = [p[0][k] for p in parts]
+        if all(isinstance(v, (int, np.integer)) for v in vals):
+            out[k] = int(sum(int(v) for v in vals))
+        else:
+            acc = 0.0
+            for v in vals:
+                acc = acc + float(v)
+            out[k] = acc
+    out["max_ms"] = max(p[1] for p in parts)
+    return out

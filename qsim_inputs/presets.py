@@ -358,14 +358,3 @@ def ctmc_instance(n=50, R=8, router=ROUTER_SOLO_FIRST, gate=GATE_OCCUPANCY, B=16
                             qd=plan.qd.tolist())))
     inp.validate()
     return inp
-
-
-def ctmc_revenue_rate(inp: CtmcInputs, st: dict, separate=None) -> np.ndarray:
-    """Per-GPU revenue rate of every replication from the integer counters: bundled charging credits
-    c_p P_i + c_d D_i at decode completion (Eq. (21)-(22)); separate charging credits c_p P_i at prefill
-    completion and c_d D_i at decode completion (Eq. (23))."""
-    sep = inp.meta.get("separate", False) if separate is None else separate
-    done = (st["done_mixed"] + st["done_solo"]).astype(float)
-    pf = st["prefill_done"].astype(float) if sep else done
-    rev = (inp.prices[0] * inp.P * pf + inp.prices[1] * inp.D * done).sum(axis=1)
-    return rev / (inp.N * st["T_elapsed"])

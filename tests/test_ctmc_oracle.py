@@ -4,7 +4,7 @@ Poisson arrivals, and the optimality / occupancy-convergence theorems of Section
 import numpy as np
 import pytest
 
-from oracle import CtmcOracle, run_ctmc_oracle
+from oracle import CtmcOracle, ctmc_revenue_rate, run_ctmc_oracle
 from qsim_inputs import presets
 from qsim_inputs.spec import GATE_PRIORITY, ROUTER_SLI, ROUTER_SOLO_FIRST, CtmcInputs
 
@@ -154,7 +154,7 @@ def test_priority_gate_serves_the_first_rank_under_backlog():
 
 def revenue_window(inp, T1, T2):
     d = window(inp, T1, T2)
-    return presets.ctmc_revenue_rate(inp, d), d
+    return ctmc_revenue_rate(inp, d), d
 
 
 def test_revenue_converges_to_the_lp_optimum():

@@ -40,6 +40,9 @@ def test_ctmc_parity_element_by_element(router, gate, theta, lam):
     compare(gpu_run(inp, [120.0]), ref, "one call")
     compare(gpu_run(inp, [7.5, 7.5, 60.0, 120.0]), ref, "resumed")
     assert ref["abandoned_d"].sum() > 0 or min(theta) == 0.0
+    # revenue per GPU (qsim_ctmc_revenue, Eq. (21)-(23)) against the oracle side's own arithmetic on the oracle's counters
+    from oracle import ctmc_revenue_rate
+    assert np.allclose(gpu_run(inp, [120.0])["_revenue_rate"], ctmc_revenue_rate(inp, ref), rtol=1e-12, atol=0)
 
 
 def test_ctmc_full_size_in_the_bench_launch_configuration():

@@ -144,6 +144,14 @@ def test_tiny_queue_capacity_overflows_identically():
     assert st["overflow"].sum() > 0
 
 
+def test_small_queue_with_abandonment_from_inside():
+    # eight positions per class queue, short patience: requests leave from inside the ring, positions run out while
+    # fewer than eight wait (the ring is packed again), and arrivals overflow when eight do wait
+    inp = presets.crowded("prefill", N=4, R=6, placement=PLACE_LEAST_LOADED).with_(qcap=8)
+    st = check(inp, 20_000)
+    assert st["overflow"].sum() > 0 and st["abandoned_p"].sum() > 500
+
+
 def test_resumed_and_budget_limited_runs_are_identical():
     inp = presets.cfg2(N=48, R=5)
     a, sa = lane_run(inp, 3000)

@@ -214,6 +214,9 @@ def test_checkpoint_and_resume_in_a_new_handle():
         assert_parity(got, ref, what=f"{inp.name} resumed from a checkpoint")
     with pytest.raises(QSimError):
         QSim(presets.cfg1(R=5), checkpoint=saved)
+    # same number of bytes, another seed: the workspace's fingerprint does not match the handle
+    with pytest.raises(QSimError, match="configuration"):
+        QSim(inp.with_(seed=inp.seed + 1), checkpoint=saved)
 
 
 def test_replication_offset_shards_compose():
@@ -320,3 +323,32 @@ def test_cfg1_full_size_in_the_bench_launch_configuration():
         a = g["arrivals"][:, i].astype(float)
         assert abs(a.mean() - mean) < 5.0 * np.sqrt(mean / a.size)
         assert abs(a.var(ddof=1) / mean - 1.0) < 5.0 * np.sqrt(2.0 / (a.size - 1))
+
+
+def test_totals_reduced_on_the_device_are_the_host_totals_bit_for_bit():
+    """qsim_stats with totals only sums on the device (integer counters exactly, fp64 statistics in replication order);
+    the result must be the very bits of the host's sum over the per-replication records, in both kernel families."""
+    import os
+    from paper_2602_02987_b200 import QSim, simulate_host
+    for fam, inp, H in (("warp", presets.cfg1(R=37), 600), ("lane", presets.cfg4(N=24, R=70), 700)):
+        os.environ["QSIM_FAMILY"] = fam
+        try:
+            sim = QSim(inp)
+            sim.run(H)
+            full = sim.stats(with_totals=True)["_totals"]
+            _, _, tot = sim.totals()
+            sim.close()
+        finally:
+            del os.environ["QSIM_FAMILY"]
+        for k, v in full.items():
+            if v.ndim == 2:
+                got = np.array([[getattr(tot.cls[i], k) for i in range(inp.I)]], v.dtype)
+            else:
+                got = np.array([getattr(tot, k)], v.dtype)
+            assert np.array_equal(got, v), (fam, k, got, v)
+    # the one-call host entry point with totals only
+    inp = presets.cfg0(R=5, horizon_iters=1500)
+    a = simulate_host(inp, 1500)["_totals"]
+    b = simulate_host(inp, 1500, per_rep=False)["_totals"]
+    for k in a:
+        assert np.array_equal(a[k], b[k]), k

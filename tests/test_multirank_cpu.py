@@ -14,16 +14,21 @@ def _worker(rank, world, port, R, horizon, out_dir):
     sys.path.insert(0, ROOT)
     import torch.distributed as dist
     from oracle import run_oracle
-    from paper_2602_02987_b200.sharding import gather_stats, shard, totals
+    from paper_2602_02987_b200.sharding import combine_totals, gather_stats, shard, totals
     from qsim_inputs import presets
     dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=rank, world_size=world)
     count, offset = shard(R, world, rank)
     inp = presets.cfg0(R=count, horizon_iters=horizon).with_(rep_offset=offset)
     local = run_oracle(inp, horizon)
     everything = gather_stats(local)
+    # the benchmark's end-of-run exchange: each rank's own totals and its time
+    mine = {"iters": int(local["iters_mixed"].sum() + local["iters_solo"].sum()), "events": int(local["events"].sum()),
+            "T": float(local["T_elapsed"].sum())}
+    combined = combine_totals(mine, 100.0 + rank)
     if rank == 0:
         np.savez(os.path.join(out_dir, "gathered.npz"), **everything)
         np.savez(os.path.join(out_dir, "totals.npz"), **totals(everything))
+        np.savez(os.path.join(out_dir, "combined.npz"), **{k: np.array(v) for k, v in combined.items()})
     dist.barrier()
     dist.destroy_process_group()
 
@@ -73,6 +78,12 @@ def test_two_ranks_reproduce_the_single_process_run(tmp_path):
     wt = totals(want)
     for k in wt:
         assert np.array_equal(tot[k], wt[k]), k
+    # the benchmark's exchange of per-rank totals: integers exact, time = the slowest rank
+    comb = dict(np.load(tmp_path / "combined.npz"))
+    assert int(comb["iters"]) == int(want["iters_mixed"].sum() + want["iters_solo"].sum())
+    assert int(comb["events"]) == int(want["events"].sum())
+    assert abs(float(comb["T"]) - float(want["T_elapsed"].sum())) <= 1e-12 * float(comb["T"])
+    assert float(comb["max_ms"]) == 101.0
 
 
 def test_two_ranks_reproduce_the_exponential_service_run(tmp_path):
