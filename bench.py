@@ -40,7 +40,7 @@ N_SM, SCHEDULERS = 148, 4  # issue peak of the GPU: SMs x schedulers x one warp 
 PREWARM = 2000             # iterations of horizon before the warm-up steps (steady state)
 
 # workload -> (replications per GPU, iterations of horizon per step)
-DEFAULTS = {"cfg2": (4096, 400), "cfg1": (1024, 100_000), "cfg0": (16, 10_000), "cfg3": (2048, 300), "cfg4": (8192, 300)}
+DEFAULTS = {"cfg2": (4096, 500), "cfg1": (1024, 100_000), "cfg0": (16, 10_000), "cfg3": (2048, 300), "cfg4": (8192, 300)}
 CSRC = os.path.join(ROOT, "paper_2602_02987_b200", "csrc")
 
 

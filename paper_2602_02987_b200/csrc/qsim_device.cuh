@@ -146,6 +146,8 @@ struct Params {
     uint32_t *hist_mem;          // [R][I][2][NBIN] or null
     uint32_t *not_done;          // single counter: replications that stopped on the event budget
     uint32_t srv_bytes;
+    uint32_t tarr_global;        // pf_tarr lives in tarr_g instead of shared memory
+    double *tarr_g;              // [R][N]
     LanePar lane;
 };
 
@@ -341,7 +343,7 @@ struct Sim {
     MwRes *res;
     WarpClassStats *wcs;         // [nwarps][MAXI]
     // shared memory (lane-owned entries)
-    double *tnext, *pf_tarr, *taucur;      // taucur: duration of the running iteration
+    double *tnext, *pf_tarr;               // pf_tarr: arrival time of the request in prefill (shared memory, or global memory on large clusters)
     uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
     uint16_t *ndec, *nact, *pfcur;
     uint16_t *sfin16;            // [Npad][B]  low 16 bits of each slot's finish iteration (f_slots)
@@ -864,7 +866,6 @@ struct Sim {
             if (f_kappa()) { K[g] = Kg; Kpend[g] = 0; }
             pfcur[g] = (uint16_t)pc;
             nact[g] = (uint16_t)(nd | fl);
-            taucur[g] = tau;
             tnext[g] = __dadd_rn(ts, tau);
         }
     }
@@ -1078,7 +1079,7 @@ struct Sim {
                 itg = it[g] + 1;
                 it[g] = itg;
                 const uint32_t na = nact[g] & 0x3fffu, pc = pfcur[g], Kg = f_kappa() ? K[g] : 0u;
-                const double tau = taucur[g];
+                const double tau = iter_time(p, pc, na, Kg, f_kappa());     // duration of the iteration that ends (the chain of its start)
                 if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); }
                 else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
                 if (f_kappa()) K[g] = Kg + na;
@@ -1198,9 +1199,9 @@ struct Sim {
     {
         // straight-line: all fields are read first and the stores are predicated on `act` (see start_at)
         const uint32_t it0 = it[g], na_raw = nact[g], pc = pfcur[g], nd = ndec[g], pj = pfjob[g], pr = pfrem[g], nf = nfin[g];
-        const double tau = taucur[g];
         uint32_t K0 = 0, Kp = 0;
         if (f_kappa()) { K0 = K[g]; Kp = Kpend[g]; }
+        const double tau = iter_time(p, pc, na_raw & 0x3fffu, K0, f_kappa());   // duration of the iteration that ends (the chain of its start)
         const uint32_t itg = it0 + 1u;
         const uint32_t rem = pr - pc;                       // prompt tokens left after this iteration's chunk
         const bool retire = (na_raw & 0x4000u) != 0;        // a decode finished: the GPU waits for retire_decodes
@@ -1219,7 +1220,7 @@ struct Sim {
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
             if (f_kappa()) { K[g] = restart ? Kg : Kend; if (restart) Kpend[g] = 0; }
             pfcur[g] = restart ? (uint16_t)pc2 : (uint16_t)0;
-            if (restart) { nact[g] = (uint16_t)(nd | fl); taucur[g] = tau2; }
+            if (restart) nact[g] = (uint16_t)(nd | fl);
             tnext[g] = restart ? __dadd_rn(te, tau2) : dinf();
         }
         return act && retire;
@@ -1516,18 +1517,19 @@ struct Sim {
 
 // shared-memory carve-up for one replication (one warp per block)
 struct SmemLayout {
-    uint32_t off_tnext, off_tarr, off_tau, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
+    uint32_t off_tnext, off_tarr, off_it, off_nfin, off_pfrem, off_pfjob, off_K, off_Kpend, off_ndec, off_nact,
         off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, off_wcs, off_cmd, off_res, total;
 };
 
-__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps = 1,
-                                                  bool kappa = true)
+// tarr_global: the arrival times of the requests in prefill live in global memory (large clusters: shared memory is what
+// limits the resident replications there); I: classes (sizes the ring of arrival draws)
+__host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps, bool kappa,
+                                                  bool tarr_global, uint32_t I)
 {
     SmemLayout L;
     uint32_t o = 0;
     L.off_tnext = o; o += 8 * Npad;
-    L.off_tarr = o; o += 8 * Npad;
-    L.off_tau = o; o += 8 * Npad;
+    L.off_tarr = o; if (!tarr_global) o += 8 * Npad;
     L.off_it = o; o += 4 * Npad;
     L.off_nfin = o; o += 4 * Npad;
     L.off_pfrem = o; o += 4 * Npad;
@@ -1549,7 +1551,7 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     o = (o + 15u) & ~15u;
     L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
     o = (o + 15u) & ~15u;
-    L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * MAXI;
+    L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * I;
     L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * STAGE_CAP;
     L.off_stte = o; o += 8 * STAGE_CAP;
     L.off_pqh = o; o += (uint32_t)sizeof(QEntry) * MAXI;
@@ -1566,8 +1568,7 @@ template <int SPL, uint32_t F>
 __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const SmemLayout &L)
 {
     s.tnext = reinterpret_cast<double *>(sm + L.off_tnext);
-    s.pf_tarr = reinterpret_cast<double *>(sm + L.off_tarr);
-    s.taucur = reinterpret_cast<double *>(sm + L.off_tau);
+    s.pf_tarr = s.p.tarr_global ? s.p.tarr_g + (size_t)s.rep * s.p.N : reinterpret_cast<double *>(sm + L.off_tarr);
     s.it = reinterpret_cast<uint32_t *>(sm + L.off_it);
     s.nfin = reinterpret_cast<uint32_t *>(sm + L.off_nfin);
     s.pfrem = reinterpret_cast<uint32_t *>(sm + L.off_pfrem);
@@ -1611,7 +1612,7 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
     extern __shared__ __align__(16) char sm[];
     const int lane = threadIdx.x;
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, 1, p.coef[5] != 0.0);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, 1, p.coef[5] != 0.0, p.tarr_global != 0, p.I);
         Sim<SPLT, FT> s(p, lane, rep);
         bind_pointers(s, sm, L);
         __syncwarp();
@@ -1663,7 +1664,14 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
 
 // Advance replications to their new end time (or until the per-launch event budget runs out).
 template <int SPLT, uint32_t FT>
-__global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_kernel(Params p)
+// One-warp instances whose slot records live in global memory need little shared memory, so registers decide how many
+// replications are resident on an SM: they are compiled for at least 12 blocks per SM (at most 168 registers, a few
+// bytes of spills; +16-24 % at N = 64 with thousands of replications).  Instances with the finish stamps on chip are
+// limited by shared memory and keep all the registers they want (the cap cost them 13 %).
+#ifndef QSIM_MIN_BLOCKS
+#define QSIM_MIN_BLOCKS 12
+#endif
+__global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) || (FT & F_SLOTS)) ? 1 : QSIM_MIN_BLOCKS) qsim_run_kernel(Params p)
 {
     extern __shared__ __align__(16) char sm[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1671,7 +1679,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, 1) qsim_run_ke
     for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
         RepHeader &h = p.hdr[rep];
         if (!p.advance && h.done) continue;
-        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0);
+        const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0, p.tarr_global != 0, p.I);
         Sim<SPLT, FT> s(p, lane, rep);
         s.warp = warp;
         s.nwarps = (int)(nthr >> 5);

@@ -812,7 +812,7 @@ struct LaneSim {
         for (;;) {
             if (!cl_valid) class_candidates();
             // plain iteration ends, one after the other, while no other event comes first
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < 4; ++k) {
                 if (!nx_valid) peek();
                 if (!(nx_t < cl_t) || nx_t > tend_bits || budget == 0 || err || !end_is_plain(nx_rec)) break;
                 --budget;

@@ -38,7 +38,7 @@ size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 struct TotalsRecBytes { char b[2048]; };      // room for the device totals record (checked where the record is defined)
 
 struct Sections {
-    size_t hdr, srv, fin, rec, pq, dq, hist, flag, red, total;
+    size_t hdr, srv, fin, rec, pq, dq, hist, flag, red, tarr, total;
     // one-thread-per-replication family
     size_t l_srv, l_tarr, l_head, l_bm, l_tree, l_sfin, l_snode, l_srec, l_sfree, l_pql;
 };
@@ -51,6 +51,7 @@ struct qsim {
     double prices[2]{};
     Params par{};
     SmemLayout lay{};
+    uint32_t init_smem = 0;       // shared memory of the set-up kernel's block (one warp, same per-GPU image)
     Sections sec{};
     BlockPar *d_blocks = nullptr;
     uint32_t *d_lengths = nullptr;
@@ -73,7 +74,7 @@ struct qsim {
 
 namespace {
 
-Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
+Sections layout_sections(const qsim_config &c, uint32_t srv_bytes, bool tarr_global)
 {
     Sections s{};
     size_t o = 0;
@@ -87,6 +88,7 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes)
     s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
     s.flag = o; o = align256(o + 256);
     s.red = o; o = align256(o + sizeof(TotalsRecBytes) + R * (size_t)(c.I * 7u + 3u) * 8);    // totals record + fp64 statistics per replication
+    s.tarr = o; if (tarr_global) o = align256(o + R * (size_t)c.N * 8);
     s.total = o;
     return s;
 }
@@ -300,7 +302,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
 void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
-    uint32_t W = rows >= 64 ? 16u : (rows >= 16 ? 4u : 1u);
+    uint32_t W = rows >= 64 ? 16u : (rows >= 32 ? 4u : 1u);      // best of sweeps over 1, 2, 4, 8, 16 warps at 512, 1024, 4096 GPUs
     if (const char *e = std::getenv("QSIM_WARPS")) {
         const int v = std::atoi(e);
         if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
@@ -379,21 +381,27 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     // the per-GPU arrays are padded to the unrolled row count of the chosen instance
     if (v.spl > 0) p.Npad = (uint32_t)v.spl * 32u;
     // finish stamps + occupancy bits go to shared memory when the whole block state stays small
-    p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, kappa).total <= 40u * 1024u ? 1u : 0u;
+    p.slots_smem = smem_layout(p.Npad, p.B, 1, 1, kappa, p.Npad > 128u, cfg.I).total <= 40u * 1024u ? 1u : 0u;
     if (p.slots_smem) v = pick_run_kernel(cfg.N, feat | F_SLOTS);
     h.run_fn = v.fn;
     h.nwarps = 1;
     choose_multiwarp(cfg.N, feat, p, h.run_fn, h.nwarps);
-    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa);
+    // beyond four rows of GPUs shared memory limits the resident replications: the arrival times of the requests in
+    // prefill (read once per finished prefill) move to global memory
+    p.tarr_global = (p.Npad > 128u) ? 1u : 0u;
+    h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa, p.tarr_global != 0, cfg.I);
+    h.init_smem = smem_layout(p.Npad, p.B, p.slots_smem, 1, kappa, p.tarr_global != 0, cfg.I).total;
     p.srv_bytes = h.lay.srv_bytes;
     if (h.lay.total > 227u * 1024u)
         return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
-    h.sec = layout_sections(cfg, p.srv_bytes);
+    h.sec = layout_sections(cfg, p.srv_bytes, p.tarr_global != 0);
     for (int k = 0; k < 6; ++k) h.coef[k] = coef[k];
-    // Kernel family.  One thread per replication pays when there are enough replications to fill the device with
-    // independent chains; a warp per replication is faster for few replications.  QSIM_FAMILY=lane / warp overrides.
+    // Kernel family.  A replication advances at about the same rate on one thread whatever its cluster size, while the
+    // warp-per-replication kernels slow down in proportion to the cluster (few replications fit on an SM and their
+    // master warp searches all rows).  Measured on a B200: one thread per replication wins when R x N exceeds about
+    // 7 million (N = 1024 from R = 8192, N = 4096 from R = 2048).  QSIM_FAMILY=lane / warp overrides.
     std::memset(&p.lane, 0, sizeof p.lane);
-    bool lane = h.allow_lane && lane_supports(cfg, coef) && cfg.R >= 2048u;
+    bool lane = h.allow_lane && lane_supports(cfg, coef) && (unsigned long long)cfg.R * cfg.N >= 7000000ull;
     if (const char *e = std::getenv("QSIM_FAMILY")) {
         if (std::strcmp(e, "lane") == 0) lane = h.allow_lane && lane_supports(cfg, coef);
         else if (std::strcmp(e, "warp") == 0) lane = false;
@@ -635,6 +643,7 @@ static int attach_workspace(qsim_t *h, void *ws, size_t bytes, void *cuda_stream
     p.dq = reinterpret_cast<QEntry *>(base + h->sec.dq);
     p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h->sec.flag);
+    p.tarr_g = p.tarr_global ? reinterpret_cast<double *>(base + h->sec.tarr) : nullptr;
     if (p.lane.on) {
         LanePar &q = p.lane;
         q.srv = reinterpret_cast<LaneSrv *>(base + h->sec.l_srv);
@@ -676,7 +685,7 @@ int qsim_bind(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
         CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char *>(h->par.not_done) + 16, tag, sizeof tag, cudaMemcpyHostToDevice, h->stream));
     }
     if (h->par.lane.on) qsim_lane_init_kernel<<<(h->cfg.R + 31u) / 32u, 32, 0, h->stream>>>(h->par);
-    else qsim_init_kernel<<<h->cfg.R, 32, h->lay.total, h->stream>>>(h->par);
+    else qsim_init_kernel<<<h->cfg.R, 32, h->init_smem, h->stream>>>(h->par);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
     h->bound = true;
@@ -1178,11 +1187,12 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.dq = reinterpret_cast<QEntry *>(base + h.sec.dq);
     p.hist_mem = nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h.sec.flag);
+    p.tarr_g = p.tarr_global ? reinterpret_cast<double *>(base + h.sec.tarr) : nullptr;
     CUDA_TRY(allow_large_smem(reinterpret_cast<const void *>(h.run_fn)));
     CUDA_TRY(allow_large_smem(reinterpret_cast<const void *>(qsim_init_kernel)));
     // the array keeps the previous call's contents: the init kernel rewrites every header and GPU image;
     // queue rings and slot lists are never read before they are written, the flag is cleared per launch
-    qsim_init_kernel<<<cfg->R, 32, h.lay.total, stream>>>(p);
+    qsim_init_kernel<<<cfg->R, 32, h.init_smem, stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     bool advance = true;
     for (;;) {

@@ -197,3 +197,32 @@ def test_the_two_families_agree_and_unsupported_modes_fall_back():
     assert_parity(lane, warp, what="lane family against warp family")
     # random placement is simulated by the warp-per-replication kernels only
     check(presets.paper_instance(n=20, R=3, placement=PLACE_RANDOM), 2000, expect_lane=False)
+
+
+def test_whole_runs_in_waves_do_not_depend_on_the_wave_size():
+    """qsim_simulate_waves: replications simulated a wave at a time in one bounded workspace.  Random streams are keyed by
+    the global replication index, so waves of 64, of 148 and one wave of all give identical statistics, equal to the
+    resident run's, in both kernel families."""
+    from paper_2602_02987_b200 import QSim, simulate_waves
+    inp = presets.cfg4(N=48, R=300)
+    H = 400
+    resident = {}
+    for fam in ("warp", "lane"):
+        with family(fam):
+            sim = QSim(inp); sim.run(H); whole = resident[fam] = sim.stats(); sim.close()
+            a = simulate_waves(inp, H, wave=64)
+            b = simulate_waves(inp, H, wave=148)
+            c = simulate_waves(inp, H, wave=0)
+        assert (a["_waves"], b["_waves"], c["_waves"]) == (5, 3, 1)
+        for k in whole:
+            if k.startswith("hist"):
+                continue
+            assert np.array_equal(a[k], whole[k]) and np.array_equal(b[k], whole[k]) and np.array_equal(c[k], whole[k]), (fam, k)
+        for k in a["_totals"]:      # totals are added in replication order whatever the waves
+            assert np.array_equal(a["_totals"][k], b["_totals"][k]) and np.array_equal(a["_totals"][k], c["_totals"][k]), (fam, k)
+    # a shard of a larger job: the offset composes with the waves
+    with family("warp"):
+        tail = simulate_waves(inp.with_(R=100, rep_offset=200), H, wave=33)
+    for k in resident["warp"]:
+        if not k.startswith("hist"):
+            assert np.array_equal(tail[k], resident["warp"][k][200:]), k

@@ -70,7 +70,7 @@ def check(inp, horizon, **kw):
 
 @pytest.mark.parametrize("N,H", [(1024, 700), (4096, 450)])
 def test_cfg4_steady_state_at_benchmark_cluster_sizes(N, H):
-    # occupancy gate, SLI-aware router, histograms; four (N = 1024) and sixteen (N = 4096) warps per replication
+    # occupancy gate, SLI-aware router, histograms; four (N = 1024) and sixteen (N = 4096) warps per replication in the warp family
     st = check(presets.cfg4(N=N, R=2), H, chunks=[H // 3, H - H // 3])
     done = st["done_mixed"] + st["done_solo"]
     assert done.sum() > 20 * N and st["abandoned_p"].sum() > 0

@@ -91,3 +91,37 @@ def test_recipes_are_deterministic_and_valid():
     # sinusoid of amplitude 0.5 around 0.95 of capacity
     tot = c3.rates.sum(axis=1) / c3.meta["capacity"]
     assert math.isclose(tot.max(), 1.45, rel_tol=1e-9) and math.isclose(tot.min(), 0.45, rel_tol=1e-9)
+
+
+def test_planning_grids_show_what_the_paper_reports_for_them():
+    """Section 6.3 (figures only, so the pins are the trends the text states): prefill fairness is dear and decode
+    fairness cheap; the price of a TPOT target explodes towards the floor 1/gamma = 0.022 s and no plan exists below it;
+    revenue grows with B and saturates around B = 16; it falls with beta and alpha and rises with gamma."""
+    from qsim_inputs import lp_sweeps as S
+    inst = S.Instance()
+    free, plan = S.solve(inst, qd_zero=True)
+    pf = S.frontier(inst, "prefill_fair", [0.0, 0.05, 0.1, 0.2, 1.0])
+    df = S.frontier(inst, "decode_fair", [0.0, 1.0, 2.0, 4.0, 16.0])
+    assert np.all(np.diff(pf) >= -1e-9) and np.all(np.diff(df) >= -1e-9)          # a looser target never costs revenue
+    assert abs(pf[-1] - free) < 1e-6 and abs(df[-1] - free) < 1e-6              # and a slack one costs nothing
+    assert (free - pf[0]) > 3.0 * (free - df[0]) and pf[0] < 0.5 * free           # prefill fairness: steep; decode fairness: mild
+    etas = [0.0215, 0.02205, 0.0221, 0.0225, 0.023, 0.024, 0.026, 0.030]
+    tp = S.frontier(inst, "tpot_cap", etas)
+    assert np.isnan(tp[0]) and np.all(np.isfinite(tp[1:]))                        # nothing is feasible below 1/gamma
+    price = S.shadow_price(etas[1:], tp[1:])
+    assert np.all(np.diff(price) <= 1e-6) and price[0] > 5.0 * price[-3] > 0.0 and price[0] > 50.0 * price[-2] > 0.0   # marginal revenue per second of TPOT: steepest at the floor
+    assert abs(tp[-1] - free) < 1e-6
+    # the TPOT target is met with equality while it binds (Eq. (43))
+    _, p2 = S.solve(inst, qd_zero=True, tpot_cap=0.023)
+    assert abs(S.average_tpot(inst, float(p2.x.sum())) - 0.023) < 1e-9
+    rev_B, tpot_B = S.sensitivity(inst, "B", [2, 4, 8, 16, 32, 64])
+    assert np.all(np.diff(rev_B) >= -1e-9) and rev_B[3] > 0.97 * rev_B[-1] and rev_B[1] < 0.7 * rev_B[-1] and rev_B[-2] == rev_B[-1]
+    rev_b, tpot_b = S.sensitivity(inst, "beta", [1e-5, 6.2e-5, 3e-4, 1e-3])
+    assert np.all(np.diff(rev_b) <= 1e-9) and rev_b[-1] < 0.5 * rev_b[0] and np.all(np.diff(tpot_b) > 0)
+    rev_a, _ = S.sensitivity(inst, "alpha", [0.02, 0.05, 0.1, 0.15])
+    assert np.all(np.diff(rev_a) < 0)
+    rev_g, tpot_g = S.sensitivity(inst, "gamma", [10.0, 20.0, 30.0, 45.0])
+    assert np.all(np.diff(rev_g) > 0) and np.all(np.diff(tpot_g) < 0)
+    # the memory-speed grid: more slots help, slower prefill hurts, everywhere
+    g = S.grid(inst, "B", [4, 8, 16, 32], "beta", [3e-5, 6.2e-5, 2e-4])
+    assert np.all(np.diff(g, axis=0) >= -1e-9) and np.all(np.diff(g, axis=1) <= 1e-9)
