@@ -254,10 +254,10 @@ int qsim_simulate_waves(const qsim_config *cfg, const qsim_class *classes, const
  * Who needs it: code that runs where cudaMalloc is off limits - a plugin inside a serving process whose
  * own allocator has already reserved the whole card, so a fresh cudaMalloc would fail or evict; a
  * latency-critical section that cannot afford the device-wide synchronisation cudaMalloc / cudaFree
- * imply; a host that forbids allocation after start-up.  This entry point calls no cudaMalloc, cudaFree,
- * cudaMallocHost or any other allocating routine.  All simulation state, the rate/target table and
- * the length tables live in one array that is compiled into the library: 32 MiB of device memory on
- * every GPU that loads libqsim.so, held until the process exits.
+ * imply.  This entry point makes no device or pinned-memory allocation: no cudaMalloc, cudaFree or
+ * cudaMallocHost (it does use the host heap for small temporaries, e.g. the index of the length tables).
+ * All simulation state, the rate/target table and the length tables live in one array that is compiled
+ * into the library: 32 MiB of device memory on every GPU that loads libqsim.so, held until the process exits.
  *
  * Arguments as in qsim_simulate ([host] inputs, [host] totals / per_rep[R] outputs, either may be NULL),
  * plus cuda_stream (a cudaStream_t, NULL = default stream) on which the copies and kernels are ordered;

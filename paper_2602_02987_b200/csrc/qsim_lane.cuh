@@ -40,6 +40,11 @@ __device__ __forceinline__ uint32_t min8(const uint32_t v[8])
     return min(min(min(v[0], v[1]), min(v[2], v[3])), min(min(v[4], v[5]), min(v[6], v[7])));
 }
 
+// LF = features compiled into an instance of the lane kernels: LF_GENERIC reads every mode from the parameters; otherwise the
+// set bits say what the instance contains (abandonment, SLI-aware router, histograms, blocks) and the rest is compiled out.
+constexpr uint32_t LF_GENERIC = 1, LF_ABANDON = 2, LF_SLI = 4, LF_HIST = 8, LF_BLOCKS = 16;
+
+template <uint32_t LF>
 struct LaneSim {
     const Params &p;
     const uint32_t rep;
@@ -87,9 +92,10 @@ struct LaneSim {
 
     __device__ LaneSim(const Params &p_, uint32_t rep_) : p(p_), rep(rep_), h(p_.hdr[rep_]) {}
 
-    __device__ __forceinline__ bool f_abandon() const { return p.any_theta != 0; }
-    __device__ __forceinline__ bool f_sli() const { return p.router == 1; }
-    __device__ __forceinline__ bool f_blocks() const { return p.nblk > 1; }
+    __device__ __forceinline__ bool f_abandon() const { return (LF & LF_GENERIC) ? p.any_theta != 0 : (LF & LF_ABANDON) != 0; }
+    __device__ __forceinline__ bool f_sli() const { return (LF & LF_GENERIC) ? p.router == 1 : (LF & LF_SLI) != 0; }
+    __device__ __forceinline__ bool f_blocks() const { return (LF & LF_GENERIC) ? p.nblk > 1 : (LF & LF_BLOCKS) != 0; }
+    __device__ __forceinline__ bool f_hist() const { return (LF & LF_GENERIC) ? hist != nullptr : (LF & LF_HIST) != 0; }
     __device__ __forceinline__ double block_start(uint32_t b) const { return __dmul_rn((double)b, p.block_len); }
 
     __device__ __forceinline__ void bind()
@@ -558,7 +564,7 @@ struct LaneSim {
                 c.tok_out_done += D;
                 const double tpot = __ddiv_rn(__dsub_rn(t, r.tpf), (double)D);
                 c.sum_tpot = __dadd_rn(c.sum_tpot, tpot);
-                if (hist) atomicAdd(&hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)], 1u);
+                if (f_hist()) atomicAdd(&hist[((size_t)i * 2 + 1) * NBIN + hist_bin(tpot)], 1u);
             }
             s.nfin = (uint32_t)(root >> 16);
             s.ndec = (uint16_t)nd;
@@ -580,7 +586,7 @@ struct LaneSim {
                 c.tok_in_pf += P;                  // separate charging credits the prompt here, Eq. (23)
                 const double ttft = __dsub_rn(t, tarr[g]);
                 c.sum_ttft = __dadd_rn(c.sum_ttft, ttft);
-                if (hist) atomicAdd(&hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)], 1u);
+                if (f_hist()) atomicAdd(&hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)], 1u);
                 uint32_t pool = 0;
                 if (f_sli()) {
                     // SLI-aware router: one uniform per finished prefill decides the pool
@@ -859,7 +865,7 @@ __global__ void __launch_bounds__(32) qsim_lane_init_kernel(Params p)
     const uint32_t rep = blockIdx.x * blockDim.x + threadIdx.x;
     if (rep >= p.R) return;
     const LanePar &q = p.lane;
-    LaneSim s(p, rep);
+    LaneSim<LF_GENERIC> s(p, rep);
     s.bind();
     RepHeader &h = p.hdr[rep];
     s.cs = h.cs;               // set-up works on the records in global memory
@@ -899,13 +905,14 @@ __global__ void __launch_bounds__(32) qsim_lane_init_kernel(Params p)
 }
 
 // Advance every replication to its new end time (or until the per-launch event budget runs out).
+template <uint32_t LF>
 __global__ void __launch_bounds__(32) qsim_lane_run_kernel(Params p)
 {
     const uint32_t rep = blockIdx.x * blockDim.x + threadIdx.x;
     if (rep >= p.R) return;
     RepHeader &h = p.hdr[rep];
     if (!p.advance && h.done) return;
-    LaneSim s(p, rep);
+    LaneSim<LF> s(p, rep);
     s.bind();
     // this lane's part of shared memory: class records (stride padded so that the lanes' 8-byte accesses fall into
     // different banks) and the calendar bitmap, word-interleaved over the lanes

@@ -68,6 +68,7 @@ struct qsim {
     int device = 0;
     void (*run_fn)(qsimdev::Params) = nullptr;
     uint32_t nwarps = 1;          // warps per replication (block size / 32)
+    void (*lane_fn)(qsimdev::Params) = nullptr;     // instance of the one-thread-per-replication run kernel
     bool allow_lane = true;       // the one-thread-per-replication family may run this handle
     double coef[6]{};
 };
@@ -302,7 +303,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
 void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
-    uint32_t W = rows >= 64 ? 16u : (rows >= 32 ? 4u : 1u);      // best of sweeps over 1, 2, 4, 8, 16 warps at 512, 1024, 4096 GPUs
+    uint32_t W = rows >= 128 ? 16u : (rows >= 32 ? 4u : 1u);     // best of sweeps over 1, 2, 4, 8, 16 warps at 512, 1024, 2048, 4096 GPUs
     if (const char *e = std::getenv("QSIM_WARPS")) {
         const int v = std::atoi(e);
         if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;
@@ -407,6 +408,14 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
         else if (std::strcmp(e, "warp") == 0) lane = false;
     }
     if (lane) {
+        // the smallest instance that contains the configuration's features
+        const bool ab = p.any_theta != 0, sli = cfg.router == QSIM_ROUTER_SLI, hist = cfg.hist != 0, blk = cfg.nblk > 1;
+        const char *force = std::getenv("QSIM_KERNEL");
+        if (force && std::strcmp(force, "generic") == 0) h.lane_fn = qsim_lane_run_kernel<LF_GENERIC>;
+        else if (!sli && !hist && !blk) h.lane_fn = ab ? qsim_lane_run_kernel<LF_ABANDON> : qsim_lane_run_kernel<0u>;
+        else if (sli && hist && !blk) h.lane_fn = qsim_lane_run_kernel<LF_ABANDON | LF_SLI | LF_HIST>;
+        else if (!sli && blk && hist) h.lane_fn = qsim_lane_run_kernel<LF_ABANDON | LF_BLOCKS | LF_HIST>;
+        else h.lane_fn = qsim_lane_run_kernel<LF_GENERIC>;       // (abandonment code with theta = 0 is inert, so it may be compiled in)
         lane_shapes(cfg, coef, p.lane);
         if (p.lane.smem_bytes > 227u * 1024u) return fail(QSIM_EINVAL, "class records and calendar do not fit shared memory");
         h.sec = lane_sections(cfg, p.lane);
@@ -448,7 +457,7 @@ int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
     p.force_dispatch = h->targets_changed ? 1u : 0u;
     h->targets_changed = false;
     CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    if (p.lane.on) qsim_lane_run_kernel<<<(h->cfg.R + 31u) / 32u, 32, p.lane.smem_bytes, h->stream>>>(p);
+    if (p.lane.on) h->lane_fn<<<(h->cfg.R + 31u) / 32u, 32, p.lane.smem_bytes, h->stream>>>(p);
     else h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
     CUDA_TRY(cudaGetLastError());
     h->launches++;
@@ -600,7 +609,7 @@ int qsim_create(qsim_t **out, const qsim_config *cfg, const qsim_class *classes,
     if (e == cudaSuccess) e = cudaMallocHost(&h->h_flag, 256);
     if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(h->run_fn));
     if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(qsim_init_kernel));
-    if (e == cudaSuccess) e = allow_large_smem(reinterpret_cast<const void *>(qsim_lane_run_kernel));
+    if (e == cudaSuccess && h->lane_fn) e = allow_large_smem(reinterpret_cast<const void *>(h->lane_fn));
     if (e != cudaSuccess) {
         std::string msg = std::string("device set-up failed: ") + cudaGetErrorString(e);
         qsim_destroy(h);
@@ -1117,7 +1126,7 @@ int qsim_simulate_waves(const qsim_config *cfg, const qsim_class *classes, const
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------------
-// qsim_simulate_static: the whole simulation with no device or pinned-memory allocation at all.
+// qsim_simulate_static: the whole simulation with no device or pinned-memory allocation (host temporaries only).
 // State, tables and the completion flag live in one file-scope device array.  Host code never uses the
 // array's name as a pointer: its device address is asked for once per device (cudaGetSymbolAddress).
 // ---------------------------------------------------------------------------------------------------
@@ -1126,6 +1135,8 @@ static __device__ __align__(256) unsigned char g_static_scratch[QSIM_STATIC_SCRA
 
 namespace {
 constexpr int kMaxDevices = 64;
+// device address of the array, per device; written by the first call on a device.  No lock: calls on one device must not
+// overlap anyway (they share the array), and two first calls would store the same address.
 void *g_static_ptr[kMaxDevices] = {};
 }  // namespace
 
