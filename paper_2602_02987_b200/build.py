@@ -9,7 +9,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libqsim.so")
 SOURCES = [os.path.join(CSRC, "qsim_lib.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "qsim_device.cuh"), os.path.join(CSRC, "qsim_ctmc.cuh"),
+DEPENDS = SOURCES + [os.path.join(CSRC, "qsim_device.cuh"), os.path.join(CSRC, "qsim_lane.cuh"), os.path.join(CSRC, "qsim_ctmc.cuh"),
                      os.path.join(ROOT, "include", "qsim.h")]
 
 NVCC_FLAGS = [

@@ -81,7 +81,8 @@ struct RepHeader {
     double T_end, T_reset;
     unsigned long long place_ord, events, H_total, rounds;
     uint32_t blk, done, err, force;    // force: the next event must be followed by a dispatch (targets were replaced)
-    double t_now, t_pad;               // time of the last event handled (one-thread-per-replication kernels)
+    double t_now;                      // time of the last event handled (one-thread-per-replication kernels)
+    uint32_t seq, chunks_left;         // launches that split the horizon into chunks: hand-over stamp of the last chunk done, chunks not started yet
     uint32_t dq_head0, dq_head1, dq_n0, dq_n1;
     unsigned long long sel_ord0, sel_ord1;   // class selections drawn so far in the solo / mixed pool (general SLI router)
     unsigned long long iters_mixed[32], iters_solo[32];
@@ -110,7 +111,7 @@ struct LanePar {
     uint32_t tlev, toff[6], tsize;   // eligibility trees: internal levels, offset of every level (0 = leaves) and entries per tree
     uint32_t b8, slev, soff[5], ssize;   // slot trees: leaves per GPU, internal levels, offsets of levels 1.. and nodes per GPU
     double inv_w;                // buckets per second
-    uint32_t cs_stride, smem_bytes;  // shared memory per lane for the class records (32-bit words) and per block of 32 lanes (bytes)
+    uint32_t cs_stride, smem_bytes;  // shared memory per lane for the class records (32-bit words) and per block of 1 << lsh lanes (bytes)
     LaneSrv *srv;                // [N] GPU records
     double *tarr;                // [N] arrival time of the request in prefill
     uint16_t *cal_head;          // [nbk] first GPU of every bucket
@@ -121,7 +122,7 @@ struct LanePar {
     SlotRec *srec;               // [N][B] request in each slot
     uint16_t *sfree;             // [N][B] entries at and above the GPU's decode count are its free slots
     uint32_t *pql;               // [I][qw] live bits of the prefill-queue positions
-    uint32_t qw, qw_pad;         // words per class in pql (a multiple of four)
+    uint32_t qw, lsh;            // words per class in pql (a multiple of four); a warp runs 1 << lsh replications in its first lanes
 };
 
 struct Params {
@@ -135,6 +136,7 @@ struct Params {
     const double *inject_t;      // injected arrivals (trace replay): times [n_inject], ascending
     const uint32_t *inject_job;  // [n_inject][3] = class, P, D
     uint32_t n_inject, force_dispatch;   // force_dispatch: the policy parameters changed since the last launch
+    uint32_t nchunk, launch_tag;         // nchunk > 1: the horizon of this launch is run in that many chunks per replication (see qsim_run_kernel)
     double T_abs;                // advance == 2: absolute end time of this run
     // workspace sections (all arrays are [R][...])
     RepHeader *hdr;
@@ -144,10 +146,12 @@ struct Params {
     QEntry *pq;                  // [R][I][qcap]
     QEntry *dq;                  // [R][2][qcap]
     uint32_t *hist_mem;          // [R][I][2][NBIN] or null
-    uint32_t *not_done;          // single counter: replications that stopped on the event budget
+    uint32_t *not_done;          // [0] replications that stopped on the event budget, [1] next (chunk, replication) unit to hand out,
+                                 // [2] set when a block gave up waiting for the chunk before its own
     uint32_t srv_bytes;
     uint32_t tarr_global;        // pf_tarr lives in tarr_g instead of shared memory
     double *tarr_g;              // [R][N]
+    uint32_t *pfjob_g;           // [R][N] packed request in prefill, with tarr_g
     LanePar lane;
 };
 
@@ -344,7 +348,8 @@ struct Sim {
     WarpClassStats *wcs;         // [nwarps][MAXI]
     // shared memory (lane-owned entries)
     double *tnext, *pf_tarr;               // pf_tarr: arrival time of the request in prefill (shared memory, or global memory on large clusters)
-    uint32_t *it, *nfin, *pfrem, *pfjob, *K, *Kpend;
+    uint32_t *it, *nfin, *pfjob, *K, *Kpend;
+    uint16_t *pfrem;             // prompt tokens still to prefill (0 = no request in prefill; lengths are at most 8192)
     uint16_t *ndec, *nact, *pfcur;
     uint16_t *sfin16;            // [Npad][B]  low 16 bits of each slot's finish iteration (f_slots)
     uint32_t *socc;              // [Npad][ceil(B/32)]  slot occupancy bits; bits past B are set for good
@@ -591,7 +596,7 @@ struct Sim {
     {
         // g is always inside the padded arrays; every field is read first so that calls over rows overlap
         const uint32_t nd = ndec[g];
-        const bool pf = (pfjob[g] >> 31) != 0;
+        const bool pf = pfrem[g] != 0;
         const bool mix = g < M;
         const uint32_t cap = (mix || pf) ? p.B - 1 : p.B;   // a mixed GPU keeps one slot for prefill
         const bool ok = want == WANT_PREFILL ? (mix && !pf && nd <= p.B - 1)
@@ -609,7 +614,7 @@ struct Sim {
             const uint32_t g = (k << 5) + (uint32_t)lane;
             const uint32_t nd = ndec[g];
             const bool mix = g < M;
-            const uint32_t cap = (mix || (pfjob[g] >> 31)) ? p.B - 1 : p.B;
+            const uint32_t cap = (mix || pfrem[g] != 0) ? p.B - 1 : p.B;
             const uint32_t key = (mix ? 0x40000000u : 0u) | (nd << 16) | g;
             best = min(best, (nd < cap && g < p.N) ? key : NONE32);
         }
@@ -840,7 +845,7 @@ struct Sim {
         idle_hint = NONE32;
         if (lane == (int)(g & 31u)) {
             pfjob[g] = e.pk | 0x80000000u;
-            pfrem[g] = job_P(e.pk);
+            pfrem[g] = (uint16_t)job_P(e.pk);
             pf_tarr[g] = e.t;
         }
         touch_server(g);
@@ -854,10 +859,10 @@ struct Sim {
     __device__ __forceinline__ void start_at(uint32_t g, double ts, bool act = true)
     {
         const unsigned long long tn = (unsigned long long)__double_as_longlong(tnext[g]);
-        const uint32_t nd = ndec[g], pj = pfjob[g], rem = pfrem[g], nf = nfin[g], it0 = it[g];
+        const uint32_t nd = ndec[g], rem = pfrem[g], nf = nfin[g], it0 = it[g];
         uint32_t Kg = 0;
         if (f_kappa()) Kg = K[g] + Kpend[g];
-        const bool has_pf = (pj >> 31) != 0;
+        const bool has_pf = rem != 0;
         const uint32_t pc = has_pf ? min(p.C, rem) : 0u;
         uint32_t fl = (nf == it0 + 1u) ? 0x4000u : 0u;
         if (pc > 0 && pc == rem) fl |= 0x8000u;
@@ -1088,7 +1093,7 @@ struct Sim {
                 if (nfin[g] == itg) flags |= 1u;
                 if (pc > 0) {
                     const uint32_t rem = pfrem[g] - pc;
-                    pfrem[g] = rem;
+                    pfrem[g] = (uint16_t)rem;
                     if (rem == 0) flags |= 2u;
                 }
                 pfcur[g] = 0;
@@ -1198,14 +1203,14 @@ struct Sim {
     __device__ __forceinline__ bool local_end(uint32_t g, double te, bool act = true, bool evt = false)
     {
         // straight-line: all fields are read first and the stores are predicated on `act` (see start_at)
-        const uint32_t it0 = it[g], na_raw = nact[g], pc = pfcur[g], nd = ndec[g], pj = pfjob[g], pr = pfrem[g], nf = nfin[g];
+        const uint32_t it0 = it[g], na_raw = nact[g], pc = pfcur[g], nd = ndec[g], pr = pfrem[g], nf = nfin[g];
         uint32_t K0 = 0, Kp = 0;
         if (f_kappa()) { K0 = K[g]; Kp = Kpend[g]; }
         const double tau = iter_time(p, pc, na_raw & 0x3fffu, K0, f_kappa());   // duration of the iteration that ends (the chain of its start)
         const uint32_t itg = it0 + 1u;
         const uint32_t rem = pr - pc;                       // prompt tokens left after this iteration's chunk
         const bool retire = (na_raw & 0x4000u) != 0;        // a decode finished: the GPU waits for retire_decodes
-        const bool has_pf = (pj >> 31) != 0;
+        const bool has_pf = rem != 0;                       // (the end of a prefill is never local: rem > 0 while one runs)
         const bool restart = !retire && !evt && (nd != 0 || has_pf);
         // restart at te with what the GPU holds now (requests placed meanwhile join here)
         const uint32_t Kend = K0 + (na_raw & 0x3fffu);
@@ -1216,7 +1221,7 @@ struct Sim {
         const double tau2 = iter_time(p, pc2, nd, Kg, f_kappa());
         if (act) {
             it[g] = itg;
-            if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] = rem; }
+            if (pc > 0) { it_mixed++; busy_mixed = __dadd_rn(busy_mixed, tau); pfrem[g] = (uint16_t)rem; }
             else        { it_solo++;  busy_solo = __dadd_rn(busy_solo, tau); }
             if (f_kappa()) { K[g] = restart ? Kg : Kend; if (restart) Kpend[g] = 0; }
             pfcur[g] = restart ? (uint16_t)pc2 : (uint16_t)0;
@@ -1521,8 +1526,9 @@ struct SmemLayout {
         off_pfcur, off_sfin16, off_socc, srv_bytes, off_touch, off_gate, off_cs, off_ring, off_strec, off_stte, off_pqh, off_wcs, off_cmd, off_res, total;
 };
 
-// tarr_global: the arrival times of the requests in prefill live in global memory (large clusters: shared memory is what
-// limits the resident replications there); I: classes (sizes the ring of arrival draws)
+// tarr_global: the arrival times and the job words of the requests in prefill (read once per finished prefill) live in
+// global memory (large clusters: shared memory is what limits the resident replications there); I: classes (sizes the
+// class records and the ring of arrival draws)
 __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uint32_t slots_smem, uint32_t nwarps, bool kappa,
                                                   bool tarr_global, uint32_t I)
 {
@@ -1532,13 +1538,13 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_tarr = o; if (!tarr_global) o += 8 * Npad;
     L.off_it = o; o += 4 * Npad;
     L.off_nfin = o; o += 4 * Npad;
-    L.off_pfrem = o; o += 4 * Npad;
-    L.off_pfjob = o; o += 4 * Npad;
+    L.off_pfjob = o; if (!tarr_global) o += 4 * Npad;
     L.off_K = o; if (kappa) o += 4 * Npad;        // KV-token counts exist only when the KV slope is on
     L.off_Kpend = o; if (kappa) o += 4 * Npad;
     L.off_ndec = o; o += 2 * Npad;
     L.off_nact = o; o += 2 * Npad;
     L.off_pfcur = o; o += 2 * Npad;
+    L.off_pfrem = o; o += 2 * Npad;
     o = (o + 15u) & ~15u;
     L.off_sfin16 = o; if (slots_smem) o += 2 * Npad * B;
     o = (o + 15u) & ~15u;
@@ -1549,7 +1555,7 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     o = (o + 7u) & ~7u;
     L.off_gate = o; o += (8 + 8 + 4) * MAXI;
     o = (o + 15u) & ~15u;
-    L.off_cs = o; o += (uint32_t)sizeof(ClassState) * MAXI;
+    L.off_cs = o; o += (uint32_t)sizeof(ClassState) * I;
     o = (o + 15u) & ~15u;
     L.off_ring = o; o += (uint32_t)sizeof(ADraw) * 32 * I;
     L.off_strec = o; o += (uint32_t)sizeof(SlotRec) * STAGE_CAP;
@@ -1557,9 +1563,9 @@ __host__ __device__ inline SmemLayout smem_layout(uint32_t Npad, uint32_t B, uin
     L.off_pqh = o; o += (uint32_t)sizeof(QEntry) * MAXI;
     L.off_wcs = o; o += (uint32_t)sizeof(WarpClassStats) * MAXI * nwarps;
     o = (o + 15u) & ~15u;
-    L.off_cmd = o; o += (uint32_t)sizeof(MwCmd);
+    L.off_cmd = o; if (nwarps > 1) o += (uint32_t)sizeof(MwCmd);        // master and helpers only
     o = (o + 15u) & ~15u;
-    L.off_res = o; o += (uint32_t)sizeof(MwRes) * MW_MAX;
+    L.off_res = o; if (nwarps > 1) o += (uint32_t)sizeof(MwRes) * MW_MAX;
     L.total = (o + 15u) & ~15u;
     return L;
 }
@@ -1571,8 +1577,8 @@ __device__ __forceinline__ void bind_pointers(Sim<SPL, F> &s, char *sm, const Sm
     s.pf_tarr = s.p.tarr_global ? s.p.tarr_g + (size_t)s.rep * s.p.N : reinterpret_cast<double *>(sm + L.off_tarr);
     s.it = reinterpret_cast<uint32_t *>(sm + L.off_it);
     s.nfin = reinterpret_cast<uint32_t *>(sm + L.off_nfin);
-    s.pfrem = reinterpret_cast<uint32_t *>(sm + L.off_pfrem);
-    s.pfjob = reinterpret_cast<uint32_t *>(sm + L.off_pfjob);
+    s.pfrem = reinterpret_cast<uint16_t *>(sm + L.off_pfrem);
+    s.pfjob = s.p.tarr_global ? s.p.pfjob_g + (size_t)s.rep * s.p.N : reinterpret_cast<uint32_t *>(sm + L.off_pfjob);
     s.K = reinterpret_cast<uint32_t *>(sm + L.off_K);
     s.Kpend = reinterpret_cast<uint32_t *>(sm + L.off_Kpend);
     s.ndec = reinterpret_cast<uint16_t *>(sm + L.off_ndec);
@@ -1623,7 +1629,9 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
             const uint32_t bw = (p.B + 31u) >> 5;
             for (uint32_t g = lane; g < p.Npad; g += 32) s.socc[g * bw + bw - 1] = ~0u << (p.B & 31u);
         }
-        if (lane < MAXI) {
+        if (p.tarr_global)
+            for (uint32_t g = lane; g < p.N; g += 32) { s.pf_tarr[g] = 0.0; s.pfjob[g] = 0; }
+        if (lane < (int)p.I) {
             ClassState &c = s.cs[lane];
             c.ta = dinf();
             AbClock *clk[3] = { &c.abp, &c.abd0, &c.abd1 };
@@ -1652,7 +1660,7 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
         for (uint32_t o = lane * 4; o < sizeof(RepHeader); o += 128)
             *reinterpret_cast<uint32_t *>(reinterpret_cast<char *>(&h) + o) = 0;
         __syncwarp();
-        if (lane < MAXI) h.cs[lane] = s.cs[lane];
+        if (lane < (int)p.I) h.cs[lane] = s.cs[lane];
         char *img = p.srv + (size_t)rep * p.srv_bytes;
         for (uint32_t o = lane * 16; o < L.srv_bytes; o += 512)
             *reinterpret_cast<uint4 *>(img + o) = *reinterpret_cast<const uint4 *>(sm + o);
@@ -1661,6 +1669,20 @@ __global__ void __launch_bounds__(32) qsim_init_kernel(Params p)
         __syncwarp();
     }
 }
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *a)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_u32(uint32_t *a, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(a), "r"(v) : "memory");
+}
+// A block waits this many times about a microsecond (minutes in all) for the chunk before its own before it gives up.
+// Another block is running that chunk, so the wait lasts one chunk at most.
+constexpr uint32_t CHUNK_SPIN_LIMIT = 1u << 28;
 
 // Advance replications to their new end time (or until the per-launch event budget runs out).
 template <int SPLT, uint32_t FT>
@@ -1676,9 +1698,63 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) |
     extern __shared__ __align__(16) char sm[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t nthr = blockDim.x;
-    for (uint32_t rep = blockIdx.x; rep < p.R; rep += gridDim.x) {
+    // With nchunk = K > 1 the grid is one block per resident slot and the work is R x K units (chunk c of replication r is
+    // unit c R + r), handed out in that order through a counter: replications outnumbering the slots then finish together
+    // instead of leaving a last, nearly empty wave.  Chunk c of a replication starts when chunk c - 1 has published its
+    // stamp; that unit was handed out earlier, so the block it waits for is running.  The chunks end at the times at
+    // which K successive launches would end, so the result is theirs: that of one launch, up to the order in which the
+    // fp64 sums of finished requests are added to the totals.
+    __shared__ uint32_t sh_unit[2];
+    const uint32_t K = p.nchunk > 1 ? p.nchunk : 1u;
+    const uint32_t n_units = p.R * K;
+    for (uint32_t unit = blockIdx.x;; unit += gridDim.x) {
+        if (K > 1) {
+            if (tid == 0) sh_unit[0] = atomicAdd(p.not_done + 1, 1u);
+            if (FT & F_MW) __syncthreads(); else __syncwarp();
+            unit = sh_unit[0];
+            if (FT & F_MW) __syncthreads(); else __syncwarp();
+        }
+        if (unit >= n_units) break;
+        const uint32_t rep = unit % p.R, chunk = unit / p.R;
         RepHeader &h = p.hdr[rep];
-        if (!p.advance && h.done) continue;
+        uint32_t advance = p.advance, chunks_left = 0;
+        unsigned long long horizon_iters = p.horizon_iters;
+        if (K > 1) {
+            if (tid == 0) {
+                uint32_t ok = 1;
+                if (chunk > 0) {
+                    const uint32_t want = p.launch_tag + chunk;
+                    for (uint32_t spins = 0; ld_acquire_u32(&h.seq) != want; ++spins) {
+                        if (spins > CHUNK_SPIN_LIMIT || ld_acquire_u32(p.not_done + 2) != 0) { ok = 0; break; }
+                        __nanosleep(1000);
+                    }
+                }
+                sh_unit[1] = ok;
+            }
+            if (FT & F_MW) __syncthreads(); else __syncwarp();
+            const uint32_t ok = sh_unit[1];
+            __threadfence();
+            if (FT & F_MW) __syncthreads(); else __syncwarp();
+            if (!ok) {      // the chunk before this one did not finish in time: report, start nothing
+                if (tid == 0) { atomicExch(p.not_done + 2, 1u); atomicAdd(p.not_done, 1u); }
+                continue;
+            }
+            const bool first = chunk == 0 && p.advance == 1;
+            chunks_left = first ? K : h.chunks_left;
+            bool idle = false;
+            if (!first && !h.done) advance = 0;                 // stopped on the event budget: go on to the same end time
+            else if (chunks_left > 0) {
+                const unsigned long long j = K - chunks_left;
+                horizon_iters = p.horizon_iters * (j + 1) / K - p.horizon_iters * j / K;
+                advance = 1;
+                --chunks_left;
+            } else idle = true;
+            if (idle) {
+                if (FT & F_MW) __syncthreads(); else __syncwarp();
+                if (tid == 0) st_release_u32(&h.seq, p.launch_tag + chunk + 1u);
+                continue;
+            }
+        } else if (!p.advance && h.done) continue;
         const SmemLayout L = smem_layout(p.Npad, p.B, p.slots_smem, nthr >> 5, p.coef[5] != 0.0, p.tarr_global != 0, p.I);
         Sim<SPLT, FT> s(p, lane, rep);
         s.warp = warp;
@@ -1692,16 +1768,16 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) |
         {
             const uint4 *src = reinterpret_cast<const uint4 *>(h.cs);
             uint4 *dst = reinterpret_cast<uint4 *>(s.cs);
-            for (uint32_t o = tid; o < sizeof(ClassState) * MAXI / 16; o += nthr) dst[o] = src[o];
+            for (uint32_t o = tid; o < sizeof(ClassState) * p.I / 16; o += nthr) dst[o] = src[o];
             uint32_t *w = reinterpret_cast<uint32_t *>(s.wcs);
             for (uint32_t o = tid; o < sizeof(WarpClassStats) * MAXI * (nthr >> 5) / 4; o += nthr) w[o] = 0;
         }
         s.block_sync();
         // the end time is one rounded product of the cumulative horizon: run(a); run(b) ends where run(a+b) ends
         double T_end = h.T_end;
-        const unsigned long long H_total = h.H_total + (p.advance == 1 ? p.horizon_iters : 0ull);
-        if (p.advance == 1) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
-        if (p.advance == 2) T_end = p.T_abs;
+        const unsigned long long H_total = h.H_total + (advance == 1 ? horizon_iters : 0ull);
+        if (advance == 1) T_end = __dmul_rn((double)H_total, iter_time(p, 0, p.B, 0));
+        if (advance == 2) T_end = p.T_abs;
         s.T_end = T_end;
         s.T_reset = h.T_reset;
         s.tau_min = fmin(p.coef[0], p.coef[3]);
@@ -1711,7 +1787,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) |
         s.place_ord = h.place_ord; s.events = h.events; s.rounds = h.rounds; s.sel_ord0 = h.sel_ord0; s.sel_ord1 = h.sel_ord1;
         s.n_touch = 0; s.touch_all = false; s.need_start = 0; s.err = h.err;
         s.drain_dirty = true; s.gate_dirty = true;
-        s.force_nonlocal = p.force_dispatch != 0 || h.force != 0;
+        s.force_nonlocal = (p.force_dispatch != 0 && chunk == 0) || h.force != 0;
         s.n_idle_pf = 0;
         s.idle_hint = NONE32;
         s.it_mixed = 0; s.it_solo = 0; s.busy_mixed = 0.0; s.busy_solo = 0.0;
@@ -1742,7 +1818,7 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) |
         {
             uint4 *dst = reinterpret_cast<uint4 *>(h.cs);
             const uint4 *src = reinterpret_cast<const uint4 *>(s.cs);
-            for (uint32_t o = tid; o < sizeof(ClassState) * MAXI / 16; o += nthr) dst[o] = src[o];
+            for (uint32_t o = tid; o < sizeof(ClassState) * p.I / 16; o += nthr) dst[o] = src[o];
         }
         // per-thread partial sums go to the 32 lane slots, warp after warp (a fixed order)
         for (int w = 0; w < s.nwarps; ++w) {
@@ -1765,7 +1841,15 @@ __global__ void __launch_bounds__((FT & F_MW) ? 32 * MW_MAX : 32, ((FT & F_MW) |
             h.sel_ord0 = s.sel_ord0; h.sel_ord1 = s.sel_ord1;
             h.done = finished ? 1u : 0u;
             h.force = s.force_nonlocal ? 1u : 0u;
-            if (!finished) atomicAdd(p.not_done, 1u);
+            if (K > 1) {
+                h.chunks_left = chunks_left;
+                if (chunk == K - 1u && (!finished || chunks_left > 0)) atomicAdd(p.not_done, 1u);
+            } else if (!finished) atomicAdd(p.not_done, 1u);
+        }
+        if (K > 1) {        // hand the replication over to the unit of its next chunk
+            __threadfence();
+            s.block_sync();
+            if (tid == 0) st_release_u32(&h.seq, p.launch_tag + chunk + 1u);
         }
         s.block_sync();
     }

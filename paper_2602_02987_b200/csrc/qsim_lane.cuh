@@ -288,7 +288,7 @@ struct LaneSim {
     __device__ __forceinline__ void cache_flush() { if (cg != NONE32) { srv[cg] = crec; cg = NONE32; } }
 
     // --- calendar of iteration ends ---------------------------------------------------------------------
-    __device__ __forceinline__ uint32_t &bm(uint32_t w) const { return sbm[(w << 5)]; }
+    __device__ __forceinline__ uint32_t &bm(uint32_t w) const { return sbm[(w << p.lane.lsh)]; }
     __device__ __forceinline__ uint32_t bucket_of(double x) const
     {
         return (uint32_t)__double2ull_rd(__dmul_rn(x, p.lane.inv_w)) & (p.lane.nbk - 1u);
@@ -908,8 +908,11 @@ __global__ void __launch_bounds__(32) qsim_lane_init_kernel(Params p)
 template <uint32_t LF>
 __global__ void __launch_bounds__(32) qsim_lane_run_kernel(Params p)
 {
-    const uint32_t rep = blockIdx.x * blockDim.x + threadIdx.x;
-    if (rep >= p.R) return;
+    // A block is one warp; its first 1 << lsh lanes run a replication each.  With few replications the host picks
+    // fewer lanes per warp: more warps run, and a warp waits for fewer lanes that took another branch.
+    const uint32_t lpw = 1u << p.lane.lsh;
+    const uint32_t rep = blockIdx.x * lpw + threadIdx.x;
+    if (threadIdx.x >= lpw || rep >= p.R) return;
     RepHeader &h = p.hdr[rep];
     if (!p.advance && h.done) return;
     LaneSim<LF> s(p, rep);
@@ -919,7 +922,7 @@ __global__ void __launch_bounds__(32) qsim_lane_run_kernel(Params p)
     extern __shared__ __align__(16) uint32_t lane_sm[];
     const LanePar &lq = p.lane;
     s.cs = reinterpret_cast<ClassState *>(lane_sm + (size_t)threadIdx.x * lq.cs_stride);
-    s.sbm = lane_sm + (size_t)blockDim.x * lq.cs_stride + threadIdx.x;
+    s.sbm = lane_sm + (size_t)lpw * lq.cs_stride + threadIdx.x;
     s.cg = NONE32;
     {
         const uint32_t *src = reinterpret_cast<const uint32_t *>(h.cs);

@@ -65,6 +65,10 @@ struct qsim {
     cudaStream_t stream = nullptr;
     bool bound = false;
     uint64_t launches = 0;
+    uint32_t resident_blocks = 0; // blocks of run_fn that one device holds at a time (0 = not asked yet)
+    uint32_t chunk_K = 1;         // chunks per replication of the launch in progress (see plan_chunks)
+    uint64_t chunk_H = 0;         // and its horizon
+    uint32_t tag_base = 0;        // hand-over stamps of this handle's launches start above every stamp in the workspace
     int device = 0;
     void (*run_fn)(qsimdev::Params) = nullptr;
     uint32_t nwarps = 1;          // warps per replication (block size / 32)
@@ -89,7 +93,7 @@ Sections layout_sections(const qsim_config &c, uint32_t srv_bytes, bool tarr_glo
     s.hist = o; if (c.hist) o = align256(o + R * (size_t)c.I * 2 * NBIN * 4);
     s.flag = o; o = align256(o + 256);
     s.red = o; o = align256(o + sizeof(TotalsRecBytes) + R * (size_t)(c.I * 7u + 3u) * 8);    // totals record + fp64 statistics per replication
-    s.tarr = o; if (tarr_global) o = align256(o + R * (size_t)c.N * 8);
+    s.tarr = o; if (tarr_global) o = align256(o + R * (size_t)c.N * 12);      // arrival time (8 bytes) and job word (4) of the request in prefill
     s.total = o;
     return s;
 }
@@ -164,12 +168,20 @@ void lane_shapes(const qsim_config &c, const double *coef, LanePar &q)
     for (uint32_t l = 0; l < q.slev; ++l) q.soff[l] = off[l + 1] - off[1];      // internal levels only: the leaves are a separate array
     q.ssize = size - off[1];
     q.qw = ((c.qcap + 127u) / 128u) * 4u;
-    // shared memory of a block of 32 lanes: per lane the class records, at a stride whose half is odd (the lanes' 8-byte
+    // replications per warp: 32 when there are enough of them for 512 warps, else 16 or 8 (measured at 1024 and 4096 GPUs
+    // with 4096 and 8192 replications: +12 % and +10 % over 32; 4 per warp is slower again); QSIM_LANE_LSH overrides (2..5)
+    q.lsh = 5;
+    while (q.lsh > 3 && (c.R >> q.lsh) < 512u) --q.lsh;
+    if (const char *e = std::getenv("QSIM_LANE_LSH")) {
+        const int v = std::atoi(e);
+        if (v >= 2 && v <= 5) q.lsh = (uint32_t)v;
+    }
+    // shared memory of a block: per lane the class records, at a stride whose half is odd (the lanes' 8-byte
     // accesses then fall into different banks), and one bit per calendar bucket
     uint32_t stride = c.I * (uint32_t)(sizeof(ClassState) / 4);
     if (((stride / 2u) & 1u) == 0) stride += 2u;
     q.cs_stride = stride;
-    q.smem_bytes = 32u * (stride * 4u + q.nbk / 8u);
+    q.smem_bytes = (1u << q.lsh) * (stride * 4u + q.nbk / 8u);
 }
 
 int validate(const qsim_config *cfg, const qsim_class *classes, const double *rates, const uint32_t *lengths,
@@ -387,13 +399,13 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     h.run_fn = v.fn;
     h.nwarps = 1;
     choose_multiwarp(cfg.N, feat, p, h.run_fn, h.nwarps);
-    // beyond four rows of GPUs shared memory limits the resident replications: the arrival times of the requests in
-    // prefill (read once per finished prefill) move to global memory
+    // beyond four rows of GPUs shared memory limits the resident replications: the arrival times and the job words of
+    // the requests in prefill (read once per finished prefill) move to global memory
     p.tarr_global = (p.Npad > 128u) ? 1u : 0u;
     h.lay = smem_layout(p.Npad, p.B, p.slots_smem, h.nwarps, kappa, p.tarr_global != 0, cfg.I);
     h.init_smem = smem_layout(p.Npad, p.B, p.slots_smem, 1, kappa, p.tarr_global != 0, cfg.I).total;
     p.srv_bytes = h.lay.srv_bytes;
-    if (h.lay.total > 227u * 1024u)
+    if (h.lay.total > 227u * 1024u - 64u)       // a few bytes of the block are the kernel's own
         return fail(QSIM_EINVAL, "N too large: per-replication GPU state does not fit shared memory");
     h.sec = layout_sections(cfg, p.srv_bytes, p.tarr_global != 0);
     for (int k = 0; k < 6; ++k) h.coef[k] = coef[k];
@@ -430,8 +442,10 @@ cudaError_t allow_large_smem(const void *fn)
 {
     int dev = 0, optin = 0;
     cudaError_t e = cudaGetDevice(&dev);
+    cudaFuncAttributes fa{};
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, optin);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, fn);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)fa.sharedSizeBytes);   // the kernel's static part counts too
     return e;
 }
 
@@ -448,6 +462,38 @@ void fill_blocks(BlockPar *blocks, const qsim_config &cfg, const double *rates, 
     }
 }
 
+// When the replications outnumber the blocks the device holds at a time, but not by much, a launch of one block per
+// replication ends with a nearly empty last wave.  Such a launch is run as K chunks of the horizon per replication by one
+// block per resident slot (qsim_run_kernel), with K the smallest count that fills the last wave to 97 % (chunks of at
+// least 32 iterations of horizon, at most 64 chunks).  QSIM_CHUNKS overrides the choice (1 = off).
+uint32_t plan_chunks(qsim *h, uint64_t horizon)
+{
+    if (h->par.lane.on) return 1;
+    if (h->resident_blocks == 0) {
+        int per_sm = 0, sms = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, reinterpret_cast<const void *>(h->run_fn), (int)(32 * h->nwarps), h->lay.total) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess || per_sm < 1 || sms < 1) {
+            cudaGetLastError();
+            return 1;
+        }
+        h->resident_blocks = (uint32_t)per_sm * (uint32_t)sms;
+    }
+    const uint64_t R = h->cfg.R, G = h->resident_blocks, max_K = std::min<uint64_t>(64, horizon / 32);
+    if (const char *e = std::getenv("QSIM_CHUNKS")) {
+        const long v = std::atol(e);
+        return (uint32_t)std::max<long>(1, std::min<long>(v, (long)std::max<uint64_t>(max_K, 1)));
+    }
+    if (R <= G || R * 64 >= (1ull << 32)) return 1;
+    auto fill = [&](uint64_t K) { return (double)(K * R) / (double)(((K * R + G - 1) / G) * G); };
+    if (fill(1) >= 0.95) return 1;
+    uint64_t best = 1;
+    for (uint64_t K = 2; K <= max_K; ++K) {
+        if (fill(K) > fill(best) + 1e-9) best = K;
+        if (fill(best) >= 0.97) break;
+    }
+    return (uint32_t)best;
+}
+
 int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
 {
     Params p = h->par;
@@ -456,12 +502,27 @@ int launch_run(qsim *h, uint32_t advance, uint64_t horizon, double T_abs = 0.0)
     p.T_abs = T_abs;
     p.force_dispatch = h->targets_changed ? 1u : 0u;
     h->targets_changed = false;
-    CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 4, h->stream));
-    if (p.lane.on) h->lane_fn<<<(h->cfg.R + 31u) / 32u, 32, p.lane.smem_bytes, h->stream>>>(p);
-    else h->run_fn<<<h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
-    CUDA_TRY(cudaGetLastError());
+    if (advance == 1) { h->chunk_K = plan_chunks(h, horizon); h->chunk_H = horizon; }
+    else if (advance == 2) h->chunk_K = 1;
+    // a launch that continues a chunked one (advance 0) keeps its chunks: every replication goes on where it stopped
+    p.nchunk = h->chunk_K;
+    if (p.nchunk > 1) p.horizon_iters = h->chunk_H;
     h->launches++;
-    CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 4, cudaMemcpyDeviceToHost, h->stream));
+    p.launch_tag = (h->tag_base + (uint32_t)h->launches) << 8;
+    CUDA_TRY(cudaMemsetAsync(p.not_done, 0, 12, h->stream));
+    if (p.lane.on) h->lane_fn<<<(h->cfg.R + (1u << p.lane.lsh) - 1u) >> p.lane.lsh, 32, p.lane.smem_bytes, h->stream>>>(p);
+    else h->run_fn<<<p.nchunk > 1 ? h->resident_blocks : h->cfg.R, 32 * h->nwarps, h->lay.total, h->stream>>>(p);
+    CUDA_TRY(cudaGetLastError());
+    CUDA_TRY(cudaMemcpyAsync(h->h_flag, p.not_done, 12, cudaMemcpyDeviceToHost, h->stream));
+    return QSIM_OK;
+}
+
+// After the stream has been synchronised: did every replication reach its end time (1), are more launches needed (0), or
+// did a block give up waiting for a chunk (error)?
+int launch_outcome(const qsim *h, bool &finished)
+{
+    if (h->h_flag[2] != 0) return fail(QSIM_ECUDA, "a block gave up waiting for the previous chunk of its replication; the state is not usable");
+    finished = h->h_flag[0] == 0;
     return QSIM_OK;
 }
 
@@ -653,6 +714,7 @@ static int attach_workspace(qsim_t *h, void *ws, size_t bytes, void *cuda_stream
     p.hist_mem = h->cfg.hist ? reinterpret_cast<uint32_t *>(base + h->sec.hist) : nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h->sec.flag);
     p.tarr_g = p.tarr_global ? reinterpret_cast<double *>(base + h->sec.tarr) : nullptr;
+    p.pfjob_g = p.tarr_global ? reinterpret_cast<uint32_t *>(base + h->sec.tarr + (size_t)h->cfg.R * h->cfg.N * 8) : nullptr;
     if (p.lane.on) {
         LanePar &q = p.lane;
         q.srv = reinterpret_cast<LaneSrv *>(base + h->sec.l_srv);
@@ -719,6 +781,10 @@ int qsim_bind_restore(qsim_t *h, void *ws, size_t bytes, void *cuda_stream)
     for (uint32_t r = 0; r < h->cfg.R; ++r)
         if (hdr[r].err != 0 || !(hdr[r].T_end >= 0.0) || !std::isfinite(hdr[r].T_end))
             return fail(QSIM_ESTATE, "the workspace does not hold a resumable state (replication " + std::to_string(r) + ")");
+    // hand-over stamps of chunked launches (qsim_run_kernel) must not repeat a stamp that the saved state still holds
+    uint32_t top = 0;
+    for (uint32_t r = 0; r < h->cfg.R; ++r) top = std::max(top, hdr[r].seq >> 8);
+    h->tag_base = top + 1u;
     const RepHeader &first = hdr[0];
     h->T_end_abs = first.T_end;
     h->bound = true;
@@ -734,7 +800,10 @@ int qsim_run(qsim_t *h, uint64_t horizon_iters)
     // a replication that used up its per-launch event budget is continued by further launches
     for (;;) {
         CUDA_TRY(cudaStreamSynchronize(h->stream));
-        if (*h->h_flag == 0) break;
+        bool finished = false;
+        rc = launch_outcome(h, finished);
+        if (rc != QSIM_OK) return rc;
+        if (finished) break;
         rc = launch_run(h, 0u, 0);
         if (rc != QSIM_OK) return rc;
     }
@@ -751,7 +820,10 @@ int qsim_run_until(qsim_t *h, double T)
     if (rc != QSIM_OK) return rc;
     for (;;) {
         CUDA_TRY(cudaStreamSynchronize(h->stream));
-        if (*h->h_flag == 0) break;
+        bool finished = false;
+        rc = launch_outcome(h, finished);
+        if (rc != QSIM_OK) return rc;
+        if (finished) break;
         rc = launch_run(h, 0u, 0);
         if (rc != QSIM_OK) return rc;
     }
@@ -1011,14 +1083,13 @@ int qsim_server_state(qsim_t *h, uint32_t r, uint32_t *n_dec, uint32_t *it, doub
     CUDA_TRY(cudaStreamSynchronize(h->stream));
     const double *tn = reinterpret_cast<const double *>(img.data() + h->lay.off_tnext);
     const uint32_t *itv = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_it);
-    const uint32_t *rem = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_pfrem);
-    const uint32_t *pj = reinterpret_cast<const uint32_t *>(img.data() + h->lay.off_pfjob);
+    const uint16_t *rem = reinterpret_cast<const uint16_t *>(img.data() + h->lay.off_pfrem);
     const uint16_t *nd = reinterpret_cast<const uint16_t *>(img.data() + h->lay.off_ndec);
     for (uint32_t g = 0; g < h->cfg.N; ++g) {
         if (n_dec) n_dec[g] = nd[g];
         if (it) it[g] = itv[g];
         if (t_next) t_next[g] = tn[g];
-        if (pf_rem) pf_rem[g] = (pj[g] >> 31) ? rem[g] : 0u;
+        if (pf_rem) pf_rem[g] = rem[g];
     }
     return QSIM_OK;
 }
@@ -1199,6 +1270,7 @@ extern "C" int qsim_simulate_static(const qsim_config *cfg, const qsim_class *cl
     p.hist_mem = nullptr;
     p.not_done = reinterpret_cast<uint32_t *>(base + h.sec.flag);
     p.tarr_g = p.tarr_global ? reinterpret_cast<double *>(base + h.sec.tarr) : nullptr;
+    p.pfjob_g = p.tarr_global ? reinterpret_cast<uint32_t *>(base + h.sec.tarr + (size_t)h.cfg.R * h.cfg.N * 8) : nullptr;
     CUDA_TRY(allow_large_smem(reinterpret_cast<const void *>(h.run_fn)));
     CUDA_TRY(allow_large_smem(reinterpret_cast<const void *>(qsim_init_kernel)));
     // the array keeps the previous call's contents: the init kernel rewrites every header and GPU image;
