@@ -148,8 +148,8 @@ int qsim_bind(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_stream);
  * Checkpoint / resume.  All state of the replications lives in the caller's workspace, so a checkpoint is a copy of
  * its first qsim_workspace_bytes bytes taken between calls (after qsim_run / qsim_run_until has returned), and a
  * resume is: qsim_create with the same arguments, copy the bytes into a [device] workspace, then this call in place of
- * qsim_bind.  Nothing is initialised; the next qsim_run continues where the checkpointed run stopped, with bit-identical
- * results [the time horizon of Eq. (21)-(23) composes: run(a); run(b) is run(a+b)].  Targets installed with
+ * qsim_bind.  Nothing is initialised; the next qsim_run continues where the checkpointed run stopped, with the results
+ * of an uninterrupted sequence of the same calls [the time horizon of Eq. (21)-(23) composes, see qsim_run].  Targets installed with
  * qsim_set_targets are part of the handle, not of the workspace: install them again.  QSIM_ESTATE if the bytes hold
  * no resumable state (some replication stopped on an internal error) or were saved by a handle of another configuration or
  * layout (a fingerprint of both is kept in the workspace).
@@ -160,7 +160,13 @@ int qsim_bind_restore(qsim_t *h, void *dev_workspace, size_t bytes, void *cuda_s
  * Advance every replication by horizon_iters more iterations of horizon [event-driven dynamics of
  * Section 2.3 under the policies of Sections 4-5]: the new end time is H * tau_ref, H the total horizon
  * requested so far and tau_ref = tau(0, B, 0) (one full solo iteration).  Events with time <= the new end
- * are processed.  Calls compose: run(a); run(b) leaves exactly the state of run(a + b).
+ * are processed.  Calls compose: run(a); run(b) leaves exactly the simulated state and the integer statistics of
+ * run(a + b); the fp64 sums over finished requests (areas of Y_m and Y_s, TPOT sums) are added to the totals once per
+ * launch in the warp-per-replication kernels, so there they agree up to the order of additions.  When the replications
+ * outnumber the blocks the device holds at a time by a small factor, a call runs its horizon in several chunks per
+ * replication inside one launch, with the result of as many successive calls (environment variable QSIM_CHUNKS=1
+ * turns that off, QSIM_CHUNKS=K asks for K chunks).  QSIM_ECUDA if a block of such a launch gave up waiting for the
+ * chunk before its own (the wait is bounded; the state is then unusable).
  * qsim_stats / qsim_sync wait for completion.
  */
 int qsim_run(qsim_t *h, uint64_t horizon_iters);
