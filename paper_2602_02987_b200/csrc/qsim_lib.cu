@@ -315,7 +315,7 @@ uint32_t features_of(const qsim_config &c, const qsim_class *cls, const double *
 void choose_multiwarp(uint32_t N, uint32_t feat, Params &p, RunKernel &fn, uint32_t &nwarps)
 {
     const uint32_t rows = (N + 31u) / 32u;
-    uint32_t W = rows >= 128 ? 16u : (rows >= 32 ? 4u : 1u);     // best of sweeps over 1, 2, 4, 8, 16 warps at 512, 1024, 2048, 4096 GPUs
+    uint32_t W = rows >= 128 ? 16u : (rows >= 64 ? 4u : (rows >= 32 ? 2u : 1u));     // best of sweeps over 1, 2, 4, 8, 16 warps at 512, 768, 1024, 2048, 4096 GPUs
     if (const char *e = std::getenv("QSIM_WARPS")) {
         const int v = std::atoi(e);
         if (v >= 1 && v <= MW_MAX) W = (uint32_t)v;

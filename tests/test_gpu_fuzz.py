@@ -89,7 +89,7 @@ def test_random_sizes_on_the_benchmark_feature_sets(seed):
 
 @pytest.mark.parametrize("recipe,N,B", [("cfg2", 1024, 100), ("cfg4", 2049, 17), ("cfg2", 2049, 33), ("cfg4", 1023, 256)])
 def test_sizes_around_the_warp_count_thresholds(recipe, N, B):
-    # 1024 GPUs = 32 rows (four warps per replication), 2049 = 65 rows (eight warps, last row holds one GPU)
+    # 1024 GPUs = 32 rows (two warps per replication, 1023 still one), 2049 = 65 rows (four warps, last row holds one GPU)
     from oracle import OracleSim
     from paper_2602_02987_b200 import QSim
     inp = getattr(presets, recipe)(N=N, R=2).with_(B=B, seed=N + B)

@@ -105,7 +105,7 @@ def test_prefill_backlog_with_the_sli_router_on_a_large_cluster():
     assert st["abandoned_p"].sum() > 1000
 
 
-@pytest.mark.parametrize("warps", [2, 8, 16])
+@pytest.mark.parametrize("warps", [2, 4, 8, 16])
 def test_every_warp_count_gives_the_same_trajectory(warps):
     # the number of warps per replication is a launch parameter, not part of the method
     for inp, H in ((presets.cfg4(N=640, R=2), 400), (presets.crowded("decode", N=530, R=2), 500),
@@ -114,8 +114,8 @@ def test_every_warp_count_gives_the_same_trajectory(warps):
 
 
 def test_one_warp_instances_agree_on_a_cluster_that_defaults_to_several_warps():
-    inp = presets.cfg2(N=512, R=2)
-    check(inp, 300, warps=1)
+    inp = presets.cfg2(N=1024, R=2)
+    check(inp, 200, warps=1)
 
 
 def test_handles_of_different_sizes_share_kernels():

@@ -140,3 +140,20 @@ def test_replications_per_warp_do_not_matter(make, horizon):
     for lsh in (2, 3, 4):
         got = run(inp, [horizon], QSIM_FAMILY="lane", QSIM_LANE_LSH=lsh)
         same(got, base, f"{inp.name}: {1 << lsh} replications per warp")
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_configurations_in_chunks_against_the_oracle(seed):
+    """The seeded random configurations of the fuzz test, run as launches of 3 and of 7 chunks per replication."""
+    from oracle import OracleSim
+    from test_gpu_fuzz import random_case
+    inp = random_case(40 + seed)
+    H = int(np.random.default_rng(seed).choice([300, 1500, 4000]))
+    o = OracleSim(inp)
+    o.run(H)
+    ref = o.stats()
+    ostate = [o.server_state(r) for r in range(inp.R)]
+    o.close()
+    for K in (3, 7):
+        got = run(inp, [H // 2, H - H // 2], states=inp.R, QSIM_FAMILY="warp", QSIM_CHUNKS=K)
+        same(got, (ref, ostate), f"{inp.name}: N={inp.N} B={inp.B} I={inp.I} router={inp.router}, {K} chunks")
