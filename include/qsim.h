@@ -281,6 +281,15 @@ int qsim_simulate_static(const qsim_config *cfg, const qsim_class *classes, cons
                          const qsim_targets *lp_targets, uint64_t horizon_iters, qsim_rep_stats *totals,
                          qsim_rep_stats *per_rep, void *cuda_stream);
 
+/*
+ * Environment variables (diagnostics and cross-checks; none of them changes a result beyond the order of fp64 additions,
+ * which the tests use): QSIM_FAMILY=warp|lane picks the kernel family (a warp, or a few warps, per replication; one
+ * thread per replication) where the configuration allows both; QSIM_WARPS=1..16 the warps per replication of the first;
+ * QSIM_LANE_LSH=2..5 the binary logarithm of the replications per warp of the second; QSIM_KERNEL=generic the kernel
+ * instance that reads every feature from its parameters; QSIM_CHUNKS, see qsim_run.  Read when a handle is created
+ * (QSIM_CHUNKS: at every qsim_run).
+ */
+
 /* Diagnostic: look-ahead rounds executed since the last reset, summed over replications (a round handles at
  * most one non-local event and every local iteration end before it).  Synchronises the stream. */
 int qsim_round_count(qsim_t *h, uint64_t *rounds);
