@@ -938,10 +938,8 @@ struct Sim {
                 if (g < p.N) start_if_needed(g);
             }
         } else {
-            for (uint32_t k = 0; k < n_touch; ++k) {
-                const uint32_t g = touch[k];
-                if (lane == (int)(g & 31u)) start_if_needed(g);
-            }
+            // one lane per touched GPU (a GPU noted twice is started by two lanes with the same result)
+            for (uint32_t k = (uint32_t)lane; k < n_touch; k += 32u) start_if_needed(touch[k]);
         }
         n_touch = 0;
         touch_all = false;
@@ -1132,7 +1130,7 @@ struct Sim {
                 c.tok_in_pf += P;                  // separate charging credits the prompt here, Eq. (23)
                 const double ttft = __dsub_rn(t, tarr);
                 c.sum_ttft = __dadd_rn(c.sum_ttft, ttft);
-                if (f_hist()) hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)]++;
+                if (f_hist()) atomicAdd(&hist[((size_t)i * 2 + 0) * NBIN + hist_bin(ttft)], 1u);
                 if (f_sli()) c.sli_ord++;
             }
             __syncwarp();   // every lane has read the finished job before its owner clears it
@@ -1268,13 +1266,12 @@ struct Sim {
     // This warp's share of the local iteration ends below the limit key, with their retirements.
     __device__ bool ends_share(unsigned long long lim_t, uint32_t lim_s, bool buffered)
     {
-        const unsigned long long INF = 0x7ff0000000000000ull;
         bool progressed = false;
         for (uint32_t k = (uint32_t)warp; k < n_rows(); k += (uint32_t)nwarps) {
             const uint32_t g = (k << 5) + (uint32_t)lane;
             const unsigned long long v = (unsigned long long)__double_as_longlong(tnext[g]);
             bool retire = false;
-            if (v < INF && is_local(g, buffered) && (v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s))) {
+            if ((v < lim_t || (v == lim_t && SRC_SERVER + g < lim_s)) && is_local(g, buffered)) {     // (the limit is finite)
                 retire = local_end(g, __longlong_as_double((long long)v));
                 progressed = true;
             }
