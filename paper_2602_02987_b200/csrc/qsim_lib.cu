@@ -411,13 +411,12 @@ int configure(qsim &h, const qsim_config &cfg, const qsim_class *classes, const 
     for (int k = 0; k < 6; ++k) h.coef[k] = coef[k];
     // Kernel family.  A replication advances at about the same rate on one thread whatever its cluster size, while the
     // warp-per-replication kernels slow down in proportion to the cluster (few replications fit on an SM and their
-    // master warp searches all rows).  Measured on a B200: from 1024 GPUs one thread per replication wins when R x N
-    // exceeds about 7 million (N = 1024 from R = 8192, N = 2048 from R = 4096, N = 4096 from R = 2048); below, where twelve
-    // one-warp replications fit on an SM, only from about 16 million (N = 512, R = 16384: 3.5e8 against 5.4e8 it/s).
-    // QSIM_FAMILY=lane / warp overrides.
+    // master warp searches all rows).  Measured on a B200: one thread per replication wins from 2048 GPUs when R x N
+    // exceeds about 7 million (N = 2048, R = 4096: 2.26e8 against 2.18e8 it/s; N = 4096, R = 4096: 2.1e8 against 5.3e7),
+    // and not below (N = 1024: 3.35e8 against 3.47e8 at R = 8192, 3.15e8 against 3.53e8 at R = 16384; N = 512,
+    // R = 16384: 3.5e8 against 7e8).  QSIM_FAMILY=lane / warp overrides.
     std::memset(&p.lane, 0, sizeof p.lane);
-    bool lane = h.allow_lane && lane_supports(cfg, coef) &&
-                (unsigned long long)cfg.R * cfg.N >= (cfg.N >= 1024u ? 7000000ull : 16000000ull);
+    bool lane = h.allow_lane && lane_supports(cfg, coef) && cfg.N >= 2048u && (unsigned long long)cfg.R * cfg.N >= 7000000ull;
     if (const char *e = std::getenv("QSIM_FAMILY")) {
         if (std::strcmp(e, "lane") == 0) lane = h.allow_lane && lane_supports(cfg, coef);
         else if (std::strcmp(e, "warp") == 0) lane = false;
