@@ -1106,7 +1106,14 @@ struct Sim {
         if (flags & 1u) {
             drain_dirty = true;
             gate_dirty = true;   // a promoted GPU at the cap may now take a prefill
-            recount_idle = true;
+            if (SPL > 0) {
+                recount_idle = true;
+            } else if (!(flags & 2u) && g < M && pfrem[g] == 0 && nd > p.B - 1 && ndec[g] <= p.B - 1) {
+                // Only g changed: its idle prefill slot counts again once its decodes fit under the mixed cap (a prefill
+                // that finishes in this event is counted below, with the decode count after the retirement).
+                n_idle_pf++;
+                idle_hint = (n_idle_pf == 1) ? g : NONE32;
+            }
         }
         if (flags & 2u) {
             // prefill finished: account, then hand the request to the decode stage
